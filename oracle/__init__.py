@@ -1,0 +1,161 @@
+"""CPU oracle for the DEFT gradient-selection path: TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes/numpy marshalling around ``deft_oracle.cpp`` (plain single-threaded
+C++, fp64 norms, sort-based selection, literal Algorithm 3 / Algorithm 4).  Only
+the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the CUDA library never does, and this package never imports the CUDA
+library.  No arithmetic of the method lives in this file: every function below
+only converts arguments and calls the C++ routine of the same name.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "deft_oracle.cpp")
+_LIB = os.path.join(_HERE, "libdeft_oracle.so")
+
+MODE_PAPER = 0
+MODE_EXACT = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(
+            ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared", _SRC, "-o", tmp]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_split_layers.restype = ctypes.c_int64
+        _lib.oracle_allocate_k.restype = ctypes.c_int64
+        _lib.oracle_rank_bin.restype = ctypes.c_int64
+        _lib.oracle_partition_optimum.restype = ctypes.c_double
+        _lib.oracle_select_rank.restype = ctypes.c_int64
+    return _lib
+
+
+def _p(a):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _i64(x):
+    return ctypes.c_int64(int(x))
+
+
+def split_layers(tensor_sizes, n_workers):
+    """Algorithm 2. Returns (layer_start[L+1] int64, layer_tensor[L] int32)."""
+    sizes = np.ascontiguousarray(tensor_sizes, dtype=np.int64)
+    cap = int(sizes.size) * int(n_workers)
+    start = np.zeros(cap + 1, dtype=np.int64)
+    tensor = np.zeros(cap, dtype=np.int32)
+    L = _load().oracle_split_layers(_p(sizes), _i64(sizes.size), _i64(n_workers), _p(start), _p(tensor), _i64(cap))
+    if L < 0:
+        raise ValueError("oracle_split_layers: invalid input")
+    return start[: L + 1].copy(), tensor[:L].copy()
+
+
+def accumulate(e, g):
+    """Algorithm 1 line 5, in place over ``e`` (fp32)."""
+    assert e.dtype == np.float32 and g.dtype == np.float32 and e.flags.c_contiguous and g.flags.c_contiguous
+    assert e.size == g.size
+    _load().oracle_accumulate(_p(e), _p(g), _i64(e.size))
+    return e
+
+
+def layer_norms(acc, layer_start):
+    """Per-layer L2 norms in fp64 (Section 4.2)."""
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    ls = np.ascontiguousarray(layer_start, dtype=np.int64)
+    norms = np.zeros(ls.size - 1, dtype=np.float64)
+    _load().oracle_layer_norms(_p(acc), _p(ls), _i64(ls.size - 1), _p(norms))
+    return norms
+
+
+def allocate_k(norms, layer_size, k, mode=MODE_EXACT):
+    """Algorithm 3. Returns (k_l int64[L], sum_k)."""
+    nr = np.ascontiguousarray(norms, dtype=np.float64)
+    sz = np.ascontiguousarray(layer_size, dtype=np.int64)
+    k_l = np.zeros(sz.size, dtype=np.int64)
+    s = ctypes.c_int64(0)
+    rc = _load().oracle_allocate_k(_p(nr), _p(sz), _i64(sz.size), _i64(k), _i64(mode), _p(k_l), ctypes.byref(s))
+    if rc != 0:
+        raise ValueError("oracle_allocate_k failed with %d" % rc)
+    return k_l, int(s.value)
+
+
+def partition(layer_size, k_l, n_workers):
+    """Algorithm 4 packing. Returns (bin_of_layer int32[L], bin_load float64[N])."""
+    sz = np.ascontiguousarray(layer_size, dtype=np.int64)
+    kl = np.ascontiguousarray(k_l, dtype=np.int64)
+    bins = np.zeros(sz.size, dtype=np.int32)
+    load = np.zeros(int(n_workers), dtype=np.float64)
+    _load().oracle_partition(_p(sz), _p(kl), _i64(sz.size), _i64(n_workers), _p(bins), _p(load))
+    return bins, load
+
+
+def rank_bin(iteration, rank, n_workers):
+    """Algorithm 4 lines 1-2."""
+    return int(_load().oracle_rank_bin(_i64(iteration), _i64(rank), _i64(n_workers)))
+
+
+def partition_optimum(cost, n_workers):
+    """Exhaustive minimum of the maximum bin load (tiny inputs only)."""
+    c = np.ascontiguousarray(cost, dtype=np.float64)
+    return float(_load().oracle_partition_optimum(_p(c), _i64(c.size), _i64(n_workers)))
+
+
+def select_layer(acc, st, end, k):
+    """Algorithm 5 on one layer: (values fp32[k], indices int64[k]), ascending index."""
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    val = np.zeros(int(k), dtype=np.float32)
+    idx = np.zeros(int(k), dtype=np.int64)
+    _load().oracle_select_layer(_p(acc), _i64(st), _i64(end), _i64(k), _p(val), _p(idx))
+    return val, idx
+
+
+def select_rank(acc, layer_start, k_l, my_layers):
+    """Algorithm 5 over a rank's layers (ascending ids)."""
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    ls = np.ascontiguousarray(layer_start, dtype=np.int64)
+    kl = np.ascontiguousarray(k_l, dtype=np.int64)
+    my = np.ascontiguousarray(my_layers, dtype=np.int32)
+    total = int(kl[my].sum()) if my.size else 0
+    val = np.zeros(total, dtype=np.float32)
+    idx = np.zeros(total, dtype=np.int64)
+    got = _load().oracle_select_rank(_p(acc), _p(ls), _p(kl), _p(my), _i64(my.size), _p(val), _p(idx))
+    assert got == total
+    return val, idx
+
+
+def topk(acc, k):
+    """Conventional full-vector Top-k (Section 3.1): Algorithm 5 with one layer."""
+    return select_layer(acc, 0, acc.size, k)
+
+
+def residual_update(acc, idx):
+    """Algorithm 1 lines 11-12, in place."""
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    ix = np.ascontiguousarray(idx, dtype=np.int64)
+    _load().oracle_residual_update(_p(acc), _p(ix), _i64(ix.size))
+    return acc
+
+
+def my_layers(bin_of_layer, iteration, rank, n_workers):
+    """Layer ids (ascending) whose bin is the one ``rank`` reads this iteration."""
+    b = rank_bin(iteration, rank, n_workers)
+    return np.nonzero(np.asarray(bin_of_layer) == b)[0].astype(np.int32)

@@ -1,0 +1,302 @@
+// DEFT gradient-selection oracle: TEST INFRASTRUCTURE, NOT THE PRODUCT.
+//
+// A plain, slow, single-threaded CPU statement of what the DEFT hot path
+// computes (Yoon & Oh, "DEFT: Exploiting Gradient Norm Difference between
+// Model Layers for Scalable Gradient Sparsification", ICPP 2023).  It is
+// used only by the tests, the smoke check and the benchmark's CPU-baseline
+// leg.  It shares no code, header, table or helper with the CUDA library
+// and neither side includes or links the other.
+//
+// Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared (no fast-math,
+// no FTZ/DAZ), so every fp64 operation below is one IEEE round-to-nearest
+// operation in the order written.
+//
+// Parity pins (all in tests/, run without a GPU): every function here is
+// pinned by closed forms, invariants, library routines, exact rational
+// arithmetic or brute force; none is "parity unpinned".
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <utility>
+#include <vector>
+
+extern "C" {
+
+// ---------------------------------------------------------------------------
+// Algorithm 2 (two-stage gradient vector partitioning), Section 4.1.
+// A tensor whose size exceeds n_g / n_workers is cut into n_workers
+// contiguous fragments; the first (size % n_workers) fragments hold one
+// element more than the quotient.  Every fragment and every unsplit tensor
+// is a "layer".  The comparison `size > n_g / N` is evaluated as
+// `size * N > n_g` in integers, which is the same predicate for real and
+// for floor division.  Fragments of size zero (only possible when a split
+// tensor has fewer elements than workers) are dropped.
+// Returns the number of layers L, or -1 if cap is too small / input invalid.
+// layer_start has L+1 entries, layer_tensor[l] is the source tensor id.
+// ---------------------------------------------------------------------------
+int64_t oracle_split_layers(const int64_t* tensor_sizes, int64_t T, int64_t n_workers,
+                            int64_t* layer_start, int32_t* layer_tensor, int64_t cap) {
+    if (T < 1 || n_workers < 1) return -1;
+    int64_t n_g = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        if (tensor_sizes[t] < 1) return -1;
+        n_g += tensor_sizes[t];
+    }
+    int64_t L = 0;
+    int64_t alloc_pos = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        const int64_t size = tensor_sizes[t];
+        if ((__int128)size * (__int128)n_workers > (__int128)n_g) {
+            const int64_t quotient = size / n_workers;
+            int64_t remainder = size % n_workers;
+            for (int64_t i = 0; i < n_workers; ++i) {
+                int64_t size_layer = quotient;
+                if (remainder > 0) {
+                    size_layer = size_layer + 1;
+                    remainder = remainder - 1;
+                }
+                if (size_layer == 0) continue;
+                if (L >= cap) return -1;
+                layer_start[L] = alloc_pos;
+                layer_tensor[L] = (int32_t)t;
+                alloc_pos = alloc_pos + size_layer;
+                ++L;
+            }
+        } else {
+            if (L >= cap) return -1;
+            layer_start[L] = alloc_pos;
+            layer_tensor[L] = (int32_t)t;
+            alloc_pos = alloc_pos + size;
+            ++L;
+        }
+    }
+    layer_start[L] = alloc_pos;
+    return L;
+}
+
+// ---------------------------------------------------------------------------
+// Algorithm 1, line 5: acc = e + eta*G.  The caller passes the already
+// scaled gradient, so this is one fp32 round-to-nearest add per element,
+// written over e.
+// ---------------------------------------------------------------------------
+void oracle_accumulate(float* e, const float* g, int64_t n_g) {
+    for (int64_t i = 0; i < n_g; ++i) {
+        volatile float s = e[i] + g[i];  // volatile: forces the fp32 rounding
+        e[i] = s;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Section 4.2: the gradient norm of each layer (L2, the paper's only stated
+// norm, Section 2).  norm_l = sqrt(sum_i acc_i^2), summed sequentially in
+// fp64 over the layer.
+// ---------------------------------------------------------------------------
+void oracle_layer_norms(const float* acc, const int64_t* layer_start, int64_t L, double* norms) {
+    for (int64_t l = 0; l < L; ++l) {
+        double s = 0.0;
+        for (int64_t i = layer_start[l]; i < layer_start[l + 1]; ++i) {
+            const double x = (double)acc[i];
+            s = s + x * x;
+        }
+        norms[l] = std::sqrt(s);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Algorithm 3 (gradient-norm-based local k assignment), Section 4.2.
+// Layers are visited in priority order (norm descending, equal norms by
+// lower layer id).  Each layer receives
+//     k_temp = floor(k_remain * (norm / norm_remain))   (0 if norm_remain <= 0)
+//     k_l    = size        if size < k_temp
+//              max(1, k_temp) otherwise
+// and k_remain is reduced by k_l.  norm_remain for the layer at priority
+// position p is the sum of the norms at positions p..L-1, accumulated from
+// the back (the same quantity the listing maintains by subtraction, without
+// its cancellation error; the last ratio is exactly 1).
+//
+// mode 0 (PAPER): stop there; sum k_l may differ from k.
+// mode 1 (EXACT): integer-only repair so that sum k_l == k.  Shortfall is
+//   handed out in priority order up to each layer's size; excess is taken
+//   back one element per layer per round, in priority order, never below 1.
+//   Needs L <= k <= n_g.
+// Returns 0 on success, -2 if EXACT is infeasible, -3 if a norm is not
+// finite or negative, -1 on other bad input.  k_l is indexed by layer id.
+// ---------------------------------------------------------------------------
+int64_t oracle_allocate_k(const double* norms, const int64_t* layer_size, int64_t L, int64_t k,
+                          int64_t mode, int64_t* k_l, int64_t* sum_k_out) {
+    if (L < 1 || k < 1) return -1;
+    int64_t n_g = 0;
+    for (int64_t l = 0; l < L; ++l) {
+        if (layer_size[l] < 1) return -1;
+        if (!std::isfinite(norms[l]) || norms[l] < 0.0) return -3;
+        n_g += layer_size[l];
+    }
+    if (mode == 1 && (k < L || k > n_g)) return -2;
+
+    // priority order
+    std::vector<int64_t> order(L);
+    for (int64_t l = 0; l < L; ++l) order[l] = l;
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int64_t a, int64_t b) { return norms[a] > norms[b]; });
+
+    // norm_remain at each priority position
+    std::vector<double> norm_remain(L + 1);
+    norm_remain[L] = 0.0;
+    for (int64_t p = L - 1; p >= 0; --p) norm_remain[p] = norms[order[p]] + norm_remain[p + 1];
+
+    int64_t k_remain = k;
+    for (int64_t p = 0; p < L; ++p) {
+        const int64_t l = order[p];
+        double k_temp;
+        if (norm_remain[p] > 0.0) {
+            const double ratio = norms[l] / norm_remain[p];
+            k_temp = std::floor((double)k_remain * ratio);
+        } else {
+            k_temp = 0.0;
+        }
+        int64_t kl;
+        if ((double)layer_size[l] < k_temp) {
+            kl = layer_size[l];
+        } else {
+            kl = (k_temp < 1.0) ? 1 : (int64_t)k_temp;
+        }
+        k_l[l] = kl;
+        k_remain = k_remain - kl;
+    }
+
+    if (mode == 1) {
+        int64_t sum = 0;
+        for (int64_t l = 0; l < L; ++l) sum += k_l[l];
+        int64_t rem = k - sum;
+        if (rem > 0) {
+            for (int64_t p = 0; p < L && rem > 0; ++p) {
+                const int64_t l = order[p];
+                int64_t add = layer_size[l] - k_l[l];
+                if (add > rem) add = rem;
+                k_l[l] += add;
+                rem -= add;
+            }
+        }
+        while (rem < 0) {
+            for (int64_t p = 0; p < L && rem < 0; ++p) {
+                const int64_t l = order[p];
+                if (k_l[l] > 1) {
+                    k_l[l] -= 1;
+                    rem += 1;
+                }
+            }
+        }
+    }
+    int64_t sum = 0;
+    for (int64_t l = 0; l < L; ++l) sum += k_l[l];
+    if (sum_k_out) *sum_k_out = sum;
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Algorithm 4 (bin-packing-based layer allocation), Section 4.3, Eq. 3.
+// cost_l = size_l * ln(k_l).  L times: take the layer of largest cost (first
+// occurrence), put it in the bin of smallest load (first occurrence), add
+// its cost to that bin, mark the layer with cost -1.  Layer ids are
+// positions in address order.
+// ---------------------------------------------------------------------------
+void oracle_partition(const int64_t* layer_size, const int64_t* k_l, int64_t L, int64_t n_workers,
+                      int32_t* bin_of_layer, double* size_bin /* n_workers */) {
+    std::vector<double> cost(L);
+    for (int64_t i = 0; i < L; ++i) cost[i] = (double)layer_size[i] * std::log((double)k_l[i]);
+    for (int64_t b = 0; b < n_workers; ++b) size_bin[b] = 0.0;
+    for (int64_t it = 0; it < L; ++it) {
+        int64_t idx_max = 0;
+        for (int64_t i = 1; i < L; ++i)
+            if (cost[i] > cost[idx_max]) idx_max = i;
+        const double val_max = cost[idx_max];
+        int64_t bin_min = 0;
+        for (int64_t b = 1; b < n_workers; ++b)
+            if (size_bin[b] < size_bin[bin_min]) bin_min = b;
+        bin_of_layer[idx_max] = (int32_t)bin_min;
+        size_bin[bin_min] = size_bin[bin_min] + val_max;
+        cost[idx_max] = -1.0;
+    }
+}
+
+// Algorithm 4, lines 1-2: the bin a rank reads in a given iteration.
+int64_t oracle_rank_bin(int64_t iteration, int64_t rank, int64_t n_workers) {
+    const int64_t cycle = iteration % n_workers;
+    return (cycle + rank) % n_workers;
+}
+
+// Smallest possible maximum bin load (Eq. 5 minimised over all n_workers^L
+// assignments), by exhaustive enumeration.  For tiny inputs only.
+double oracle_partition_optimum(const double* cost, int64_t L, int64_t n_workers) {
+    std::vector<int64_t> assign(L, 0);
+    std::vector<double> load(n_workers);
+    double best = -1.0;
+    for (;;) {
+        for (int64_t b = 0; b < n_workers; ++b) load[b] = 0.0;
+        for (int64_t i = 0; i < L; ++i) load[assign[i]] += cost[i];
+        double mx = 0.0;
+        for (int64_t b = 0; b < n_workers; ++b) mx = std::max(mx, load[b]);
+        if (best < 0.0 || mx < best) best = mx;
+        int64_t i = 0;
+        while (i < L) {
+            if (++assign[i] < n_workers) break;
+            assign[i] = 0;
+            ++i;
+        }
+        if (i == L) break;
+    }
+    return best;
+}
+
+// ---------------------------------------------------------------------------
+// Algorithm 5 (layer-wise gradient selection), Section 4.4: topk(|acc|, k)
+// on one layer [st, end).  Magnitudes are compared as the IEEE bit pattern
+// with the sign bit cleared; equal magnitudes are won by the lower index.
+// Output: the k selected entries in ascending index, as signed values and
+// int64 global indices.  Definition written out: sort everything.
+// ---------------------------------------------------------------------------
+void oracle_select_layer(const float* acc, int64_t st, int64_t end, int64_t k,
+                         float* val_out, int64_t* idx_out) {
+    const int64_t n = end - st;
+    std::vector<std::pair<uint32_t, int64_t>> items(n);
+    for (int64_t i = 0; i < n; ++i) {
+        uint32_t bits;
+        std::memcpy(&bits, &acc[st + i], 4);
+        items[i] = std::make_pair(bits & 0x7fffffffu, st + i);
+    }
+    std::sort(items.begin(), items.end(),
+              [](const std::pair<uint32_t, int64_t>& a, const std::pair<uint32_t, int64_t>& b) {
+                  if (a.first != b.first) return a.first > b.first;
+                  return a.second < b.second;
+              });
+    std::vector<int64_t> chosen(k);
+    for (int64_t j = 0; j < k; ++j) chosen[j] = items[j].second;
+    std::sort(chosen.begin(), chosen.end());
+    for (int64_t j = 0; j < k; ++j) {
+        idx_out[j] = chosen[j];
+        val_out[j] = acc[chosen[j]];
+    }
+}
+
+// Algorithm 5 over a rank's allocated layers (ascending layer ids): the
+// per-layer results concatenated.  Returns the rank's k (sum of k_l).
+int64_t oracle_select_rank(const float* acc, const int64_t* layer_start, const int64_t* k_l,
+                           const int32_t* my_layers, int64_t n_my, float* val_out,
+                           int64_t* idx_out) {
+    int64_t k = 0;
+    for (int64_t j = 0; j < n_my; ++j) {
+        const int64_t part = my_layers[j];
+        oracle_select_layer(acc, layer_start[part], layer_start[part + 1], k_l[part], val_out + k,
+                            idx_out + k);
+        k = k + k_l[part];
+    }
+    return k;
+}
+
+// Algorithm 1, lines 11-12: acc[idx] = 0; the buffer then is e_{t+1}.
+void oracle_residual_update(float* acc, const int64_t* idx, int64_t count) {
+    for (int64_t j = 0; j < count; ++j) acc[idx[j]] = 0.0f;
+}
+
+}  // extern "C"

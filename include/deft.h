@@ -1,0 +1,194 @@
+/*
+ * libdeft — the gradient-selection hot path of DEFT (Yoon & Oh, "DEFT: Exploiting
+ * Gradient Norm Difference between Model Layers for Scalable Gradient
+ * Sparsification", ICPP 2023) for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only.  Pointer names end in `_h` (host memory)
+ * or `_d` (device memory of the current CUDA device).  The library never allocates
+ * or frees device memory: the caller owns every buffer, including the workspace
+ * sized by deft_workspace_bytes().  Host calls are pure functions, thread-safe,
+ * and touch no CUDA state.  Device calls enqueue work on `stream` (a cudaStream_t
+ * passed as void*; NULL is the legacy default stream) and return without waiting;
+ * results are valid once the stream has reached that point.
+ *
+ * Every call returns a deft_status: 0 = DEFT_OK, > 0 a warning (results valid),
+ * < 0 an error (outputs unspecified unless stated).  Nothing throws or aborts.
+ *
+ * Vocabulary (Section 4 of the paper): the flat gradient vector has n_g elements;
+ * Algorithm 2 cuts it into L contiguous "layers"; `layer_start[L+1]` holds their
+ * boundaries in address order and a layer id is a position in that table; N is the
+ * number of workers; k = d * n_g gradients are selected per step, k_l of them in
+ * layer l.  One call of deft_select() does the work of ONE worker (rank).
+ */
+#ifndef DEFT_H_
+#define DEFT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Every entry point is exported with default visibility; nothing else leaves the library. */
+#if defined(__GNUC__)
+#define DEFT_API __attribute__((visibility("default")))
+#else
+#define DEFT_API
+#endif
+
+typedef int32_t deft_status;
+
+#define DEFT_OK                   0
+#define DEFT_WARN_K_INEXACT       1   /* PAPER mode only: sum of k_l differs from k              */
+#define DEFT_ERR_INVALID_ARG     -1   /* null pointer, non-positive size, unsorted table, ...    */
+#define DEFT_ERR_INFEASIBLE_K    -2   /* EXACT mode needs L <= k <= n_g                          */
+#define DEFT_ERR_NONFINITE_NORM  -3   /* a norm is NaN, infinite or negative; nothing written    */
+#define DEFT_ERR_CAPACITY        -4   /* an output buffer or the workspace is too small          */
+#define DEFT_ERR_CUDA            -5   /* a CUDA call failed; see deft_last_cuda_error()          */
+
+#define DEFT_MODE_PAPER 0  /* Algorithm 3 exactly as listed                                      */
+#define DEFT_MODE_EXACT 1  /* Algorithm 3 followed by an integer repair so that sum k_l == k     */
+
+/* Largest layer (and largest n for deft_topk_baseline) the selection kernels accept. */
+#define DEFT_MAX_LAYER_ELEMS 2147483647LL
+
+/* Human-readable name of a status code (static string). */
+DEFT_API const char* deft_status_string(deft_status s);
+
+/* The cudaError_t value behind the calling thread's most recent DEFT_ERR_CUDA (0 if none). */
+DEFT_API int32_t deft_last_cuda_error(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Host planners (cheap, O(L) .. O(L^2); run on the CPU as in the paper)
+ * ---------------------------------------------------------------------------------------- */
+
+/*
+ * Two-stage gradient vector partitioning — Algorithm 2, Section 4.1.
+ * A tensor with size > n_g / N (tested as size * N > n_g) is cut into N contiguous
+ * fragments of floor(size/N) elements, the first size % N of them one larger; all
+ * other tensors stay whole.  Fragments and whole tensors are the "layers".  A
+ * fragment that would be empty (size < N) is dropped.
+ *   tensor_sizes_h[T]   in   element count of each tensor in address order, each >= 1
+ *   layer_start_h[cap+1] out boundaries: layer l is [layer_start[l], layer_start[l+1])
+ *   layer_tensor_h[cap] out  source tensor of each layer (may be NULL)
+ *   L_out               out  number of layers
+ * Errors: INVALID_ARG (null, T < 1, N < 1, a size < 1), CAPACITY (cap too small;
+ * *L_out then holds the required count).
+ */
+DEFT_API deft_status deft_split_layers(const int64_t* tensor_sizes_h, int32_t T, int32_t N,
+                              int64_t* layer_start_h, int32_t* layer_tensor_h, int32_t cap,
+                              int32_t* L_out);
+
+/*
+ * Gradient-norm-based local k assignment — Algorithm 3, Section 4.2.
+ * Layers are visited by descending norm (equal norms: lower id first).  With
+ * norm_remain = the sum of the norms not yet visited (accumulated from the back,
+ * so the last ratio is exactly 1) and k_remain = k minus what was handed out:
+ *     k_temp = floor(k_remain * (norm_l / norm_remain))      (0 if norm_remain <= 0)
+ *     k_l    = size_l if size_l < k_temp, else max(1, k_temp)
+ * All of it in IEEE fp64 / int64, in exactly this operation order.
+ * DEFT_MODE_PAPER stops there and returns DEFT_WARN_K_INEXACT when sum k_l != k
+ * (the listing guarantees only "approximately k").  DEFT_MODE_EXACT then repairs the
+ * sum with integers only: a shortfall is handed out in priority order up to each
+ * layer's size; a surplus is taken back one per layer per round in priority order,
+ * never below 1.
+ *   norms_h[L], layer_size_h[L] in;  k_l_h[L] out (by layer id);  sum_k_out out (may be NULL)
+ * Errors: INVALID_ARG, NONFINITE_NORM, INFEASIBLE_K (EXACT with k < L or k > n_g).
+ */
+DEFT_API deft_status deft_allocate_k(const double* norms_h, const int64_t* layer_size_h, int32_t L,
+                            int64_t k, int32_t mode, int64_t* k_l_h, int64_t* sum_k_out);
+
+/*
+ * Bin-packing-based layer allocation — Algorithm 4, Section 4.3, Eq. 3.
+ * cost_l = size_l * ln(k_l).  L times: the layer of largest remaining cost (lowest id
+ * on ties) goes to the bin of smallest load (lowest id on ties).
+ *   bin_of_layer_h[L] out  bin of each layer
+ *   bin_load_h[N]     out  summed cost per bin (Eq. 4); may be NULL
+ * Errors: INVALID_ARG (null, L < 1, N < 1, a size < 1, a k_l < 1).
+ */
+DEFT_API deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L,
+                           int32_t N, int32_t* bin_of_layer_h, double* bin_load_h);
+
+/*
+ * Which bin a rank reads in a given iteration — Algorithm 4, lines 1-2:
+ * (iteration % N + rank) % N.  Returns -1 on invalid arguments.
+ */
+DEFT_API int32_t deft_rank_bin(int64_t iteration, int32_t rank, int32_t N);
+
+/*
+ * The layer ids of one bin, ascending (alloc_part of Algorithm 4, line 20).
+ *   my_layers_h[cap] out, n_my_out out.  Errors: INVALID_ARG, CAPACITY.
+ */
+DEFT_API deft_status deft_bin_layers(const int32_t* bin_of_layer_h, int32_t L, int32_t bin,
+                            int32_t* my_layers_h, int32_t cap, int32_t* n_my_out);
+
+/* ------------------------------------------------------------------------------------------
+ * Device calls
+ * ---------------------------------------------------------------------------------------- */
+
+/*
+ * Workspace size in bytes that is enough for every device call below on vectors of
+ * up to max_elems elements cut into up to max_layers layers.  The workspace must be
+ * 256-byte aligned; its contents need not be preserved between calls.  Calls that
+ * share a workspace must not overlap on the GPU.
+ */
+DEFT_API size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers);
+
+/*
+ * Error-feedback accumulate fused with the per-layer gradient norms —
+ * Algorithm 1 line 5 and the per-layer L2 norm that Section 4.2 ranks layers by.
+ *   resid_acc_d[n_g]  in/out  on entry the local error e; on exit acc = e + grad
+ *                             (one fp32 round-to-nearest add per element; the caller
+ *                             passes the gradient already scaled by the learning rate)
+ *   grad_d[n_g]       in      may be NULL: then nothing is written and the norms are
+ *                             those of resid_acc_d as it stands
+ *   layer_start_d[L+1] in     DEVICE copy of the layer table (int64, ascending)
+ *   norms_d[L]        out     DEVICE, fp64: sqrt(sum of acc_i^2) per layer; squares are
+ *                             summed in fp32 over runs of 8 elements and in fp64 beyond,
+ *                             in a fixed order (bit-identical from run to run)
+ * resid_acc_d and grad_d must be 16-byte aligned.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+DEFT_API deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_g,
+                             const int64_t* layer_start_d, int32_t L, double* norms_d,
+                             void* ws_d, size_t ws_bytes, void* stream);
+
+/*
+ * Layer-wise gradient selection for ONE worker — Algorithm 5, Section 4.4.
+ * For each layer l in my_layers_h (ascending ids) selects the k_l entries of largest
+ * magnitude.  Magnitudes compare as the IEEE-754 bit pattern with the sign cleared
+ * (so NaN > Inf > finite, denormals are not flushed); equal magnitudes are won by the
+ * lower index.  Output: the selected entries of all those layers in ascending global
+ * index — signed values and int64 indices — exactly sum of k_l of them.
+ *   acc_d             in   the accumulated vector (16-byte aligned); not modified
+ *   layer_start_h[L+1], k_l_h[L]   HOST tables for the whole model
+ *   my_layers_h[n_my] HOST, ascending; n_my may be 0 (nothing is written)
+ *   val_d, idx_d      out  DEVICE buffers of out_cap entries
+ * Errors: INVALID_ARG (null, ids not ascending, k_l outside [1, size_l], a layer
+ * larger than DEFT_MAX_LAYER_ELEMS), CAPACITY (out_cap < sum k_l, or ws too small), CUDA.
+ */
+DEFT_API deft_status deft_select(const float* acc_d, const int64_t* layer_start_h, const int64_t* k_l_h,
+                        const int32_t* my_layers_h, int32_t n_my, float* val_d, int64_t* idx_d,
+                        int64_t out_cap, void* ws_d, size_t ws_bytes, void* stream);
+
+/*
+ * Residual update — Algorithm 1 lines 11-12: acc[idx[j]] = +0.0f for j < count; the
+ * buffer is then the next step's local error.  Indices must be distinct and < n_g.
+ *   idx_d[count] DEVICE.  count may be 0.  Errors: INVALID_ARG, CUDA.
+ */
+DEFT_API deft_status deft_residual_update(float* acc_d, int64_t n_g, const int64_t* idx_d, int64_t count,
+                                 void* stream);
+
+/*
+ * Conventional Top-k over the whole vector — the comparison sparsifier of Sections 1
+ * and 3.1: the k entries of largest magnitude among acc_d[0..n), same ordering, tie
+ * rule and output format as deft_select (it is deft_select with a single layer).
+ * Errors: INVALID_ARG (k outside [1, n], n > DEFT_MAX_LAYER_ELEMS), CAPACITY, CUDA.
+ */
+DEFT_API deft_status deft_topk_baseline(const float* acc_d, int64_t n, int64_t k, float* val_d,
+                               int64_t* idx_d, void* ws_d, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEFT_H_ */

@@ -1,0 +1,192 @@
+// Host-side planners of libdeft: Algorithm 2 (layer table), Algorithm 3 (local k),
+// Algorithm 4 (bin packing) of the DEFT paper.  Pure functions, no CUDA.
+// Compiled with -ffp-contract=off: every fp64 operation is a single IEEE operation.
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <numeric>
+#include <vector>
+
+#include "deft.h"
+
+extern "C" {
+
+const char* deft_status_string(deft_status s) {
+    switch (s) {
+        case DEFT_OK: return "DEFT_OK";
+        case DEFT_WARN_K_INEXACT: return "DEFT_WARN_K_INEXACT";
+        case DEFT_ERR_INVALID_ARG: return "DEFT_ERR_INVALID_ARG";
+        case DEFT_ERR_INFEASIBLE_K: return "DEFT_ERR_INFEASIBLE_K";
+        case DEFT_ERR_NONFINITE_NORM: return "DEFT_ERR_NONFINITE_NORM";
+        case DEFT_ERR_CAPACITY: return "DEFT_ERR_CAPACITY";
+        case DEFT_ERR_CUDA: return "DEFT_ERR_CUDA";
+        default: return "DEFT_UNKNOWN_STATUS";
+    }
+}
+
+// Algorithm 2.
+deft_status deft_split_layers(const int64_t* tensor_sizes_h, int32_t T, int32_t N,
+                              int64_t* layer_start_h, int32_t* layer_tensor_h, int32_t cap,
+                              int32_t* L_out) {
+    if (!tensor_sizes_h || !layer_start_h || !L_out || T < 1 || N < 1 || cap < 0)
+        return DEFT_ERR_INVALID_ARG;
+    unsigned __int128 total = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        if (tensor_sizes_h[t] < 1) return DEFT_ERR_INVALID_ARG;
+        total += (unsigned __int128)tensor_sizes_h[t];
+    }
+    // First pass: count the layers so that a short buffer is reported, not overrun.
+    int64_t need = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t sz = tensor_sizes_h[t];
+        const bool split = (unsigned __int128)sz * (unsigned __int128)N > total;
+        need += split ? std::min<int64_t>(sz, N) : 1;
+    }
+    if (need > INT32_MAX) return DEFT_ERR_INVALID_ARG;
+    *L_out = (int32_t)need;
+    if (need > cap) return DEFT_ERR_CAPACITY;
+
+    int32_t l = 0;
+    int64_t pos = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t sz = tensor_sizes_h[t];
+        const bool split = (unsigned __int128)sz * (unsigned __int128)N > total;
+        const int64_t pieces = split ? N : 1;
+        const int64_t base = sz / pieces;
+        const int64_t extra = sz % pieces;  // the first `extra` pieces are one longer
+        for (int64_t i = 0; i < pieces; ++i) {
+            const int64_t len = base + (i < extra ? 1 : 0);
+            if (len == 0) continue;
+            layer_start_h[l] = pos;
+            if (layer_tensor_h) layer_tensor_h[l] = t;
+            pos += len;
+            ++l;
+        }
+    }
+    layer_start_h[l] = pos;
+    return DEFT_OK;
+}
+
+// Algorithm 3.
+deft_status deft_allocate_k(const double* norms_h, const int64_t* layer_size_h, int32_t L,
+                            int64_t k, int32_t mode, int64_t* k_l_h, int64_t* sum_k_out) {
+    if (!norms_h || !layer_size_h || !k_l_h || L < 1 || k < 1 ||
+        (mode != DEFT_MODE_PAPER && mode != DEFT_MODE_EXACT))
+        return DEFT_ERR_INVALID_ARG;
+    int64_t n_g = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        if (layer_size_h[l] < 1) return DEFT_ERR_INVALID_ARG;
+        n_g += layer_size_h[l];
+    }
+    for (int32_t l = 0; l < L; ++l)
+        if (!(norms_h[l] >= 0.0) || std::isinf(norms_h[l])) return DEFT_ERR_NONFINITE_NORM;
+    if (mode == DEFT_MODE_EXACT && (k < (int64_t)L || k > n_g)) return DEFT_ERR_INFEASIBLE_K;
+
+    // Priority: larger norm first, equal norms by lower id.
+    std::vector<int32_t> prio(L);
+    std::iota(prio.begin(), prio.end(), 0);
+    std::sort(prio.begin(), prio.end(), [norms_h](int32_t a, int32_t b) {
+        if (norms_h[a] != norms_h[b]) return norms_h[a] > norms_h[b];
+        return a < b;
+    });
+
+    // tail[p] = norms of priority positions p, p+1, ..., L-1 added from the back.
+    std::vector<double> tail((size_t)L + 1);
+    tail[L] = 0.0;
+    for (int32_t p = L; p-- > 0;) tail[p] = norms_h[prio[p]] + tail[p + 1];
+
+    int64_t left = k;
+    for (int32_t p = 0; p < L; ++p) {
+        const int32_t l = prio[p];
+        double want = 0.0;
+        if (tail[p] > 0.0) {
+            const double share = norms_h[l] / tail[p];
+            const double prod = (double)left * share;
+            want = std::floor(prod);
+        }
+        const int64_t sz = layer_size_h[l];
+        int64_t give;
+        if ((double)sz < want) give = sz;
+        else if (want < 1.0) give = 1;
+        else give = (int64_t)want;
+        k_l_h[l] = give;
+        left -= give;
+    }
+
+    int64_t sum = k - left;
+    if (mode == DEFT_MODE_EXACT && sum != k) {
+        int64_t gap = k - sum;  // > 0: hand out more; < 0: take back
+        if (gap > 0) {
+            for (int32_t p = 0; p < L && gap > 0; ++p) {
+                const int32_t l = prio[p];
+                const int64_t room = layer_size_h[l] - k_l_h[l];
+                const int64_t add = room < gap ? room : gap;
+                k_l_h[l] += add;
+                gap -= add;
+            }
+        } else {
+            while (gap < 0) {
+                for (int32_t p = 0; p < L && gap < 0; ++p) {
+                    const int32_t l = prio[p];
+                    if (k_l_h[l] > 1) {
+                        --k_l_h[l];
+                        ++gap;
+                    }
+                }
+            }
+        }
+        sum = k;
+    }
+    if (sum_k_out) *sum_k_out = sum;
+    return (sum == k) ? DEFT_OK : DEFT_WARN_K_INEXACT;
+}
+
+// Algorithm 4 (packing part) with the load model of Eq. 3.
+deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L,
+                           int32_t N, int32_t* bin_of_layer_h, double* bin_load_h) {
+    if (!layer_size_h || !k_l_h || !bin_of_layer_h || L < 1 || N < 1) return DEFT_ERR_INVALID_ARG;
+    for (int32_t l = 0; l < L; ++l)
+        if (layer_size_h[l] < 1 || k_l_h[l] < 1) return DEFT_ERR_INVALID_ARG;
+
+    std::vector<double> c(L);
+    for (int32_t l = 0; l < L; ++l) c[l] = (double)layer_size_h[l] * std::log((double)k_l_h[l]);
+    std::vector<char> placed(L, 0);
+    std::vector<double> load(N, 0.0);
+    for (int32_t round = 0; round < L; ++round) {
+        int32_t pick = -1;
+        for (int32_t l = 0; l < L; ++l) {
+            if (placed[l]) continue;
+            if (pick < 0 || c[l] > c[pick]) pick = l;
+        }
+        int32_t lightest = 0;
+        for (int32_t b = 1; b < N; ++b)
+            if (load[b] < load[lightest]) lightest = b;
+        bin_of_layer_h[pick] = lightest;
+        load[lightest] += c[pick];
+        placed[pick] = 1;
+    }
+    if (bin_load_h)
+        for (int32_t b = 0; b < N; ++b) bin_load_h[b] = load[b];
+    return DEFT_OK;
+}
+
+int32_t deft_rank_bin(int64_t iteration, int32_t rank, int32_t N) {
+    if (N < 1 || rank < 0 || rank >= N || iteration < 0) return -1;
+    return (int32_t)((iteration % N + rank) % N);
+}
+
+deft_status deft_bin_layers(const int32_t* bin_of_layer_h, int32_t L, int32_t bin,
+                            int32_t* my_layers_h, int32_t cap, int32_t* n_my_out) {
+    if (!bin_of_layer_h || !n_my_out || L < 1 || bin < 0 || cap < 0 || (cap > 0 && !my_layers_h))
+        return DEFT_ERR_INVALID_ARG;
+    int32_t n = 0;
+    for (int32_t l = 0; l < L; ++l) n += (bin_of_layer_h[l] == bin);
+    *n_my_out = n;
+    if (n > cap) return DEFT_ERR_CAPACITY;
+    n = 0;
+    for (int32_t l = 0; l < L; ++l)
+        if (bin_of_layer_h[l] == bin) my_layers_h[n++] = l;
+    return DEFT_OK;
+}
+
+}  // extern "C"

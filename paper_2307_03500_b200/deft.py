@@ -1,0 +1,238 @@
+"""Thin binding over libdeft.so (ctypes): the same names as the C ABI, argument marshalling only.
+
+Host tables are numpy arrays, device buffers are torch CUDA tensors (used for memory and
+streams only).  Nothing here computes anything of the method, and there is no fallback:
+if the CUDA library is missing or fails to load, importing a device call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdeft.so")
+
+OK = 0
+WARN_K_INEXACT = 1
+ERR_INVALID_ARG = -1
+ERR_INFEASIBLE_K = -2
+ERR_NONFINITE_NORM = -3
+ERR_CAPACITY = -4
+ERR_CUDA = -5
+MODE_PAPER = 0
+MODE_EXACT = 1
+
+
+class DeftError(RuntimeError):
+    def __init__(self, call: str, status: int, detail: str = ""):
+        self.status = status
+        super().__init__("%s failed: %s%s" % (call, status_string(status), detail))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdeft.so from the package directory.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                "libdeft.so is missing at %s: build it with `python -m paper_2307_03500_b200.build` "
+                "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        vp, i32, i64, sz = c.c_void_p, c.c_int32, c.c_int64, c.c_size_t
+        L.deft_status_string.restype = c.c_char_p
+        L.deft_status_string.argtypes = [i32]
+        L.deft_last_cuda_error.restype = i32
+        L.deft_last_cuda_error.argtypes = []
+        L.deft_split_layers.restype = i32
+        L.deft_split_layers.argtypes = [vp, i32, i32, vp, vp, i32, vp]
+        L.deft_allocate_k.restype = i32
+        L.deft_allocate_k.argtypes = [vp, vp, i32, i64, i32, vp, vp]
+        L.deft_partition.restype = i32
+        L.deft_partition.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.deft_rank_bin.restype = i32
+        L.deft_rank_bin.argtypes = [i64, i32, i32]
+        L.deft_bin_layers.restype = i32
+        L.deft_bin_layers.argtypes = [vp, i32, i32, vp, i32, vp]
+        L.deft_workspace_bytes.restype = sz
+        L.deft_workspace_bytes.argtypes = [i64, i32]
+        L.deft_layer_norms.restype = i32
+        L.deft_layer_norms.argtypes = [vp, vp, i64, vp, i32, vp, vp, sz, vp]
+        L.deft_select.restype = i32
+        L.deft_select.argtypes = [vp, vp, vp, vp, i32, vp, vp, i64, vp, sz, vp]
+        L.deft_residual_update.restype = i32
+        L.deft_residual_update.argtypes = [vp, i64, vp, i64, vp]
+        L.deft_topk_baseline.restype = i32
+        L.deft_topk_baseline.argtypes = [vp, i64, i64, vp, vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().deft_status_string(int(status)).decode()
+
+
+def _check(call: str, status: int, allow_warn: bool = False) -> int:
+    if status < 0 or (status > 0 and not allow_warn):
+        detail = ""
+        if status == ERR_CUDA:
+            detail = " (cudaError %d)" % lib().deft_last_cuda_error()
+        raise DeftError(call, status, detail)
+    return status
+
+
+def _np(a, dtype) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _hp(a: Optional[np.ndarray]):
+    return None if a is None else ctypes.c_void_p(a.ctypes.data)
+
+
+def _dp(t, dtype=None):
+    """Device pointer of a contiguous CUDA tensor."""
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+# ------------------------------------------------------------------------------------------
+# host planners
+# ------------------------------------------------------------------------------------------
+def deft_split_layers(tensor_sizes, n_workers: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 2 -> (layer_start int64[L+1], layer_tensor int32[L])."""
+    sizes = _np(tensor_sizes, np.int64)
+    L = ctypes.c_int32(0)
+    st = lib().deft_split_layers(_hp(sizes), sizes.size, int(n_workers), _hp(np.zeros(1, np.int64)), None, 0,
+                                 ctypes.byref(L))
+    if st != ERR_CAPACITY:
+        _check("deft_split_layers", st)
+    cap = int(L.value)
+    start = np.zeros(cap + 1, dtype=np.int64)
+    tensor = np.zeros(cap, dtype=np.int32)
+    _check("deft_split_layers",
+           lib().deft_split_layers(_hp(sizes), sizes.size, int(n_workers), _hp(start), _hp(tensor), cap,
+                                   ctypes.byref(L)))
+    return start, tensor
+
+
+def deft_allocate_k(norms, layer_size, k: int, mode: int = MODE_EXACT) -> Tuple[np.ndarray, int, int]:
+    """Algorithm 3 -> (k_l int64[L], sum_k, status) ; status may be WARN_K_INEXACT in PAPER mode."""
+    nr = _np(norms, np.float64)
+    sz = _np(layer_size, np.int64)
+    if nr.size != sz.size:
+        raise ValueError("norms and layer_size differ in length")
+    k_l = np.zeros(sz.size, dtype=np.int64)
+    s = ctypes.c_int64(0)
+    st = _check("deft_allocate_k",
+                lib().deft_allocate_k(_hp(nr), _hp(sz), sz.size, int(k), int(mode), _hp(k_l), ctypes.byref(s)),
+                allow_warn=True)
+    return k_l, int(s.value), st
+
+
+def deft_partition(layer_size, k_l, n_workers: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 4 packing -> (bin_of_layer int32[L], bin_load float64[N])."""
+    sz = _np(layer_size, np.int64)
+    kl = _np(k_l, np.int64)
+    if kl.size != sz.size:
+        raise ValueError("k_l and layer_size differ in length")
+    bins = np.zeros(sz.size, dtype=np.int32)
+    load = np.zeros(int(n_workers), dtype=np.float64)
+    _check("deft_partition", lib().deft_partition(_hp(sz), _hp(kl), sz.size, int(n_workers), _hp(bins), _hp(load)))
+    return bins, load
+
+
+def deft_rank_bin(iteration: int, rank: int, n_workers: int) -> int:
+    b = lib().deft_rank_bin(int(iteration), int(rank), int(n_workers))
+    if b < 0:
+        raise DeftError("deft_rank_bin", ERR_INVALID_ARG)
+    return int(b)
+
+
+def deft_bin_layers(bin_of_layer, bin_id: int) -> np.ndarray:
+    bins = _np(bin_of_layer, np.int32)
+    out = np.zeros(bins.size, dtype=np.int32)
+    n = ctypes.c_int32(0)
+    _check("deft_bin_layers", lib().deft_bin_layers(_hp(bins), bins.size, int(bin_id), _hp(out), out.size,
+                                                    ctypes.byref(n)))
+    return out[: n.value].copy()
+
+
+# ------------------------------------------------------------------------------------------
+# device calls
+# ------------------------------------------------------------------------------------------
+def deft_workspace_bytes(max_elems: int, max_layers: int) -> int:
+    return int(lib().deft_workspace_bytes(int(max_elems), int(max_layers)))
+
+
+def alloc_workspace(max_elems: int, max_layers: int, device="cuda"):
+    """A torch uint8 tensor of deft_workspace_bytes() bytes (torch allocations are 512-byte aligned)."""
+    import torch
+    return torch.empty(deft_workspace_bytes(max_elems, max_layers), dtype=torch.uint8, device=device)
+
+
+def deft_layer_norms(resid_acc, grad, layer_start_d, norms_d, ws, stream=None) -> None:
+    import torch
+    n_g = resid_acc.numel()
+    L = layer_start_d.numel() - 1
+    if grad is not None and grad.numel() != n_g:
+        raise ValueError("grad and resid_acc differ in length")
+    if norms_d.numel() < L:
+        raise ValueError("norms_d too small")
+    _check("deft_layer_norms",
+           lib().deft_layer_norms(_dp(resid_acc, torch.float32), _dp(grad, torch.float32), n_g,
+                                  _dp(layer_start_d, torch.int64), L, _dp(norms_d, torch.float64),
+                                  _dp(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_select(acc, layer_start_h, k_l_h, my_layers_h, val_d, idx_d, ws, stream=None) -> int:
+    """Algorithm 5 for one rank.  Returns the number of entries written (sum of k_l over my layers)."""
+    import torch
+    ls = _np(layer_start_h, np.int64)
+    kl = _np(k_l_h, np.int64)
+    my = _np(my_layers_h, np.int32)
+    if kl.size != ls.size - 1:
+        raise ValueError("k_l_h and layer_start_h disagree")
+    if my.size and (my.min() < 0 or my.max() >= kl.size):
+        raise ValueError("layer id out of range")
+    cap = min(val_d.numel(), idx_d.numel())
+    _check("deft_select",
+           lib().deft_select(_dp(acc, torch.float32), _hp(ls), _hp(kl), _hp(my), my.size,
+                             _dp(val_d, torch.float32), _dp(idx_d, torch.int64), cap, _dp(ws),
+                             ws.numel() * ws.element_size(), _stream(stream)))
+    return int(kl[my].sum()) if my.size else 0
+
+
+def deft_residual_update(acc, idx_d, count: int, stream=None) -> None:
+    import torch
+    if count > idx_d.numel():
+        raise ValueError("count exceeds idx_d")
+    _check("deft_residual_update",
+           lib().deft_residual_update(_dp(acc, torch.float32), acc.numel(), _dp(idx_d, torch.int64), int(count),
+                                      _stream(stream)))
+
+
+def deft_topk_baseline(acc, k: int, val_d, idx_d, ws, stream=None) -> None:
+    import torch
+    if min(val_d.numel(), idx_d.numel()) < k:
+        raise DeftError("deft_topk_baseline", ERR_CAPACITY)
+    _check("deft_topk_baseline",
+           lib().deft_topk_baseline(_dp(acc, torch.float32), acc.numel(), int(k), _dp(val_d, torch.float32),
+                                    _dp(idx_d, torch.int64), _dp(ws), ws.numel() * ws.element_size(),
+                                    _stream(stream)))

@@ -1,0 +1,286 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bars: indices, values, k_l and partitions are bit-exact; norms agree to 1e-5 relative
+(fp32 squares over runs of 8 elements, fp64 beyond, against the oracle's sequential fp64).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2307_03500_b200 import build as deft_build
+from paper_2307_03500_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+NORM_RTOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def deft():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    deft_build.build()
+    from paper_2307_03500_b200 import deft as d
+    d.lib()
+    return d
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _gpu_norms(deft, e, g, layer_start):
+    e_d = _dev(e)
+    g_d = _dev(g) if g is not None else None
+    ls_d = _dev(np.asarray(layer_start, dtype=np.int64))
+    L = len(layer_start) - 1
+    norms_d = torch.full((L,), -1.0, dtype=torch.float64, device="cuda")
+    ws = deft.alloc_workspace(e.size, L)
+    deft.deft_layer_norms(e_d, g_d, ls_d, norms_d, ws)
+    torch.cuda.synchronize()
+    return e_d.cpu().numpy(), norms_d.cpu().numpy()
+
+
+def _gpu_select(deft, acc_d, layer_start, k_l, my, ws=None, n_elems=None):
+    total = int(np.asarray(k_l)[my].sum()) if len(my) else 0
+    val_d = torch.full((total + 8,), 7.0, dtype=torch.float32, device="cuda")
+    idx_d = torch.full((total + 8,), -7, dtype=torch.int64, device="cuda")
+    if ws is None:
+        ws = deft.alloc_workspace(int(layer_start[-1]), len(layer_start) - 1)
+    n = deft.deft_select(acc_d, layer_start, k_l, my, val_d, idx_d, ws)
+    torch.cuda.synchronize()
+    assert n == total
+    # canaries behind the output are untouched
+    assert torch.all(val_d[total:] == 7.0) and torch.all(idx_d[total:] == -7)
+    return val_d[:total].cpu().numpy(), idx_d[:total].cpu().numpy()
+
+
+# ------------------------------------------------------------------------------------------
+# step 1: accumulate + norms
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wl", ["tiny", "resnet18", "bert_div64", "gpt2_div64_N64"])
+def test_accumulate_and_norms(deft, wl):
+    w = {"tiny": W.tiny(), "resnet18": W.resnet18(), "bert_div64": W.scaled_down(W.bert_large(), 64),
+         "gpt2_div64_N64": W.scaled_down(W.gpt2_medium(64, 0.01), 64)}[wl]
+    rng = np.random.default_rng(7)
+    e = (rng.standard_normal(w.n_g, dtype=np.float32) * np.float32(1e-3))
+    g = w.gradient(0)
+    start, _ = oracle.split_layers(w.sizes, w.n_workers)
+    want_acc = oracle.accumulate(e.copy(), g)
+    want = oracle.layer_norms(want_acc, start)
+    got_acc, got = _gpu_norms(deft, e, g, start)
+    assert got_acc.tobytes() == want_acc.tobytes()          # one fp32 add per element: bit-exact
+    assert np.all(np.abs(got - want) <= NORM_RTOL * want)
+    assert np.all((want > 0) | (got == 0))
+    # run-to-run bit-identical
+    _, again = _gpu_norms(deft, e, g, start)
+    assert again.tobytes() == got.tobytes()
+    # norms-only mode: nothing written, same norms
+    kept, only = _gpu_norms(deft, want_acc, None, start)
+    assert kept.tobytes() == want_acc.tobytes() and only.tobytes() == got.tobytes()
+
+
+def test_norms_ragged_layers_and_closed_forms(deft):
+    # layer boundaries that are not multiples of anything, tiny layers, a zero layer, a tail
+    sizes = [1, 3, 8191, 8192, 8193, 10, 64, 37 * 37, 100, 5, 20001]
+    start = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    rng = np.random.default_rng(8)
+    e = rng.standard_normal(int(start[-1]), dtype=np.float32)
+    e[start[7]:start[8]] = 1.0     # all ones, 37*37 elements -> norm 37
+    e[start[8]:start[9]] = 0.0     # zero layer
+    got_acc, got = _gpu_norms(deft, e, None, start)
+    want = oracle.layer_norms(e, start)
+    assert np.all(np.abs(got - want) <= NORM_RTOL * want)
+    assert got[7] == 37.0 and got[8] == 0.0
+
+
+# ------------------------------------------------------------------------------------------
+# the whole path on the paper-shaped workloads (scaled so the oracle sorts in seconds)
+# ------------------------------------------------------------------------------------------
+def _whole_path(deft, w, steps=1, mode=None, iteration=0):
+    from paper_2307_03500_b200.pipeline import DeftStep
+    mode = deft.MODE_EXACT if mode is None else mode
+    N = w.n_workers
+    ds = DeftStep(w.sizes, N, w.density, mode=mode)
+    start, _ = oracle.split_layers(w.sizes, N)
+    assert ds.layer_start.tolist() == start.tolist()
+    size = np.diff(start)
+    e_cpu = np.zeros(w.n_g, dtype=np.float32)
+    e_gpu = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+    for t in range(steps):
+        g = w.gradient(t)
+        g_d = _dev(g)
+        # GPU
+        norms_gpu = ds.layer_norms(e_gpu, g_d).copy()
+        # oracle
+        oracle.accumulate(e_cpu, g)
+        norms_cpu = oracle.layer_norms(e_cpu, start)
+        assert e_gpu.cpu().numpy().tobytes() == e_cpu.tobytes()
+        assert np.all(np.abs(norms_gpu - norms_cpu) <= NORM_RTOL * norms_cpu)
+        # both planners get identical norms (the GPU's): k_l and bins must then be bit-exact
+        plan = ds.plan(norms_gpu, iteration + t)
+        k_l, s = oracle.allocate_k(norms_gpu, size, ds.k, mode)
+        bins, load = oracle.partition(size, k_l, N)
+        assert plan.k_l.tolist() == k_l.tolist() and plan.sum_k == s
+        assert plan.bin_of_layer.tolist() == bins.tolist() and plan.bin_load.tobytes() == load.tobytes()
+        if mode == deft.MODE_EXACT:
+            assert s == ds.k
+        seen = np.zeros(w.n_g, dtype=np.int8)
+        all_idx = []
+        for r in range(N):
+            my = oracle.my_layers(bins, iteration + t, r, N)
+            assert plan.rank_layers[r].tolist() == my.tolist()
+            val_d, idx_d = ds.select_rank(e_gpu, plan, r)
+            torch.cuda.synchronize()
+            want_val, want_idx = oracle.select_rank(e_cpu, start, k_l, my)
+            assert idx_d.cpu().numpy().tolist() == want_idx.tolist()
+            assert val_d.cpu().numpy().tobytes() == want_val.tobytes()
+            seen[want_idx] += 1
+            all_idx.append(idx_d)
+        assert seen.max() == 1 and int(seen.sum()) == s       # disjoint, density kept
+        for idx_d in all_idx:
+            ds.residual_update(e_gpu, idx_d)
+        torch.cuda.synchronize()
+        oracle.residual_update(e_cpu, np.nonzero(seen)[0])
+        assert e_gpu.cpu().numpy().tobytes() == e_cpu.tobytes()
+
+
+def test_whole_path_tiny(deft):
+    _whole_path(deft, W.tiny())
+    _whole_path(deft, W.tiny(), mode=0, iteration=5)
+
+
+def test_whole_path_resnet18(deft):
+    _whole_path(deft, W.resnet18())
+
+
+def test_whole_path_lstm_three_steps_with_residual(deft):
+    _whole_path(deft, W.scaled_down(W.lstm_lm(), 16), steps=3)
+
+
+def test_whole_path_bert_shaped(deft):
+    _whole_path(deft, W.scaled_down(W.bert_large(), 32))
+
+
+@pytest.mark.parametrize("N,d", [(1, 0.1), (8, 0.01), (64, 0.001)])
+def test_whole_path_gpt2_shaped(deft, N, d):
+    _whole_path(deft, W.scaled_down(W.gpt2_medium(N, d), 32))
+
+
+# ------------------------------------------------------------------------------------------
+# selection edge cases
+# ------------------------------------------------------------------------------------------
+KINDS = ["gauss", "few_values", "all_equal", "all_zero", "signed_zero", "mostly_zero", "outlier",
+         "bf16_like", "denormal", "wide_exponent"]
+
+
+@pytest.mark.parametrize("kind", KINDS)
+def test_select_adversarial_layers(deft, kind):
+    # one vector holding layers of awkward sizes at awkward offsets; every layer is its own case
+    sizes = [1, 10, 31, 32, 33, 4095, 4096, 4097, 5, 12289, 20000, 3]
+    start = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    x = W.adversarial_vector(kind, int(start[-1]), seed=3)
+    acc_d = _dev(x)
+    ws = deft.alloc_workspace(x.size, len(sizes))
+    for pick in ("one", "all", "mid", "most"):
+        k_l = np.array([{"one": 1, "all": s, "mid": max(1, s // 3), "most": max(1, s - 1)}[pick] for s in sizes],
+                       dtype=np.int64)
+        for my in ([0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11], [5], [1, 4, 7, 10], [11]):
+            my = np.array(my, dtype=np.int32)
+            val, idx = _gpu_select(deft, acc_d, start, k_l, my, ws)
+            want_val, want_idx = oracle.select_rank(x, start, k_l, my)
+            assert idx.tolist() == want_idx.tolist(), (kind, pick, my.tolist())
+            assert val.tobytes() == want_val.tobytes()
+
+
+def test_select_threshold_value_repeated_across_tiles(deft):
+    # the k-th magnitude occurs many times, spread over several tiles and both signs
+    n = 50000
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal(n, dtype=np.float32) * np.float32(0.1)
+    x[np.abs(x) > 0.25] = 0.1
+    rep = rng.choice(n, size=3000, replace=False)
+    x[rep] = np.where(rng.random(3000) < 0.5, 0.25, -0.25).astype(np.float32)
+    big = rng.choice(np.setdiff1d(np.arange(n), rep), size=100, replace=False)
+    x[big] = 1.0 + rng.random(100).astype(np.float32)
+    acc_d = _dev(x)
+    start = np.array([0, n], dtype=np.int64)
+    for k in (100, 101, 1500, 3099, 3100, 3101):
+        val, idx = _gpu_select(deft, acc_d, start, np.array([k]), np.array([0], dtype=np.int32))
+        want_val, want_idx = oracle.select_layer(x, 0, n, k)
+        assert idx.tolist() == want_idx.tolist() and val.tobytes() == want_val.tobytes()
+
+
+def test_empty_rank_and_single_layer_equals_topk(deft):
+    x = W.adversarial_vector("gauss", 70001, seed=6)
+    acc_d = _dev(x)
+    ws = deft.alloc_workspace(x.size, 4)
+    start = np.array([0, 70001], dtype=np.int64)
+    val_d = torch.empty(16, dtype=torch.float32, device="cuda")
+    idx_d = torch.empty(16, dtype=torch.int64, device="cuda")
+    assert deft.deft_select(acc_d, start, np.array([5]), np.array([], dtype=np.int32), val_d, idx_d, ws) == 0
+    k = 701
+    v1, i1 = _gpu_select(deft, acc_d, start, np.array([k]), np.array([0], dtype=np.int32), ws)
+    val_d = torch.empty(k, dtype=torch.float32, device="cuda")
+    idx_d = torch.empty(k, dtype=torch.int64, device="cuda")
+    deft.deft_topk_baseline(acc_d, k, val_d, idx_d, ws)
+    torch.cuda.synchronize()
+    want_val, want_idx = oracle.topk(x, k)
+    assert idx_d.cpu().numpy().tolist() == want_idx.tolist() == i1.tolist()
+    assert val_d.cpu().numpy().tobytes() == want_val.tobytes() == v1.tobytes()
+
+
+@pytest.mark.parametrize("n,k", [(1, 1), (4097, 4097), (1 << 20, 1), (3_000_001, 30_000), (3_000_001, 2_999_999)])
+def test_topk_baseline(deft, n, k):
+    x = W.adversarial_vector("gauss", n, seed=n % 97)
+    acc_d = _dev(x)
+    ws = deft.alloc_workspace(n, 1)
+    val_d = torch.empty(k, dtype=torch.float32, device="cuda")
+    idx_d = torch.empty(k, dtype=torch.int64, device="cuda")
+    deft.deft_topk_baseline(acc_d, k, val_d, idx_d, ws)
+    torch.cuda.synchronize()
+    want_val, want_idx = oracle.topk(x, k)
+    assert np.array_equal(idx_d.cpu().numpy(), want_idx)
+    assert val_d.cpu().numpy().tobytes() == want_val.tobytes()
+
+
+def test_select_is_bit_deterministic_run_to_run(deft):
+    w = W.scaled_down(W.gpt2_medium(4, 0.01), 16)
+    x = w.gradient(0)
+    acc_d = _dev(x)
+    start, _ = oracle.split_layers(w.sizes, 4)
+    size = np.diff(start)
+    k_l = np.maximum(1, size // 100)
+    my = np.arange(0, size.size, 2, dtype=np.int32)
+    a = _gpu_select(deft, acc_d, start, k_l, my)
+    b = _gpu_select(deft, acc_d, start, k_l, my)
+    assert a[0].tobytes() == b[0].tobytes() and a[1].tobytes() == b[1].tobytes()
+
+
+def test_residual_update(deft):
+    x = W.adversarial_vector("gauss", 100003, seed=8)
+    acc_d = _dev(x)
+    _, idx = oracle.topk(x, 5000)
+    idx_d = _dev(idx)
+    deft.deft_residual_update(acc_d, idx_d, idx.size)
+    deft.deft_residual_update(acc_d, idx_d, 0)
+    torch.cuda.synchronize()
+    want = oracle.residual_update(x.copy(), idx)
+    assert acc_d.cpu().numpy().tobytes() == want.tobytes()
+
+
+def test_capacity_errors_are_reported_not_faulted(deft):
+    x = W.adversarial_vector("gauss", 10000, seed=1)
+    acc_d = _dev(x)
+    start = np.array([0, 10000], dtype=np.int64)
+    val_d = torch.empty(10, dtype=torch.float32, device="cuda")
+    idx_d = torch.empty(10, dtype=torch.int64, device="cuda")
+    ws = deft.alloc_workspace(10000, 1)
+    with pytest.raises(deft.DeftError) as ei:
+        deft.deft_select(acc_d, start, np.array([11]), np.array([0], dtype=np.int32), val_d, idx_d, ws)
+    assert ei.value.status == deft.ERR_CAPACITY
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(deft.DeftError) as ei:
+        deft.deft_select(acc_d, start, np.array([5]), np.array([0], dtype=np.int32), val_d, idx_d, small)
+    assert ei.value.status == deft.ERR_CAPACITY

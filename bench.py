@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the DEFT gradient-selection hot path on B200.
+
+One step = the whole path on one synthetic gradient vector: fused accumulate + per-layer
+norms over n_g, norms to the host, Algorithm 3 + Algorithm 4 on the host, then Algorithm 5
+and the residual update for EVERY one of the N simulated workers, one after the other on the
+same GPU.  `value` = n_g / (device-timed duration of that whole step).  The per-worker view
+the paper plots (slowest worker) is reported beside it under "worker_view".
+
+    python bench.py [--gpus G] [--steps K] [--warmup W] [--workload bert_large] [--impl reference]
+
+With G > 1 (torchrun) every GPU runs an independent replica of the same step (the path has
+no exchange step); the time is the max over ranks and value = G * n_g / time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2307_03500_b200 import workloads as W  # noqa: E402
+
+METRIC = "gradient-selection Gelem/s (n_g / ms per step, all N simulated workers; worker_view = slowest worker)"
+UNIT = "Gelem/s"
+
+
+def make_workload(args):
+    if args.workload == "gpt2_medium":
+        return W.gpt2_medium(args.n_workers or 16, args.density or 0.01)
+    w = W.WORKLOADS[args.workload]()
+    if args.n_workers:
+        w.n_workers = args.n_workers
+    if args.density:
+        w.density = args.density
+    return w
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# clocks during the timed region (NVML, read-only)
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    def __init__(self, index: int):
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as ex:  # noqa: BLE001
+            self.error = repr(ex)
+
+    def _loop(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "hw_power_brake": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:  # noqa: BLE001
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------
+# the oracle on the host cores (CPU baseline and --impl reference)
+# ------------------------------------------------------------------------------------------
+def oracle_step_sample(w, g, budget_ranks: int = 4):
+    """One step of the oracle on a bounded sample: accumulate + norms over the whole vector,
+    both planners, then selection + zeroing for `budget_ranks` evenly spaced ranks; the rank
+    part is scaled to all N ranks by the elements scanned."""
+    import oracle
+    N = w.n_workers
+    start, _ = oracle.split_layers(w.sizes, N)
+    size = np.diff(start)
+    e = np.zeros(w.n_g, dtype=np.float32)
+    t0 = time.perf_counter()
+    oracle.accumulate(e, g)
+    norms = oracle.layer_norms(e, start)
+    t1 = time.perf_counter()
+    k = max(w.k, size.size)
+    k_l, _ = oracle.allocate_k(norms, size, k, oracle.MODE_EXACT)
+    bins, _ = oracle.partition(size, k_l, N)
+    t2 = time.perf_counter()
+    ranks = sorted(set(int(round(i * N / budget_ranks)) % N for i in range(min(budget_ranks, N))))
+    elems = 0
+    t_sel = 0.0
+    for r in ranks:
+        my = oracle.my_layers(bins, 0, r, N)
+        ta = time.perf_counter()
+        val, idx = oracle.select_rank(e, start, k_l, my)
+        oracle.residual_update(e, idx)
+        t_sel += time.perf_counter() - ta
+        elems += int(size[my].sum())
+    scale = w.n_g / max(1, elems)
+    est = (t1 - t0) + (t2 - t1) + t_sel * scale
+    return {
+        "est_step_s": est, "t_acc_norms_s": t1 - t0, "t_planners_s": t2 - t1, "t_select_sampled_s": t_sel,
+        "ranks_sampled": ranks, "elems_sampled": elems, "scale": scale,
+        "sample": "accumulate+norms over all %d elements, Algorithms 3+4, then selection+zeroing of ranks %s "
+                  "(%d elements) scaled by %.2f to all %d ranks" % (w.n_g, ranks, elems, scale, N),
+    }
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_workload(args)
+    g = w.gradient(0)
+    steps = max(1, min(args.steps, 3))
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
+        oracle_step_sample(w, g, 1)
+    res = [oracle_step_sample(w, g, args.cpu_ranks) for _ in range(steps)]
+    est = float(np.mean([r["est_step_s"] for r in res]))
+    val = w.n_g / est / 1e9
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "n_g": w.n_g, "n_workers": w.n_workers, "density": w.density, "k": w.k,
+                   "seed": w.seed},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": res[-1]["sample"]},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2307_03500_b200 import build as deft_build
+    deft_build.build()
+    from paper_2307_03500_b200 import deft
+    from paper_2307_03500_b200.pipeline import DeftStep
+
+    w = make_workload(args)
+    N = w.n_workers
+    g_host = torch.from_numpy(w.gradient(0)).pin_memory()
+    ds = DeftStep(w.sizes, N, w.density, device=dev)
+    n_g, L, k = ds.n_g, ds.L, ds.k
+    g = g_host.to(dev)
+    e = torch.zeros(n_g, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    launches = {"n": 0}
+
+    def one_step(it, rec=None, grad=g):
+        """The whole path for all N simulated ranks.  rec: optional dict collecting events."""
+        e0 = ev(); e0.record(stream)
+        deft.deft_layer_norms(e, grad, ds.layer_start_d, ds.norms_d, ds.ws)
+        e1 = ev(); e1.record(stream)
+        ds.norms_h.copy_(ds.norms_d, non_blocking=True)
+        stream.synchronize()
+        th0 = time.perf_counter()
+        plan = ds.plan(ds.norms_h.numpy(), it)
+        th1 = time.perf_counter()
+        launches["n"] += 2
+        marks = []
+        for r in range(N):
+            a = ev(); a.record(stream)
+            val, idx = ds.select_rank(e, plan, r)
+            b = ev(); b.record(stream)
+            ds.residual_update(e, idx)
+            c = ev(); c.record(stream)
+            marks.append((a, b, c))
+            if idx.numel():
+                launches["n"] += 10
+        if rec is not None:
+            rec.append({"acc": (e0, e1), "host_s": th1 - th0, "ranks": marks, "plan": plan})
+        return plan
+
+    if args.mode != "step":
+        # profiling helper: repeat one call only (no JSON line; use it under ncu on a small workload)
+        deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)
+        ds.norms_h.copy_(ds.norms_d)
+        plan = ds.plan(ds.norms_h.numpy(), 0)
+        tk_val = torch.empty(k, dtype=torch.float32, device=dev)
+        tk_idx = torch.empty(k, dtype=torch.int64, device=dev)
+        r_big = int(np.argmax(plan.rank_elems))
+        times = []
+        for it in range(args.warmup + args.steps):
+            a, b = ev(), ev()
+            a.record(stream)
+            if args.mode == "topk":
+                deft.deft_topk_baseline(e, k, tk_val, tk_idx, ds.ws)
+            elif args.mode == "norms":
+                deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)
+            else:
+                ds.select_rank(e, plan, r_big)
+            b.record(stream)
+            stream.synchronize()
+            times.append(a.elapsed_time(b))
+        print("mode=%s workload=%s n_g=%d k=%d rank=%d rank_elems=%d median_ms=%.4f" % (
+            args.mode, w.name, n_g, k, r_big, int(plan.rank_elems[r_big]), float(np.median(times[args.warmup:]))),
+            file=sys.stderr)
+        return
+
+    # warm-up
+    for it in range(args.warmup):
+        one_step(it)
+    barrier()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    recs = []
+    launches["n"] = 0
+    t_begin, t_end = ev(), ev()
+    barrier()
+    t_begin.record(stream)
+    for it in range(args.steps):
+        one_step(args.warmup + it, recs)
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_begin.elapsed_time(t_end)
+    gpu_launches = launches["n"]
+
+    # per-call statistics from the events recorded inside the timed region
+    t_acc = np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in recs])
+    t_host = np.array([r["host_s"] * 1e3 for r in recs])
+    t_sel = np.array([[a.elapsed_time(b) for (a, b, c) in r["ranks"]] for r in recs])      # [steps, N]
+    t_upd = np.array([[b.elapsed_time(c) for (a, b, c) in r["ranks"]] for r in recs])
+    plan = recs[-1]["plan"]
+    sel_med = np.median(t_sel, axis=0)
+    upd_med = np.median(t_upd, axis=0)
+    worker_ms = float(np.median(t_acc) + np.median(t_host) + np.max(sel_med + upd_med))
+
+    # full-vector Top-k on the same GPU (comparison sparsifier), timed alone
+    tk_val = torch.empty(k, dtype=torch.float32, device=dev)
+    tk_idx = torch.empty(k, dtype=torch.int64, device=dev)
+    tk = []
+    for i in range(3 + 10):
+        a, b = ev(), ev()
+        a.record(stream)
+        deft.deft_topk_baseline(e, k, tk_val, tk_idx, ds.ws)
+        b.record(stream)
+        stream.synchronize()
+        if i >= 3:
+            tk.append(a.elapsed_time(b))
+    t_topk = float(np.median(tk))
+
+    # end to end through the public call with HOST buffers: gradient from pinned host memory,
+    # selected (value, index) pairs and norms back to the host, every step
+    out_val_h = torch.empty(ds.val_d.numel(), dtype=torch.float32).pin_memory()
+    out_idx_h = torch.empty(ds.idx_d.numel(), dtype=torch.int64).pin_memory()
+    g_stage = torch.empty_like(g)
+    e2e_steps = max(3, min(args.steps, 20))
+    barrier()
+    te0, te1 = ev(), ev()
+    te0.record(stream)
+    for it in range(e2e_steps):
+        g_stage.copy_(g_host, non_blocking=True)
+        pl = one_step(args.warmup + args.steps + it, None, g_stage)
+        out_val_h[:pl.sum_k].copy_(ds.val_d[:pl.sum_k], non_blocking=True)
+        out_idx_h[:pl.sum_k].copy_(ds.idx_d[:pl.sum_k], non_blocking=True)
+        stream.synchronize()
+    te1.record(stream)
+    barrier()
+    e2e_ms = te0.elapsed_time(te1) / e2e_steps
+
+    # max over ranks of the job
+    ms_per_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_per_step, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        value = world * n_g / (ms_per_step * 1e-3) / 1e9
+        acc_bytes = 12.0 * n_g
+        acc_ms = float(np.median(t_acc))
+        acc_gbs = acc_bytes / (acc_ms * 1e-3) / 1e9
+        sel_bytes = 8.0 * plan.rank_elems + 12.0 * plan.rank_k
+        with np.errstate(divide="ignore", invalid="ignore"):
+            sel_gbs = np.where(sel_med > 0, sel_bytes / (sel_med * 1e-3) / 1e9, 0.0)
+        busy = plan.rank_elems > 0
+        r_max = int(np.argmax(sel_med))
+        cost_max = float(plan.bin_load.max())
+        lnk = math.log(k)
+        cpu = None
+        if not args.no_cpu_baseline:
+            c = oracle_step_sample(w, g_host.numpy(), args.cpu_ranks)
+            cpu = {"value": n_g / c["est_step_s"] / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                   "sample": c["sample"], "est_ms_per_step": c["est_step_s"] * 1e3}
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n_g": n_g, "layers": L, "n_workers": N, "density": w.density, "k": k,
+                       "sum_k": int(plan.sum_k), "seed": w.seed, "k_mode": "EXACT",
+                       "l2": "inputs larger than L2 (%.2f GB vector, no flush)" % (4.0 * n_g / 1e9),
+                       "multi_gpu": "replicas only"},
+            "clocks": clocks,
+            "e2e": {"value": world * n_g / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": 4 * n_g, "d2h_bytes_per_step": 12 * int(plan.sum_k) + 8 * L},
+            "gpu_launches": gpu_launches,
+            "roofline": {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,
+                         "peak": peak, "unit": "GB/s", "frac": acc_gbs / peak, "peak_kind": peak_kind,
+                         "traffic": None, "bytes_per_launch": acc_bytes, "ms_per_launch": acc_ms,
+                         "frac_of_nominal_8TBs": acc_gbs / 8000.0},
+            "roofline_select": {"bound": "hbm", "call": "deft_select (one rank)", "bytes_per_elem": 8,
+                                "bytes_per_selected": 12, "unit": "GB/s", "peak": peak,
+                                "achieved_mean": float(sel_gbs[busy].mean()), "achieved_min": float(sel_gbs[busy].min()),
+                                "achieved_max": float(sel_gbs[busy].max()),
+                                "frac_mean": float(sel_gbs[busy].mean() / peak),
+                                "frac_slowest_rank": float(sel_gbs[r_max] / peak)},
+            "worker_view": {"ms_per_step_slowest_worker": worker_ms, "gelems": n_g / (worker_ms * 1e-3) / 1e9,
+                            "t_acc_norms_ms": acc_ms, "t_host_ms": float(np.median(t_host)),
+                            "select_ms_max": float(sel_med.max()), "select_ms_mean": float(sel_med[busy].mean()),
+                            "select_ms_min": float(sel_med[busy].min()), "update_ms_max": float(upd_med.max()),
+                            "select_gelems_system": n_g / (float(sel_med.max()) * 1e-3) / 1e9,
+                            "slowest_rank": r_max, "slowest_rank_elems": int(plan.rank_elems[r_max]),
+                            "slowest_rank_k": int(plan.rank_k[r_max]),
+                            "rank_elems_max_over_mean": float(plan.rank_elems.max() / plan.rank_elems.mean()),
+                            "rank_k_min": int(plan.rank_k.min()), "rank_k_max": int(plan.rank_k.max())},
+            "topk_baseline": {"ms": t_topk, "gbs": 8.0 * n_g / (t_topk * 1e-3) / 1e9,
+                              "speedup_vs_slowest_rank": t_topk / float(sel_med.max()),
+                              "model_f_n": n_g * lnk / cost_max if cost_max > 0 else None,
+                              "model_f_trivial_n": N * lnk / math.log(k / N) if k > N else None},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="bert_large", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--n-workers", type=int, default=0)
+    ap.add_argument("--density", type=float, default=0.0)
+    ap.add_argument("--cpu-ranks", type=int, default=4, help="ranks the oracle runs for the CPU baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select"],
+                    help="step = the benchmark; the others repeat one call only, for profiler captures")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

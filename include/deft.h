@@ -59,6 +59,15 @@ DEFT_API const char* deft_status_string(deft_status s);
 /* The cudaError_t value behind the calling thread's most recent DEFT_ERR_CUDA (0 if none). */
 DEFT_API int32_t deft_last_cuda_error(void);
 
+/*
+ * Diagnostic: when timing_d (DEVICE, 16 x uint64, zeroed by the caller) is not NULL every
+ * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs):
+ * [0] kernel start, [1] end of histogram pass, [2] after barrier, [3] end of staging pass,
+ * [4] after barrier, [5] end of per-layer finish, [6] end of the general path (0 if not
+ * taken).  Pass NULL to switch it off.  Not thread-safe; not for production use.
+ */
+DEFT_API void deft_debug_select_timing(void* timing_d);
+
 /* ------------------------------------------------------------------------------------------
  * Host planners (cheap, O(L) .. O(L^2); run on the CPU as in the paper)
  * ---------------------------------------------------------------------------------------- */
@@ -160,6 +169,8 @@ DEFT_API deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, i
  * (so NaN > Inf > finite, denormals are not flushed); equal magnitudes are won by the
  * lower index.  Output: the selected entries of all those layers in ascending global
  * index — signed values and int64 indices — exactly sum of k_l of them.
+ * This one-shot form builds a single-rank plan, stages it through the workspace and
+ * launches; per-step use should go through deft_plan_build/deft_select_planned.
  *   acc_d             in   the accumulated vector (16-byte aligned); not modified
  *   layer_start_h[L+1], k_l_h[L]   HOST tables for the whole model
  *   my_layers_h[n_my] HOST, ascending; n_my may be 0 (nothing is written)
@@ -170,6 +181,68 @@ DEFT_API deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, i
 DEFT_API deft_status deft_select(const float* acc_d, const int64_t* layer_start_h, const int64_t* k_l_h,
                         const int32_t* my_layers_h, int32_t n_my, float* val_d, int64_t* idx_d,
                         int64_t out_cap, void* ws_d, size_t ws_bytes, void* stream);
+
+/*
+ * The per-step plan — Algorithm 4, lines 1-2 and 20 for every rank at once.
+ * Once k_l (Algorithm 3) and the bins (Algorithm 4) of a step are known, the layer
+ * lists of all N ranks are laid out in one position-independent blob: rank r owns the
+ * layers of bin (iteration % N + r) % N, ascending.  The blob is built on the host
+ * (deft_plan_build), copied to the device once (deft_plan_upload, which also clears the
+ * per-layer counters in the workspace), and then deft_select_planned() runs any rank
+ * with a single kernel launch and no further host-to-device traffic.  Ranks of one plan
+ * use disjoint parts of the workspace.
+ *
+ * deft_plan_bytes: size of the blob for L layers and N ranks (0 on invalid arguments;
+ * N <= 4096).
+ * deft_plan_build: plan_h[plan_bytes] out (HOST; pinned memory makes the upload
+ * asynchronous).  Errors: INVALID_ARG (null, a bin outside [0,N), k_l outside
+ * [1, size_l], a layer above DEFT_MAX_LAYER_ELEMS), CAPACITY (blob too small).
+ * deft_plan_rank_info: what rank `rank` will do: number of layers, elements scanned,
+ * entries selected (sum of its k_l), and the sum of k over lower ranks (a convenient
+ * offset into one shared output buffer).  Any out pointer may be NULL.
+ * deft_plan_rank_table: the same four numbers for all N ranks at once (arrays of N).
+ * deft_plan_upload: plan_d (DEVICE, 16-byte aligned, deft_plan_bytes) <- plan_h, on
+ * `stream`.  Must be called again before the plan's ranks are re-run (the counters it
+ * clears are consumed by the selection).  Errors: INVALID_ARG, CAPACITY (workspace), CUDA.
+ */
+DEFT_API size_t deft_plan_bytes(int32_t L, int32_t N);
+DEFT_API deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
+                                     const int32_t* bin_of_layer_h, int32_t L, int32_t N,
+                                     int64_t iteration, void* plan_h, size_t plan_bytes);
+DEFT_API deft_status deft_plan_rank_info(const void* plan_h, int32_t rank, int32_t* n_layers_out,
+                                         int64_t* elems_out, int64_t* k_out, int64_t* out_off_out);
+DEFT_API deft_status deft_plan_rank_table(const void* plan_h, int32_t N, int32_t* n_layers_h,
+                                          int64_t* elems_h, int64_t* k_h, int64_t* out_off_h);
+DEFT_API deft_status deft_plan_upload(const void* plan_h, void* plan_d, void* ws_d, size_t ws_bytes,
+                                      void* stream);
+
+/*
+ * Layer-wise gradient selection for rank `rank` of an uploaded plan — Algorithm 5.
+ * Same result as deft_select() on that rank's layer list: the rank's selected entries in
+ * ascending global index, exactly deft_plan_rank_info().k of them, written to val_d/idx_d
+ * (the rank's own output; out_cap entries available).  A rank without layers writes
+ * nothing.  plan_h is read on the host for the rank's sizes; plan_d is what the kernel
+ * reads.  Errors: INVALID_ARG, CAPACITY (out_cap or workspace), CUDA.
+ */
+DEFT_API deft_status deft_select_planned(const float* acc_d, const void* plan_h, const void* plan_d,
+                                         int32_t rank, float* val_d, int64_t* idx_d, int64_t out_cap,
+                                         void* ws_d, size_t ws_bytes, void* stream);
+
+/*
+ * Simulation driver: Algorithm 5 followed by the residual update (Algorithm 1 lines 11-12)
+ * for the ranks rank_begin <= r < rank_end of an uploaded plan, one after the other on
+ * `stream` — what N workers would each do on their own GPU, replayed on one.  Rank r
+ * writes its entries at offset deft_plan_rank_info().out_off of val_d / idx_d (shared
+ * buffers of out_cap >= total k entries) and then zeroes them in acc_d.  Because ranks own
+ * disjoint layers the result equals zeroing the union after all selections.
+ * events: NULL, or 3 cudaEvent_t per rank (HOST array of handles): recorded before the
+ * selection, between selection and update, and after the update, for per-rank timing.
+ * Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+DEFT_API deft_status deft_select_update_ranks(float* acc_d, int64_t n_g, const void* plan_h,
+                                              const void* plan_d, int32_t rank_begin, int32_t rank_end,
+                                              float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d,
+                                              size_t ws_bytes, void* const* events, void* stream);
 
 /*
  * Residual update — Algorithm 1 lines 11-12: acc[idx[j]] = +0.0f for j < count; the

@@ -1,5 +1,6 @@
-// C-ABI entry points of libdeft that touch the GPU: argument checks, workspace carve-up,
-// the small host-built layer table of one rank, and the kernel launch sequence.
+// C-ABI entry points of libdeft that touch the GPU: argument checks, the per-step plan
+// (host-built tables of every rank's layers), workspace carve-up and kernel launches.
+#include <cstring>
 #include <vector>
 
 #include "deft_common.cuh"
@@ -7,6 +8,7 @@
 namespace deft {
 
 static thread_local int32_t g_last_cuda_error = 0;
+static unsigned long long* g_select_timing = nullptr;
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int32_t)e; }
 
@@ -30,54 +32,131 @@ namespace {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
-// Builds the rank's layer table (with sentinel) on the host.  Returns a status.
-deft_status build_rank_table(const int64_t* layer_start_h, const int64_t* k_l_h,
-                             const int32_t* my_layers_h, int32_t n_my, std::vector<LayerDesc>& out,
-                             int64_t& tiles, int64_t& elems, int64_t& k_total) {
-    out.resize((size_t)n_my + 1);
-    tiles = elems = k_total = 0;
-    for (int32_t j = 0; j < n_my; ++j) {
-        const int32_t l = my_layers_h[j];
-        if (l < 0 || (j > 0 && l <= my_layers_h[j - 1])) return DEFT_ERR_INVALID_ARG;
-        const int64_t s = layer_start_h[l], e = layer_start_h[l + 1];
-        if (s < 0 || e <= s || e - s > DEFT_MAX_LAYER_ELEMS) return DEFT_ERR_INVALID_ARG;
-        if (j > 0 && s < out[j - 1].end) return DEFT_ERR_INVALID_ARG;
-        const int64_t k = k_l_h[l];
-        if (k < 1 || k > e - s) return DEFT_ERR_INVALID_ARG;
-        if (tiles > INT32_MAX - (e - s) / kTile - 2) return DEFT_ERR_INVALID_ARG;
-        LayerDesc& d = out[j];
-        d.start = s;
-        d.end = e;
-        d.k = k;
-        d.out_off = k_total;
-        d.elem_off = elems;
-        d.tile_first = (int32_t)tiles;
-        d.pad = 0;
-        tiles += (e - 1) / kTile - s / kTile + 1;
-        elems += e - s;
-        k_total += k;
+struct LayerItem { int64_t start, end, k; int32_t layer_id; };
+
+// Writes the plan blob for `ranks` lists of layers (each ascending in address).
+deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteration,
+                      const std::vector<std::vector<LayerItem>>& ranks) {
+    const int64_t N = (int64_t)ranks.size();
+    if (blob_bytes < plan_bytes(L, N)) return DEFT_ERR_CAPACITY;
+    char* base = static_cast<char*>(blob);
+    PlanHeader* hdr = reinterpret_cast<PlanHeader*>(base);
+    RankInfo* ri = reinterpret_cast<RankInfo*>(base + sizeof(PlanHeader));
+    LayerDesc* desc = reinterpret_cast<LayerDesc*>(base + sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)N);
+    std::memset(blob, 0, plan_bytes(L, N));
+    int64_t tiles_all = 0, elems_all = 0, k_all = 0;
+    int64_t d = 0;
+    for (int64_t r = 0; r < N; ++r) {
+        RankInfo& R = ri[r];
+        R.desc_first = (int32_t)d;
+        R.n_my = (int32_t)ranks[r].size();
+        R.tile_base = (int32_t)tiles_all;
+        R.elem_base = elems_all;
+        R.out_off = k_all;
+        int64_t tiles = 0, elems = 0, k = 0, prev_end = -1;
+        for (const LayerItem& it : ranks[r]) {
+            if (it.start < 0 || it.end <= it.start || it.end - it.start > DEFT_MAX_LAYER_ELEMS)
+                return DEFT_ERR_INVALID_ARG;
+            if (it.start < prev_end) return DEFT_ERR_INVALID_ARG;
+            if (it.k < 1 || it.k > it.end - it.start) return DEFT_ERR_INVALID_ARG;
+            LayerDesc& D = desc[d++];
+            D.start = it.start;
+            D.end = it.end;
+            D.k = it.k;
+            D.out_off = k;
+            D.elem_off = elems_all + elems;
+            D.tile_first = (int32_t)tiles;
+            D.layer_id = it.layer_id;
+            tiles += (it.end - 1) / kTile - it.start / kTile + 1;
+            elems += it.end - it.start;
+            k += it.k;
+            prev_end = it.end;
+            if (tiles_all + tiles > INT32_MAX) return DEFT_ERR_INVALID_ARG;
+        }
+        LayerDesc& Z = desc[d++];   // sentinel
+        Z.out_off = k;
+        Z.elem_off = elems_all + elems;
+        Z.tile_first = (int32_t)tiles;
+        Z.layer_id = -1;
+        R.tiles = (int32_t)tiles;
+        R.elems = elems;
+        R.k = k;
+        tiles_all += tiles;
+        elems_all += elems;
+        k_all += k;
     }
-    LayerDesc& z = out[n_my];
-    z.start = z.end = 0;
-    z.k = 0;
-    z.out_off = k_total;
-    z.elem_off = elems;
-    z.tile_first = (int32_t)tiles;
-    z.pad = 0;
+    hdr->magic = kPlanMagic;
+    hdr->L = L;
+    hdr->N = (int32_t)N;
+    hdr->total_tiles = (int32_t)tiles_all;
+    hdr->total_elems = elems_all;
+    hdr->total_k = k_all;
+    hdr->iteration = iteration;
     return DEFT_OK;
 }
 
-deft_status select_common(const float* acc_d, const std::vector<LayerDesc>& table, int32_t n_my,
-                          int64_t tiles, int64_t elems, int64_t k_total, float* val_d, int64_t* idx_d,
-                          int64_t out_cap, void* ws_d, size_t ws_bytes, cudaStream_t stream) {
-    if (out_cap < k_total) return DEFT_ERR_CAPACITY;
-    const SelectWorkspace w = carve_select_ws(ws_d, n_my, tiles, elems);
-    if (w.total_bytes > ws_bytes) return DEFT_ERR_CAPACITY;
-    // The table lives in pageable host memory: the runtime stages it before returning, so
-    // the vector may be released as soon as this call returns.
-    DEFT_CUDA_TRY(cudaMemcpyAsync(w.desc, table.data(), sizeof(LayerDesc) * ((size_t)n_my + 1),
-                                  cudaMemcpyHostToDevice, stream));
-    return launch_select(acc_d, w, n_my, (int32_t)tiles, val_d, idx_d, stream);
+inline bool plan_ok(const void* plan_h) {
+    return plan_h && static_cast<const PlanHeader*>(plan_h)->magic == kPlanMagic;
+}
+
+deft_status upload_plan(const void* plan_h, void* plan_d, void* ws_d, size_t ws_bytes, cudaStream_t stream) {
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    const WsLayout w = ws_layout(hdr->total_elems, hdr->L, hdr->total_tiles);
+    if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
+    DEFT_CUDA_TRY(cudaMemcpyAsync(plan_d, plan_h, plan_bytes(hdr->L, hdr->N), cudaMemcpyHostToDevice, stream));
+    DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + w.zero_begin, 0, w.zero_end - w.zero_begin, stream));
+    return DEFT_OK;
+}
+
+deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan_d, int32_t rank,
+                        float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
+                        cudaStream_t stream) {
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    if (rank < 0 || rank >= hdr->N) return DEFT_ERR_INVALID_ARG;
+    const RankInfo& R = plan_ranks(plan_h)[rank];
+    if (R.n_my == 0) return DEFT_OK;
+    if (out_cap < R.k) return DEFT_ERR_CAPACITY;
+    const WsLayout w = ws_layout(hdr->total_elems, hdr->L, hdr->total_tiles);
+    if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
+    char* ws = static_cast<char*>(ws_d);
+    SelParams p;
+    p.acc = acc_d;
+    p.desc = plan_descs(plan_d, hdr->N) + R.desc_first;
+    p.n_my = R.n_my;
+    p.tiles = R.tiles;
+    p.state = reinterpret_cast<LayerState*>(ws + w.state);
+    p.flags = reinterpret_cast<RankFlags*>(ws + w.flags) + rank;
+    p.hist1 = reinterpret_cast<uint32_t*>(ws + w.hist1);
+    p.hist2 = reinterpret_cast<uint32_t*>(ws + w.hist2);
+    p.hist3 = reinterpret_cast<uint32_t*>(ws + w.hist3);
+    const size_t slot0 = 2 * ((size_t)R.tile_base + (size_t)rank);
+    p.runcnt = reinterpret_cast<uint32_t*>(ws + w.cnt) + slot0;
+    p.runge = reinterpret_cast<uint2*>(ws + w.ge) + slot0;
+    p.staging = reinterpret_cast<uint2*>(ws + w.staging);
+    p.val = val_d;
+    p.idx = idx_d;
+    p.timing = g_select_timing;
+    return launch_select(p, stream);
+}
+
+// One-shot path: plan for a single rank, kept in the scratch area at the head of the workspace.
+deft_status select_once(const float* acc_d, const std::vector<LayerItem>& items, float* val_d,
+                        int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes, cudaStream_t stream) {
+    const int32_t L = (int32_t)items.size();
+    std::vector<std::vector<LayerItem>> ranks(1, items);
+    std::vector<char> blob(plan_bytes(L, 1));
+    deft_status s = fill_plan(blob.data(), blob.size(), L, 0, ranks);
+    if (s != DEFT_OK) return s;
+    const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(blob.data());
+    if (out_cap < hdr->total_k) return DEFT_ERR_CAPACITY;
+    const WsLayout w = ws_layout(hdr->total_elems, hdr->L, hdr->total_tiles);
+    if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
+    void* plan_d = static_cast<char*>(ws_d) + w.plan;
+    // The blob is pageable host memory: the runtime stages it before returning, so it may
+    // be released as soon as this call returns.
+    s = upload_plan(blob.data(), plan_d, ws_d, ws_bytes, stream);
+    if (s != DEFT_OK) return s;
+    return select_rank(acc_d, blob.data(), plan_d, 0, val_d, idx_d, out_cap, ws_d, ws_bytes, stream);
 }
 
 }  // namespace
@@ -89,11 +168,11 @@ extern "C" {
 
 int32_t deft_last_cuda_error(void) { return g_last_cuda_error; }
 
+void deft_debug_select_timing(void* timing_d) { g_select_timing = static_cast<unsigned long long*>(timing_d); }
+
 size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers) {
     if (max_elems < 1 || max_layers < 1) return 0;
-    const SelectWorkspace w =
-        carve_select_ws(nullptr, max_layers, max_tiles(max_elems, max_layers), max_elems);
-    const size_t a = w.total_bytes;
+    const size_t a = ws_layout(max_elems, max_layers, max_tiles(max_elems, max_layers)).total;
     const size_t b = align_up(norms_ws_bytes(max_elems, max_layers), 256);
     return a > b ? a : b;
 }
@@ -110,6 +189,101 @@ deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_
                               static_cast<double*>(ws_d), static_cast<cudaStream_t>(stream));
 }
 
+size_t deft_plan_bytes(int32_t L, int32_t N) {
+    if (L < 1 || N < 1 || N > kMaxRanks) return 0;
+    return plan_bytes(L, N);
+}
+
+deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
+                            const int32_t* bin_of_layer_h, int32_t L, int32_t N, int64_t iteration,
+                            void* plan_h, size_t plan_bytes_cap) {
+    if (!layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || L < 1 || N < 1 || N > kMaxRanks ||
+        iteration < 0)
+        return DEFT_ERR_INVALID_ARG;
+    std::vector<std::vector<LayerItem>> ranks((size_t)N);
+    const int32_t cycle = (int32_t)(iteration % N);
+    for (int32_t l = 0; l < L; ++l) {
+        const int32_t b = bin_of_layer_h[l];
+        if (b < 0 || b >= N) return DEFT_ERR_INVALID_ARG;
+        // rank r reads bin (cycle + r) % N  <=>  bin b is read by rank (b - cycle) mod N
+        const int32_t r = ((b - cycle) % N + N) % N;
+        ranks[r].push_back(LayerItem{layer_start_h[l], layer_start_h[l + 1], k_l_h[l], l});
+    }
+    return fill_plan(plan_h, plan_bytes_cap, L, iteration, ranks);
+}
+
+deft_status deft_plan_rank_info(const void* plan_h, int32_t rank, int32_t* n_layers_out,
+                                int64_t* elems_out, int64_t* k_out, int64_t* out_off_out) {
+    if (!plan_ok(plan_h)) return DEFT_ERR_INVALID_ARG;
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    if (rank < 0 || rank >= hdr->N) return DEFT_ERR_INVALID_ARG;
+    const RankInfo& R = plan_ranks(plan_h)[rank];
+    if (n_layers_out) *n_layers_out = R.n_my;
+    if (elems_out) *elems_out = R.elems;
+    if (k_out) *k_out = R.k;
+    if (out_off_out) *out_off_out = R.out_off;
+    return DEFT_OK;
+}
+
+deft_status deft_plan_rank_table(const void* plan_h, int32_t N, int32_t* n_layers_h, int64_t* elems_h,
+                                 int64_t* k_h, int64_t* out_off_h) {
+    if (!plan_ok(plan_h)) return DEFT_ERR_INVALID_ARG;
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    if (N != hdr->N) return DEFT_ERR_INVALID_ARG;
+    const RankInfo* R = plan_ranks(plan_h);
+    for (int32_t r = 0; r < N; ++r) {
+        if (n_layers_h) n_layers_h[r] = R[r].n_my;
+        if (elems_h) elems_h[r] = R[r].elems;
+        if (k_h) k_h[r] = R[r].k;
+        if (out_off_h) out_off_h[r] = R[r].out_off;
+    }
+    return DEFT_OK;
+}
+
+deft_status deft_plan_upload(const void* plan_h, void* plan_d, void* ws_d, size_t ws_bytes, void* stream) {
+    if (!plan_ok(plan_h) || !plan_d || !ws_d || !aligned16(plan_d) || !aligned256(ws_d))
+        return DEFT_ERR_INVALID_ARG;
+    return upload_plan(plan_h, plan_d, ws_d, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+deft_status deft_select_planned(const float* acc_d, const void* plan_h, const void* plan_d,
+                                int32_t rank, float* val_d, int64_t* idx_d, int64_t out_cap,
+                                void* ws_d, size_t ws_bytes, void* stream) {
+    if (!plan_ok(plan_h) || !plan_d || !acc_d || !ws_d || out_cap < 0) return DEFT_ERR_INVALID_ARG;
+    if (!aligned16(acc_d) || !aligned16(plan_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    if (rank < 0 || rank >= hdr->N) return DEFT_ERR_INVALID_ARG;
+    if (plan_ranks(plan_h)[rank].n_my > 0 && (!val_d || !idx_d)) return DEFT_ERR_INVALID_ARG;
+    return select_rank(acc_d, plan_h, plan_d, rank, val_d, idx_d, out_cap, ws_d, ws_bytes,
+                       static_cast<cudaStream_t>(stream));
+}
+
+deft_status deft_select_update_ranks(float* acc_d, int64_t n_g, const void* plan_h, const void* plan_d,
+                                     int32_t rank_begin, int32_t rank_end, float* val_d, int64_t* idx_d,
+                                     int64_t out_cap, void* ws_d, size_t ws_bytes, void* const* events,
+                                     void* stream) {
+    if (!plan_ok(plan_h) || !plan_d || !acc_d || !ws_d || !val_d || !idx_d || n_g < 1)
+        return DEFT_ERR_INVALID_ARG;
+    if (!aligned16(acc_d) || !aligned16(plan_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    if (rank_begin < 0 || rank_end > hdr->N || rank_begin > rank_end) return DEFT_ERR_INVALID_ARG;
+    if (out_cap < hdr->total_k) return DEFT_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int32_t r = rank_begin; r < rank_end; ++r) {
+        const RankInfo& R = plan_ranks(plan_h)[r];
+        void* const* ev = events ? events + 3 * (size_t)(r - rank_begin) : nullptr;
+        if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[0]), st));
+        deft_status s = select_rank(acc_d, plan_h, plan_d, r, val_d + R.out_off, idx_d + R.out_off, R.k,
+                                    ws_d, ws_bytes, st);
+        if (s != DEFT_OK) return s;
+        if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[1]), st));
+        s = launch_residual_update(acc_d, idx_d + R.out_off, R.k, st);
+        if (s != DEFT_OK) return s;
+        if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[2]), st));
+    }
+    return DEFT_OK;
+}
+
 deft_status deft_select(const float* acc_d, const int64_t* layer_start_h, const int64_t* k_l_h,
                         const int32_t* my_layers_h, int32_t n_my, float* val_d, int64_t* idx_d,
                         int64_t out_cap, void* ws_d, size_t ws_bytes, void* stream) {
@@ -118,13 +292,14 @@ deft_status deft_select(const float* acc_d, const int64_t* layer_start_h, const 
     if (!acc_d || !layer_start_h || !k_l_h || !my_layers_h || !val_d || !idx_d || !ws_d)
         return DEFT_ERR_INVALID_ARG;
     if (!aligned16(acc_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
-    std::vector<LayerDesc> table;
-    int64_t tiles, elems, k_total;
-    const deft_status s =
-        build_rank_table(layer_start_h, k_l_h, my_layers_h, n_my, table, tiles, elems, k_total);
-    if (s != DEFT_OK) return s;
-    return select_common(acc_d, table, n_my, tiles, elems, k_total, val_d, idx_d, out_cap, ws_d,
-                         ws_bytes, static_cast<cudaStream_t>(stream));
+    std::vector<LayerItem> items((size_t)n_my);
+    for (int32_t j = 0; j < n_my; ++j) {
+        const int32_t l = my_layers_h[j];
+        if (l < 0 || (j > 0 && l <= my_layers_h[j - 1])) return DEFT_ERR_INVALID_ARG;
+        items[j] = LayerItem{layer_start_h[l], layer_start_h[l + 1], k_l_h[l], j};
+    }
+    return select_once(acc_d, items, val_d, idx_d, out_cap, ws_d, ws_bytes,
+                       static_cast<cudaStream_t>(stream));
 }
 
 deft_status deft_topk_baseline(const float* acc_d, int64_t n, int64_t k, float* val_d,
@@ -132,14 +307,8 @@ deft_status deft_topk_baseline(const float* acc_d, int64_t n, int64_t k, float* 
     if (!acc_d || !val_d || !idx_d || !ws_d || n < 1 || n > DEFT_MAX_LAYER_ELEMS || k < 1 || k > n)
         return DEFT_ERR_INVALID_ARG;
     if (!aligned16(acc_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
-    const int64_t layer_start[2] = {0, n};
-    const int32_t only = 0;
-    std::vector<LayerDesc> table;
-    int64_t tiles, elems, k_total;
-    const deft_status s = build_rank_table(layer_start, &k, &only, 1, table, tiles, elems, k_total);
-    if (s != DEFT_OK) return s;
-    return select_common(acc_d, table, 1, tiles, elems, k_total, val_d, idx_d, k, ws_d, ws_bytes,
-                         static_cast<cudaStream_t>(stream));
+    std::vector<LayerItem> items(1, LayerItem{0, n, k, 0});
+    return select_once(acc_d, items, val_d, idx_d, k, ws_d, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 deft_status deft_residual_update(float* acc_d, int64_t n_g, const int64_t* idx_d, int64_t count,

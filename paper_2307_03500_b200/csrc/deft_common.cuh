@@ -14,77 +14,124 @@ namespace deft {
 // (multiples of kTile elements from the start of the vector), so that every full tile
 // is read with aligned 128-bit loads whatever the layer boundaries are; the first and
 // last tile of a layer may be partial and are read element-wise under a mask.
+// One warp processes one tile at a time.  Every CTA owns a contiguous run of a rank's
+// tiles; the entries it stages for one layer form one contiguous "run" of the staging stream.
 // ---------------------------------------------------------------------------------
-constexpr int kTile = 4096;      // elements per tile
-constexpr int kThreads = 256;    // threads per CTA in the streaming kernels
-constexpr int kWarps = kThreads / 32;
-constexpr int kSlabs = 4;        // float4 loads per thread per tile (kTile = kThreads*4*kSlabs)
+constexpr int kTile = 2048;          // elements per tile
+constexpr int kSelThreads = 512;     // one persistent CTA per SM (128 registers per thread)
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSlots = 8;            // per-CTA shared-memory histograms live at once
 
 // Radix digits over the 31-bit magnitude key (IEEE bits with the sign cleared):
-// level 1 = bits 30..20 (exponent + 3 mantissa bits), level 2 = bits 19..9, level 3 = bits 8..0.
-constexpr int kBins1 = 2048, kBins2 = 2048, kBins3 = 512;
-constexpr int kShift1 = 20, kShift2 = 9;
+// level 1 = bits 30..19 (exponent + 4 mantissa bits), level 2 = bits 18..9, level 3 = bits 8..0.
+constexpr int kBins1 = 4096, kBins2 = 1024, kBins3 = 512;
+constexpr int kShift1 = 19, kShift2 = 9;
+
+// A layer is "small" when one CTA can finish it from shared memory: at most kSmallTiles
+// chunks and at most kSmallEntries staged entries.  Everything else takes the general path.
+constexpr int kSmallTiles = 4096;
+constexpr int kSmallEntries = 20480;
+
+constexpr int kMaxRanks = 4096;      // workers per plan
 
 // Accumulate+norm geometry.
-constexpr int kTileA = 8192;     // elements per CTA iteration
+constexpr int kNormThreads = 256;
+constexpr int kNormWarps = kNormThreads / 32;
+constexpr int kTileA = 8192;         // elements per CTA iteration
 
-struct LayerDesc {               // one per layer of the rank (+1 sentinel), 48 bytes
-    int64_t start, end;          // element range in the flat vector
-    int64_t k;                   // entries to select (1..size)
-    int64_t out_off;             // position of the layer's first output entry
-    int64_t elem_off;            // elements in the rank's earlier layers (= staging base)
-    int32_t tile_first;          // rank-local id of the layer's first tile
-    int32_t pad;
+// ---------------------------------------------------------------------------------
+// The plan: a position-independent blob built on the host once per step, copied to the
+// device as it is.  [PlanHeader][RankInfo x N][LayerDesc x (L + N)] — each rank's layer
+// list is followed by one sentinel entry.
+// ---------------------------------------------------------------------------------
+constexpr uint32_t kPlanMagic = 0x44454654u;  // "DEFT"
+
+struct PlanHeader {                  // 64 bytes
+    uint32_t magic;
+    int32_t L, N;
+    int32_t total_tiles;
+    int64_t total_elems;             // elements over all ranks' layers
+    int64_t total_k;                 // entries over all ranks
+    int64_t iteration;
+    int64_t reserved[3];
 };
-static_assert(sizeof(LayerDesc) == 48, "LayerDesc layout");
+static_assert(sizeof(PlanHeader) == 64, "PlanHeader layout");
 
-struct LayerState {              // written by the scan kernels, 32 bytes
-    uint32_t b1, krem1;          // level-1 bucket of the k-th key; how many still to take inside it
-    uint32_t b2, krem2;          // same for level 2 (inside bucket b1)
-    uint32_t T, need;            // exact threshold key; how many entries equal to T to take
-    uint32_t pad0, pad1;
+struct RankInfo {                    // 64 bytes
+    int32_t desc_first;              // index of the rank's first LayerDesc
+    int32_t n_my;                    // layers of the rank
+    int32_t tiles;                   // tiles (= chunks) of the rank
+    int32_t tile_base;               // first chunk of the rank in the chunk arrays
+    int64_t elems;                   // elements the rank scans
+    int64_t k;                       // entries the rank selects
+    int64_t out_off;                 // sum of k over lower ranks
+    int64_t elem_base;               // first staging entry of the rank
+    int64_t reserved[2];
+};
+static_assert(sizeof(RankInfo) == 64, "RankInfo layout");
+
+struct LayerDesc {                   // 64 bytes
+    int64_t start, end;              // element range in the flat vector
+    int64_t k;                       // entries to select (1..size)
+    int64_t out_off;                 // position of the layer's first output entry within the rank
+    int64_t elem_off;                // absolute staging index of the layer's first slot
+    int32_t tile_first;              // rank-local id of the layer's first tile
+    int32_t layer_id;                // id in the model's layer table (state / histogram index)
+    int64_t reserved[2];
+};
+static_assert(sizeof(LayerDesc) == 64, "LayerDesc layout");
+
+inline size_t plan_bytes(int64_t L, int64_t N) {
+    return sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)N + sizeof(LayerDesc) * (size_t)(L + N);
+}
+inline const RankInfo* plan_ranks(const void* plan) {
+    return reinterpret_cast<const RankInfo*>(static_cast<const char*>(plan) + sizeof(PlanHeader));
+}
+inline const LayerDesc* plan_descs(const void* plan, int64_t N) {
+    return reinterpret_cast<const LayerDesc*>(static_cast<const char*>(plan) + sizeof(PlanHeader) +
+                                              sizeof(RankInfo) * (size_t)N);
+}
+
+struct LayerState {                  // per layer, written by the kernels; 32 bytes
+    uint32_t b1, above1;             // level-1 bucket of the k-th key; keys strictly above that bucket
+    uint32_t cand1, big;             // keys inside bucket b1; 1 = layer takes the general path
+    uint32_t b2, krem2;              // level 2 (inside b1): bucket, and how many still to take inside it
+    uint32_t T, need;                // exact threshold key; entries equal to T to take (lowest indices)
 };
 static_assert(sizeof(LayerState) == 32, "LayerState layout");
 
-struct SelectWorkspace {         // carve-up of the caller's workspace for one selection call
-    LayerDesc* desc;             // [n_my + 1]
-    LayerState* state;           // [n_my]            \  zeroed
-    uint32_t* hist1;             // [n_my][kBins1]     | at the start
-    uint32_t* hist2;             // [n_my][kBins2]     | of every
-    uint32_t* hist3;             // [n_my][kBins3]    /  call
-    size_t zero_bytes;           // bytes from `state` to the end of hist3
-    uint32_t* cnt;               // [tiles] staged entries per tile
-    uint2* ge;                   // [tiles] (#key > T, #key == T) per tile, then their exclusive scans
-    uint2* staging;              // [n_r]   (value bits, offset in tile) of every entry with key >= bucket b1
-    size_t total_bytes;
+struct RankFlags {
+    uint32_t any_big;                // some layer of the rank takes the general path
+    uint32_t error;                  // reserved for kernel-side consistency checks
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-inline SelectWorkspace carve_select_ws(void* base, int64_t n_my, int64_t tiles, int64_t elems) {
-    SelectWorkspace w{};
+// Carve-up of the caller's workspace.  Offsets depend only on (elems, L, tiles).
+struct WsLayout {
+    size_t plan;                     // scratch device plan for the one-shot calls
+    size_t zero_begin, zero_end;     // [state | flags | hist1 | hist2 | hist3]: cleared at plan upload
+    size_t state, flags, hist1, hist2, hist3;
+    size_t cnt, ge, staging;
+    size_t total;
+};
+
+inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
+    WsLayout w{};
     size_t off = 0;
-    char* p = static_cast<char*>(base);
-    w.desc = reinterpret_cast<LayerDesc*>(p + off);
-    off = align_up(off + sizeof(LayerDesc) * (size_t)(n_my + 1), 256);
-    const size_t z0 = off;
-    w.state = reinterpret_cast<LayerState*>(p + off);
-    off = align_up(off + sizeof(LayerState) * (size_t)n_my, 256);
-    w.hist1 = reinterpret_cast<uint32_t*>(p + off);
-    off += sizeof(uint32_t) * (size_t)n_my * kBins1;
-    w.hist2 = reinterpret_cast<uint32_t*>(p + off);
-    off += sizeof(uint32_t) * (size_t)n_my * kBins2;
-    w.hist3 = reinterpret_cast<uint32_t*>(p + off);
-    off += sizeof(uint32_t) * (size_t)n_my * kBins3;
-    w.zero_bytes = off - z0;
-    off = align_up(off, 256);
-    w.cnt = reinterpret_cast<uint32_t*>(p + off);
-    off = align_up(off + sizeof(uint32_t) * (size_t)tiles, 256);
-    w.ge = reinterpret_cast<uint2*>(p + off);
-    off = align_up(off + sizeof(uint2) * (size_t)tiles, 256);
-    w.staging = reinterpret_cast<uint2*>(p + off);
-    off = align_up(off + sizeof(uint2) * (size_t)elems, 256);
-    w.total_bytes = off;
+    w.plan = off;     off += align_up(plan_bytes(L, 1), 256);
+    w.zero_begin = off;
+    w.state = off;    off += align_up(sizeof(LayerState) * (size_t)L, 256);
+    w.flags = off;    off += align_up(sizeof(RankFlags) * (size_t)kMaxRanks, 256);
+    w.hist1 = off;    off += sizeof(uint32_t) * (size_t)kBins1 * (size_t)L;
+    w.hist2 = off;    off += sizeof(uint32_t) * (size_t)kBins2 * (size_t)L;
+    w.hist3 = off;    off += sizeof(uint32_t) * (size_t)kBins3 * (size_t)L;
+    w.zero_end = off;
+    const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
+    w.cnt = off;      off += align_up(sizeof(uint32_t) * slots, 256);
+    w.ge = off;       off += align_up(sizeof(uint2) * slots, 256);
+    w.staging = off;  off += align_up(sizeof(uint2) * (size_t)elems, 256);
+    w.total = off;
     return w;
 }
 
@@ -94,6 +141,24 @@ inline int64_t max_tiles(int64_t elems, int64_t layers) { return elems / kTile +
 inline size_t norms_ws_bytes(int64_t n_g, int64_t L) {
     return sizeof(double) * (size_t)((n_g + kTileA - 1) / kTileA + L + 1);
 }
+
+// Arguments of the fused selection kernel (one rank).
+struct SelParams {
+    const float* acc;
+    const LayerDesc* desc;           // the rank's layers + sentinel (device)
+    int32_t n_my, tiles;
+    LayerState* state;               // [L]
+    RankFlags* flags;                // this rank's flags
+    uint32_t* hist1;                 // [L][kBins1]
+    uint32_t* hist2;                 // [L][kBins2]
+    uint32_t* hist3;                 // [L][kBins3]
+    uint32_t* runcnt;                // this rank's runs (slot = CTA + layer position): staged entries
+    uint2* runge;                    // this rank's runs: (#key > T, #key == T), then exclusive scans
+    uint2* staging;                  // absolute base; (value bits, offset from the run's first tile)
+    float* val;                      // the rank's output
+    int64_t* idx;
+    unsigned long long* timing;      // optional: 16 phase timestamps (ns, max over CTAs); NULL = off
+};
 
 // Sticky per-thread CUDA error code for deft_last_cuda_error().
 void set_last_cuda_error(cudaError_t e);
@@ -112,8 +177,7 @@ int sm_count();
 deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_g,
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
                                double* partial_d, cudaStream_t stream);
-deft_status launch_select(const float* acc_d, const SelectWorkspace& w, int32_t n_my, int32_t tiles,
-                          float* val_d, int64_t* idx_d, cudaStream_t stream);
+deft_status launch_select(const SelParams& p, cudaStream_t stream);
 deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t count,
                                    cudaStream_t stream);
 

@@ -4,7 +4,10 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
+#include <functional>
 #include <numeric>
+#include <queue>
+#include <utility>
 #include <vector>
 
 #include "deft.h"
@@ -150,20 +153,23 @@ deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, in
 
     std::vector<double> c(L);
     for (int32_t l = 0; l < L; ++l) c[l] = (double)layer_size_h[l] * std::log((double)k_l_h[l]);
-    std::vector<char> placed(L, 0);
+    // "largest remaining cost, lowest id on ties" L times = one stable pass over the layers
+    // sorted by descending cost; "smallest load, lowest id on ties" = a min-heap on (load, bin).
+    // Each bin receives its costs in the same order as in the listing, so the fp64 sums are the same.
+    std::vector<int32_t> by_cost(L);
+    std::iota(by_cost.begin(), by_cost.end(), 0);
+    std::stable_sort(by_cost.begin(), by_cost.end(), [&c](int32_t a, int32_t b) { return c[a] > c[b]; });
     std::vector<double> load(N, 0.0);
-    for (int32_t round = 0; round < L; ++round) {
-        int32_t pick = -1;
-        for (int32_t l = 0; l < L; ++l) {
-            if (placed[l]) continue;
-            if (pick < 0 || c[l] > c[pick]) pick = l;
-        }
-        int32_t lightest = 0;
-        for (int32_t b = 1; b < N; ++b)
-            if (load[b] < load[lightest]) lightest = b;
-        bin_of_layer_h[pick] = lightest;
-        load[lightest] += c[pick];
-        placed[pick] = 1;
+    typedef std::pair<double, int32_t> Bin;   // (load, id): smallest load first, then lowest id
+    std::priority_queue<Bin, std::vector<Bin>, std::greater<Bin>> heap;
+    for (int32_t b = 0; b < N; ++b) heap.push(Bin(0.0, b));
+    for (int32_t i = 0; i < L; ++i) {
+        const int32_t pick = by_cost[i];
+        const Bin lightest = heap.top();
+        heap.pop();
+        bin_of_layer_h[pick] = lightest.second;
+        load[lightest.second] += c[pick];
+        heap.push(Bin(load[lightest.second], lightest.second));
     }
     if (bin_load_h)
         for (int32_t b = 0; b < N; ++b) bin_load_h[b] = load[b];

@@ -28,7 +28,7 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
     double t = 0.0;
     if (threadIdx.x == 0) {
 #pragma unroll
-        for (int i = 0; i < kWarps; ++i) t += sh[i];
+        for (int i = 0; i < kNormWarps; ++i) t += sh[i];
     }
     return t;
 }
@@ -44,10 +44,10 @@ __device__ __forceinline__ int layer_of(const int64_t* __restrict__ ls, int L, i
 }
 
 template <bool kHasGrad>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kNormThreads)
 k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
               const int64_t* __restrict__ ls, int L, double* __restrict__ partial, int64_t tiles) {
-    __shared__ double sh[kWarps];
+    __shared__ double sh[kNormWarps];
     for (int64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
         const int64_t lo = t * kTileA;
         const int64_t hi = (lo + kTileA < n) ? lo + kTileA : n;
@@ -58,8 +58,8 @@ k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
             const float4* g4 = reinterpret_cast<const float4*>(g + lo);
             double acc = 0.0;
 #pragma unroll
-            for (int i = 0; i < kTileA / (kThreads * 4); i += 2) {
-                const int a = i * kThreads + threadIdx.x, b = a + kThreads;
+            for (int i = 0; i < kTileA / (kNormThreads * 4); i += 2) {
+                const int a = i * kNormThreads + threadIdx.x, b = a + kNormThreads;
                 float4 x = e4[a], y = e4[b];
                 if (kHasGrad) {
                     const float4 gx = __ldg(g4 + a), gy = __ldg(g4 + b);
@@ -85,7 +85,7 @@ k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
                 const int64_t lend = __ldg(ls + l + 1);
                 const int64_t pe = lend < hi ? lend : hi;
                 double acc = 0.0;
-                for (int64_t i = ps + threadIdx.x; i < pe; i += kThreads) {
+                for (int64_t i = ps + threadIdx.x; i < pe; i += kNormThreads) {
                     float x = e[i];
                     if (kHasGrad) {
                         x = __fadd_rn(x, __ldg(g + i));
@@ -103,16 +103,16 @@ k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
 }
 
 // One CTA per layer: add the layer's partial sums in a fixed order, take the root.
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kNormThreads)
 k_norm_finalize(const int64_t* __restrict__ ls, int L, const double* __restrict__ partial,
                 double* __restrict__ norms) {
-    __shared__ double sh[kWarps];
+    __shared__ double sh[kNormWarps];
     const int l = blockIdx.x;
     const int64_t s = ls[l], e = ls[l + 1];
     double acc = 0.0;
     if (e > s) {
         const int64_t t0 = s / kTileA, t1 = (e - 1) / kTileA;
-        for (int64_t t = t0 + threadIdx.x; t <= t1; t += kThreads) acc += partial[t + l];
+        for (int64_t t = t0 + threadIdx.x; t <= t1; t += kNormThreads) acc += partial[t + l];
     }
     const double tot = block_sum(acc, sh);
     if (threadIdx.x == 0) norms[l] = sqrt(tot);
@@ -127,13 +127,13 @@ deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t 
     const int64_t max_grid = (int64_t)sm_count() * 8;
     const int grid = (int)(tiles < max_grid ? tiles : max_grid);
     if (grad_d)
-        k_accum_norms<true><<<grid, kThreads, 0, stream>>>(resid_acc_d, grad_d, n_g, layer_start_d,
+        k_accum_norms<true><<<grid, kNormThreads, 0, stream>>>(resid_acc_d, grad_d, n_g, layer_start_d,
                                                            L, partial_d, tiles);
     else
-        k_accum_norms<false><<<grid, kThreads, 0, stream>>>(resid_acc_d, nullptr, n_g,
+        k_accum_norms<false><<<grid, kNormThreads, 0, stream>>>(resid_acc_d, nullptr, n_g,
                                                             layer_start_d, L, partial_d, tiles);
     DEFT_CUDA_TRY(cudaGetLastError());
-    k_norm_finalize<<<L, kThreads, 0, stream>>>(layer_start_d, L, partial_d, norms_d);
+    k_norm_finalize<<<L, kNormThreads, 0, stream>>>(layer_start_d, L, partial_d, norms_d);
     DEFT_CUDA_TRY(cudaGetLastError());
     return DEFT_OK;
 }

@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
         L.deft_status_string.argtypes = [i32]
         L.deft_last_cuda_error.restype = i32
         L.deft_last_cuda_error.argtypes = []
+        L.deft_debug_select_timing.restype = None
+        L.deft_debug_select_timing.argtypes = [vp]
         L.deft_split_layers.restype = i32
         L.deft_split_layers.argtypes = [vp, i32, i32, vp, vp, i32, vp]
         L.deft_allocate_k.restype = i32
@@ -66,6 +68,20 @@ def lib() -> ctypes.CDLL:
         L.deft_layer_norms.argtypes = [vp, vp, i64, vp, i32, vp, vp, sz, vp]
         L.deft_select.restype = i32
         L.deft_select.argtypes = [vp, vp, vp, vp, i32, vp, vp, i64, vp, sz, vp]
+        L.deft_plan_bytes.restype = sz
+        L.deft_plan_bytes.argtypes = [i32, i32]
+        L.deft_plan_build.restype = i32
+        L.deft_plan_build.argtypes = [vp, vp, vp, i32, i32, i64, vp, sz]
+        L.deft_plan_rank_info.restype = i32
+        L.deft_plan_rank_info.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.deft_plan_rank_table.restype = i32
+        L.deft_plan_rank_table.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.deft_plan_upload.restype = i32
+        L.deft_plan_upload.argtypes = [vp, vp, vp, sz, vp]
+        L.deft_select_planned.restype = i32
+        L.deft_select_planned.argtypes = [vp, vp, vp, i32, vp, vp, i64, vp, sz, vp]
+        L.deft_select_update_ranks.restype = i32
+        L.deft_select_update_ranks.argtypes = [vp, i64, vp, vp, i32, i32, vp, vp, i64, vp, sz, vp, vp]
         L.deft_residual_update.restype = i32
         L.deft_residual_update.argtypes = [vp, i64, vp, i64, vp]
         L.deft_topk_baseline.restype = i32
@@ -217,6 +233,97 @@ def deft_select(acc, layer_start_h, k_l_h, my_layers_h, val_d, idx_d, ws, stream
                              _dp(val_d, torch.float32), _dp(idx_d, torch.int64), cap, _dp(ws),
                              ws.numel() * ws.element_size(), _stream(stream)))
     return int(kl[my].sum()) if my.size else 0
+
+
+def deft_debug_select_timing(timing_d) -> None:
+    """Diagnostic phase stamps of the selection kernel: a zeroed CUDA uint64/int64 tensor of 16, or None."""
+    lib().deft_debug_select_timing(None if timing_d is None else _dp(timing_d))
+
+
+def deft_plan_bytes(n_layers: int, n_workers: int) -> int:
+    return int(lib().deft_plan_bytes(int(n_layers), int(n_workers)))
+
+
+def deft_plan_build(layer_start_h, k_l_h, bin_of_layer_h, n_workers: int, iteration: int,
+                    out: Optional[np.ndarray] = None) -> np.ndarray:
+    """Builds the step's plan blob on the host.  ``out`` may be a uint8 numpy view of pinned memory."""
+    ls = _np(layer_start_h, np.int64)
+    kl = _np(k_l_h, np.int64)
+    bins = _np(bin_of_layer_h, np.int32)
+    L = kl.size
+    if ls.size != L + 1 or bins.size != L:
+        raise ValueError("layer_start_h, k_l_h and bin_of_layer_h disagree")
+    need = deft_plan_bytes(L, n_workers)
+    if need == 0:
+        raise DeftError("deft_plan_bytes", ERR_INVALID_ARG)
+    if out is None:
+        out = np.empty(need, dtype=np.uint8)
+    if out.dtype != np.uint8 or not out.flags.c_contiguous or out.size < need:
+        raise ValueError("plan buffer must be contiguous uint8 of at least %d bytes" % need)
+    _check("deft_plan_build", lib().deft_plan_build(_hp(ls), _hp(kl), _hp(bins), L, int(n_workers), int(iteration),
+                                                    _hp(out), out.size))
+    return out
+
+
+def deft_plan_rank_info(plan_h: np.ndarray, rank: int) -> Tuple[int, int, int, int]:
+    """(layers, elements scanned, entries selected, sum of k over lower ranks) of one rank."""
+    n = ctypes.c_int32(0)
+    e, k, o = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+    _check("deft_plan_rank_info", lib().deft_plan_rank_info(_hp(plan_h), int(rank), ctypes.byref(n), ctypes.byref(e),
+                                                            ctypes.byref(k), ctypes.byref(o)))
+    return int(n.value), int(e.value), int(k.value), int(o.value)
+
+
+def deft_plan_rank_table(plan_h: np.ndarray, n_workers: int):
+    """(layers int32[N], elements int64[N], entries int64[N], output offsets int64[N]) of all ranks."""
+    n = np.zeros(n_workers, dtype=np.int32)
+    e = np.zeros(n_workers, dtype=np.int64)
+    k = np.zeros(n_workers, dtype=np.int64)
+    o = np.zeros(n_workers, dtype=np.int64)
+    _check("deft_plan_rank_table", lib().deft_plan_rank_table(_hp(plan_h), int(n_workers), _hp(n), _hp(e), _hp(k),
+                                                              _hp(o)))
+    return n, e, k, o
+
+
+def deft_plan_upload(plan_h: np.ndarray, plan_d, ws, stream=None) -> None:
+    if plan_d.numel() * plan_d.element_size() < plan_h.size:
+        raise ValueError("plan_d smaller than the plan")
+    _check("deft_plan_upload", lib().deft_plan_upload(_hp(plan_h), _dp(plan_d), _dp(ws),
+                                                      ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_select_planned(acc, plan_h: np.ndarray, plan_d, rank: int, val_d, idx_d, ws, stream=None) -> None:
+    """Algorithm 5 for one rank of an uploaded plan (one kernel launch)."""
+    import torch
+    cap = min(val_d.numel(), idx_d.numel())
+    _check("deft_select_planned",
+           lib().deft_select_planned(_dp(acc, torch.float32), _hp(plan_h), _dp(plan_d), int(rank),
+                                     _dp(val_d, torch.float32) if cap else None,
+                                     _dp(idx_d, torch.int64) if cap else None, cap, _dp(ws),
+                                     ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_select_update_ranks(acc, plan_h: np.ndarray, plan_d, rank_begin: int, rank_end: int, val_d, idx_d, ws,
+                             events=None, stream=None) -> None:
+    """Selection + residual update for a range of simulated ranks (one C call).
+    events: optional list of (before, between, after) torch.cuda.Event triples, one per rank."""
+    import torch
+    ev = None
+    if events is not None:
+        if len(events) != rank_end - rank_begin:
+            raise ValueError("one event triple per rank expected")
+        flat = []
+        for tri in events:
+            for e in tri:
+                if e.cuda_event == 0:   # torch creates the handle lazily, on first record
+                    e.record()
+                flat.append(e.cuda_event)
+        ev = (ctypes.c_void_p * len(flat))(*flat)
+    _check("deft_select_update_ranks",
+           lib().deft_select_update_ranks(_dp(acc, torch.float32), acc.numel(), _hp(plan_h), _dp(plan_d),
+                                          int(rank_begin), int(rank_end), _dp(val_d, torch.float32),
+                                          _dp(idx_d, torch.int64), min(val_d.numel(), idx_d.numel()), _dp(ws),
+                                          ws.numel() * ws.element_size(), ev, _stream(stream)))
 
 
 def deft_residual_update(acc, idx_d, count: int, stream=None) -> None:

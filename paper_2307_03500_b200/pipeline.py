@@ -24,10 +24,11 @@ class StepPlan:
     sum_k: int
     bin_of_layer: np.ndarray   # int32[L]
     bin_load: np.ndarray       # float64[N]  (Eq. 4 per bin)
-    rank_layers: List[np.ndarray]   # per rank: ascending layer ids
+    rank_layers_n: np.ndarray  # int32[N]  layers of each rank
     rank_k: np.ndarray         # int64[N]  entries each rank selects
     rank_elems: np.ndarray     # int64[N]  elements each rank scans
     rank_out_off: np.ndarray   # int64[N+1] offsets into the output slabs
+    plan_h: np.ndarray         # the uploaded plan blob (host copy)
 
 
 class DeftStep:
@@ -51,6 +52,10 @@ class DeftStep:
         cap = self.k + self.L + 64   # PAPER mode may overshoot by at most one per layer
         self.val_d = torch.empty(cap, dtype=torch.float32, device=self.device)
         self.idx_d = torch.empty(cap, dtype=torch.int64, device=self.device)
+        nbytes = deft.deft_plan_bytes(self.L, self.N)
+        self._plan_pin = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+        self.plan_h = self._plan_pin.numpy()
+        self.plan_d = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
 
     # -- step 1: accumulate + norms (device) ------------------------------------------------
     def layer_norms(self, resid: torch.Tensor, grad: Optional[torch.Tensor]) -> np.ndarray:
@@ -61,35 +66,45 @@ class DeftStep:
 
     # -- steps 2 and 3: local k and bins (host) ---------------------------------------------
     def plan(self, norms: np.ndarray, iteration: int = 0) -> StepPlan:
+        """Algorithm 3, Algorithm 4, then the plan of all N ranks built on the host and uploaded."""
         k_l, sum_k, _ = deft.deft_allocate_k(norms, self.layer_size, self.k, self.mode)
         bins, load = deft.deft_partition(self.layer_size, k_l, self.N)
-        rank_layers = [deft.deft_bin_layers(bins, deft.deft_rank_bin(iteration, r, self.N)) for r in range(self.N)]
-        rank_k = np.array([int(k_l[m].sum()) for m in rank_layers], dtype=np.int64)
-        rank_elems = np.array([int(self.layer_size[m].sum()) for m in rank_layers], dtype=np.int64)
+        deft.deft_plan_build(self.layer_start, k_l, bins, self.N, iteration, out=self.plan_h)
+        deft.deft_plan_upload(self.plan_h, self.plan_d, self.ws)
+        n_layers, elems, rank_k, out_off = deft.deft_plan_rank_table(self.plan_h, self.N)
         off = np.zeros(self.N + 1, dtype=np.int64)
-        np.cumsum(rank_k, out=off[1:])
-        return StepPlan(k_l, sum_k, bins, load, rank_layers, rank_k, rank_elems, off)
+        off[:-1] = out_off
+        off[-1] = out_off[-1] + rank_k[-1]
+        return StepPlan(k_l, sum_k, bins, load, n_layers, rank_k, elems, off, self.plan_h)
+
+    def rank_layers(self, plan: StepPlan, iteration: int, rank: int) -> np.ndarray:
+        return deft.deft_bin_layers(plan.bin_of_layer, deft.deft_rank_bin(iteration, rank, self.N))
 
     # -- step 4: selection + residual update for one rank (device) --------------------------
     def select_rank(self, acc: torch.Tensor, plan: StepPlan, rank: int):
         a, b = int(plan.rank_out_off[rank]), int(plan.rank_out_off[rank + 1])
         val, idx = self.val_d[a:b], self.idx_d[a:b]
         if b > a:
-            deft.deft_select(acc, self.layer_start, plan.k_l, plan.rank_layers[rank], val, idx, self.ws)
+            deft.deft_select_planned(acc, plan.plan_h, self.plan_d, rank, val, idx, self.ws)
         return val, idx
+
+    def select_and_update_all(self, acc: torch.Tensor, plan: StepPlan, events=None) -> None:
+        """Selection followed by the residual update for every simulated rank, rank after rank (one C call).
+        `events`: optional list of (before, between, after) CUDA events per rank, recorded on the stream."""
+        deft.deft_select_update_ranks(acc, plan.plan_h, self.plan_d, 0, self.N, self.val_d, self.idx_d, self.ws,
+                                      events)
 
     def residual_update(self, acc: torch.Tensor, idx: torch.Tensor) -> None:
         deft.deft_residual_update(acc, idx, idx.numel())
 
     # -- the whole step for all simulated ranks ---------------------------------------------
-    def step(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0):
+    def step(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, events=None):
+        """accumulate + norms -> plan -> (selection, residual update) for every rank.  Returns the plan and,
+        per rank, views of its selected (values, indices)."""
         norms = self.layer_norms(resid, grad)
         plan = self.plan(norms, iteration)
-        outs = []
-        for r in range(self.N):
-            val, idx = self.select_rank(resid, plan, r)
-            outs.append((val, idx))
-        # all ranks read the same accumulated vector, so zeroing starts after the last selection
-        for val, idx in outs:
-            self.residual_update(resid, idx)
+        self.select_and_update_all(resid, plan, events)
+        off = plan.rank_out_off
+        outs = [(self.val_d[int(off[r]):int(off[r + 1])], self.idx_d[int(off[r]):int(off[r + 1])])
+                for r in range(self.N)]
         return plan, outs

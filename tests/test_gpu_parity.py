@@ -130,7 +130,7 @@ def _whole_path(deft, w, steps=1, mode=None, iteration=0):
         all_idx = []
         for r in range(N):
             my = oracle.my_layers(bins, iteration + t, r, N)
-            assert plan.rank_layers[r].tolist() == my.tolist()
+            assert ds.rank_layers(plan, iteration + t, r).tolist() == my.tolist()
             val_d, idx_d = ds.select_rank(e_gpu, plan, r)
             torch.cuda.synchronize()
             want_val, want_idx = oracle.select_rank(e_cpu, start, k_l, my)

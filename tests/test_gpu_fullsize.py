@@ -1,0 +1,115 @@
+"""Parity at the benchmark's full size and launch configuration (BERT-large-shaped vector,
+N = 32 simulated workers, d = 0.001, the per-step plan and the C rank loop bench.py times).
+
+The oracle cannot sort 333 M elements in a test, so: norms, k_l and bins are compared in full;
+selections are compared element by element on sampled layers (one of the largest, a
+mid-sized one, a few small ones), and on EVERY layer through properties that pin the result
+uniquely: count = k_l, strictly ascending indices inside the layer, values are the vector's
+entries, every magnitude above the smallest selected one is selected, and among entries equal
+to it exactly the lowest indices are taken.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2307_03500_b200 import build as deft_build
+from paper_2307_03500_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def deft():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    deft_build.build()
+    from paper_2307_03500_b200 import deft as d
+    d.lib()
+    return d
+
+
+def _check_layer_properties(keys, acc, st, en, k, idx, val):
+    assert idx.size == k
+    assert idx[0] >= st and idx[-1] < en and (k == 1 or np.all(np.diff(idx) > 0))
+    assert val.tobytes() == acc[idx].tobytes()
+    lk = keys[st:en]
+    sk = keys[idx]
+    T = sk.min()
+    n_gt = int((lk > T).sum())
+    assert n_gt == int((sk > T).sum()) and n_gt < k          # everything larger is selected
+    need = k - n_gt
+    ties = np.nonzero(lk == T)[0][:need] + st                 # the lowest-index entries equal to T
+    assert np.array_equal(idx[sk == T], ties)
+
+
+def test_bench_configuration_full_size(deft):
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.bert_large()
+    N = w.n_workers
+    g = w.gradient(0)
+    ds = DeftStep(w.sizes, N, w.density)
+    e_d = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+    g_d = torch.from_numpy(g).cuda()
+    plan, outs = ds.step(e_d, g_d, iteration=0)
+    torch.cuda.synchronize()
+    val_all = ds.val_d[: plan.sum_k].cpu().numpy()
+    idx_all = ds.idx_d[: plan.sum_k].cpu().numpy()
+    resid = e_d.cpu().numpy()
+    del g_d
+
+    start, _ = oracle.split_layers(w.sizes, N)
+    size = np.diff(start)
+    assert ds.layer_start.tolist() == start.tolist()
+    # step 1: acc = 0 + g in fp32 (this turns -0.0 into +0.0); norms against fp64
+    g = oracle.accumulate(np.zeros(w.n_g, dtype=np.float32), g)
+    norms = oracle.layer_norms(g, start)
+    got = ds.norms_h.numpy()
+    assert np.all(np.abs(got - norms) <= 1e-5 * norms)
+    # steps 2, 3: identical norms in -> identical k_l and bins out
+    k_l, s = oracle.allocate_k(got, size, ds.k, oracle.MODE_EXACT)
+    bins, load = oracle.partition(size, k_l, N)
+    assert plan.k_l.tolist() == k_l.tolist() and s == plan.sum_k == ds.k == w.k
+    assert plan.bin_of_layer.tolist() == bins.tolist() and plan.bin_load.tobytes() == load.tobytes()
+
+    # step 4: every layer through properties, sampled layers element by element
+    keys = g.view(np.uint32) & np.uint32(0x7FFFFFFF)
+    order = np.argsort(size)
+    sampled = {int(order[-1]), int(order[len(order) // 2]), int(order[0]), int(order[1]), int(order[5])}
+    seen_layers = []
+    for r in range(N):
+        my = oracle.my_layers(bins, 0, r, N)
+        a, b = int(plan.rank_out_off[r]), int(plan.rank_out_off[r + 1])
+        assert b - a == int(k_l[my].sum())
+        pos = a
+        for l in my:
+            kk = int(k_l[l])
+            idx, val = idx_all[pos:pos + kk], val_all[pos:pos + kk]
+            _check_layer_properties(keys, g, int(start[l]), int(start[l + 1]), kk, idx, val)
+            if int(l) in sampled:
+                want_val, want_idx = oracle.select_layer(g, int(start[l]), int(start[l + 1]), kk)
+                assert np.array_equal(idx, want_idx) and val.tobytes() == want_val.tobytes()
+            pos += kk
+            seen_layers.append(int(l))
+        assert pos == b
+    assert sorted(seen_layers) == list(range(size.size))                  # partitions disjoint, cover all
+    assert np.unique(idx_all).size == plan.sum_k                          # union has exactly k entries
+
+    # step 5: selected entries are +0, everything else untouched
+    want = g.copy()
+    want[idx_all] = 0.0
+    assert resid.tobytes() == want.tobytes()
+
+
+def test_topk_baseline_full_size(deft):
+    w = W.gpt2_medium(1, 0.001)
+    g = w.gradient(0)
+    k = w.k
+    acc_d = torch.from_numpy(g).cuda()
+    ws = deft.alloc_workspace(w.n_g, 1)
+    val_d = torch.empty(k, dtype=torch.float32, device="cuda")
+    idx_d = torch.empty(k, dtype=torch.int64, device="cuda")
+    deft.deft_topk_baseline(acc_d, k, val_d, idx_d, ws)
+    torch.cuda.synchronize()
+    keys = g.view(np.uint32) & np.uint32(0x7FFFFFFF)
+    _check_layer_properties(keys, g, 0, w.n_g, k, idx_d.cpu().numpy(), val_d.cpu().numpy())

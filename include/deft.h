@@ -183,6 +183,30 @@ DEFT_API deft_status deft_select(const float* acc_d, const int64_t* layer_start_
                         int64_t out_cap, void* ws_d, size_t ws_bytes, void* stream);
 
 /*
+ * deft_layer_norms for callers that cannot allocate device memory (no counterpart in the
+ * paper; a deployment variant of the call above).  Some hosts of this library — a
+ * communication hook that runs inside another framework's captured or memory-pooled
+ * region, a plugin that is handed tensors but no allocator, code that runs after the
+ * memory budget has been handed out — may not call cudaMalloc or any allocating routine,
+ * so they have no workspace to pass.  This entry point takes none: its scratch (the
+ * per-tile partial sums) is a fixed 128 KB array inside the library's device image.
+ * Same arguments, same results (bit for bit) as deft_layer_norms.
+ * Limit: ceil(n_g / 8192) + L + 1 must not exceed deft_layer_norms_static_max_slots()
+ * (16384; about 100 M elements with a few thousand layers); larger inputs return
+ * DEFT_ERR_CAPACITY and nothing is launched.
+ * The first call on each device looks up the array's device address (a host-side query,
+ * no allocation); make that first call outside of any stream capture.  All calls on one
+ * device share the array, which keeps whatever the last call left in it; nothing in it has
+ * to be cleared because every slot a call reads it has written first, but two calls that
+ * overlap on the same GPU (different streams) race on it and must be serialised by the caller.
+ * Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+DEFT_API int64_t deft_layer_norms_static_max_slots(void);
+DEFT_API deft_status deft_layer_norms_static(float* resid_acc_d, const float* grad_d, int64_t n_g,
+                                             const int64_t* layer_start_d, int32_t L, double* norms_d,
+                                             void* stream);
+
+/*
  * The per-step plan — Algorithm 4, lines 1-2 and 20 for every rank at once.
  * Once k_l (Algorithm 3) and the bins (Algorithm 4) of a step are known, the layer
  * lists of all N ranks are laid out in one position-independent blob: rank r owns the

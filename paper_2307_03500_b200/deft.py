@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
         L.deft_workspace_bytes.argtypes = [i64, i32]
         L.deft_layer_norms.restype = i32
         L.deft_layer_norms.argtypes = [vp, vp, i64, vp, i32, vp, vp, sz, vp]
+        L.deft_layer_norms_static_max_slots.restype = i64
+        L.deft_layer_norms_static_max_slots.argtypes = []
+        L.deft_layer_norms_static.restype = i32
+        L.deft_layer_norms_static.argtypes = [vp, vp, i64, vp, i32, vp, vp]
         L.deft_select.restype = i32
         L.deft_select.argtypes = [vp, vp, vp, vp, i32, vp, vp, i64, vp, sz, vp]
         L.deft_plan_bytes.restype = sz
@@ -215,6 +219,22 @@ def deft_layer_norms(resid_acc, grad, layer_start_d, norms_d, ws, stream=None) -
            lib().deft_layer_norms(_dp(resid_acc, torch.float32), _dp(grad, torch.float32), n_g,
                                   _dp(layer_start_d, torch.int64), L, _dp(norms_d, torch.float64),
                                   _dp(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_layer_norms_static(resid_acc, grad, layer_start_d, norms_d, stream=None) -> None:
+    """deft_layer_norms without a workspace, for callers that may not allocate device memory: the scratch is a
+    fixed array inside the library (limit: ceil(n_g/8192) + L + 1 <= deft_layer_norms_static_max_slots())."""
+    import torch
+    n_g = resid_acc.numel()
+    L = layer_start_d.numel() - 1
+    if grad is not None and grad.numel() != n_g:
+        raise ValueError("grad and resid_acc differ in length")
+    if norms_d.numel() < L:
+        raise ValueError("norms_d too small")
+    _check("deft_layer_norms_static",
+           lib().deft_layer_norms_static(_dp(resid_acc, torch.float32), _dp(grad, torch.float32), n_g,
+                                         _dp(layer_start_d, torch.int64), L, _dp(norms_d, torch.float64),
+                                         _stream(stream)))
 
 
 def deft_select(acc, layer_start_h, k_l_h, my_layers_h, val_d, idx_d, ws, stream=None) -> int:

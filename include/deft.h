@@ -171,7 +171,10 @@ DEFT_API deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, i
  * index — signed values and int64 indices — exactly sum of k_l of them.
  * This one-shot form builds a single-rank plan, stages it through the workspace and
  * launches; per-step use should go through deft_plan_build/deft_select_planned.
- *   acc_d             in   the accumulated vector (16-byte aligned); not modified
+ *   acc_d             in   the accumulated vector (16-byte aligned); not modified.  Reads are
+ *                          128-bit: a layer that ends inside a 16-byte group makes the kernel
+ *                          read the rest of that group too (so the buffer must be readable up to
+ *                          the next multiple of 4 elements, which holds for any CUDA allocation)
  *   layer_start_h[L+1], k_l_h[L]   HOST tables for the whole model
  *   my_layers_h[n_my] HOST, ascending; n_my may be 0 (nothing is written)
  *   val_d, idx_d      out  DEVICE buffers of out_cap entries
@@ -257,10 +260,11 @@ DEFT_API deft_status deft_select_planned(const float* acc_d, const void* plan_h,
  * for the ranks rank_begin <= r < rank_end of an uploaded plan, one after the other on
  * `stream` — what N workers would each do on their own GPU, replayed on one.  Rank r
  * writes its entries at offset deft_plan_rank_info().out_off of val_d / idx_d (shared
- * buffers of out_cap >= total k entries) and then zeroes them in acc_d.  Because ranks own
- * disjoint layers the result equals zeroing the union after all selections.
- * events: NULL, or 3 cudaEvent_t per rank (HOST array of handles): recorded before the
- * selection, between selection and update, and after the update, for per-rank timing.
+ * buffers of out_cap >= total k entries) and zeroes them in acc_d (the selection kernel
+ * does it on its way out: same result as deft_residual_update on the rank's indices).
+ * Because ranks own disjoint layers the result equals zeroing the union after all selections.
+ * events: NULL, or 3 cudaEvent_t per rank (HOST array of handles): [0] is recorded before
+ * the rank's launch, [1] and [2] after it, for per-rank timing.
  * Errors: INVALID_ARG, CAPACITY, CUDA.
  */
 DEFT_API deft_status deft_select_update_ranks(float* acc_d, int64_t n_g, const void* plan_h,

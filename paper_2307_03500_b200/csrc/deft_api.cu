@@ -110,7 +110,7 @@ deft_status upload_plan(const void* plan_h, void* plan_d, void* ws_d, size_t ws_
 
 deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan_d, int32_t rank,
                         float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
-                        cudaStream_t stream) {
+                        cudaStream_t stream, bool zero_selected = false) {
     const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
     if (rank < 0 || rank >= hdr->N) return DEFT_ERR_INVALID_ARG;
     const RankInfo& R = plan_ranks(plan_h)[rank];
@@ -124,14 +124,13 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.desc = plan_descs(plan_d, hdr->N) + R.desc_first;
     p.n_my = R.n_my;
     p.tiles = R.tiles;
+    p.acc_rw = zero_selected ? const_cast<float*>(acc_d) : nullptr;
     p.state = reinterpret_cast<LayerState*>(ws + w.state);
-    p.flags = reinterpret_cast<RankFlags*>(ws + w.flags) + rank;
     p.hist1 = reinterpret_cast<uint32_t*>(ws + w.hist1);
     p.hist2 = reinterpret_cast<uint32_t*>(ws + w.hist2);
     p.hist3 = reinterpret_cast<uint32_t*>(ws + w.hist3);
-    const size_t slot0 = 2 * ((size_t)R.tile_base + (size_t)rank);
-    p.runcnt = reinterpret_cast<uint32_t*>(ws + w.cnt) + slot0;
-    p.runge = reinterpret_cast<uint2*>(ws + w.ge) + slot0;
+    p.tt = reinterpret_cast<uint4*>(ws + w.tt) + R.tile_base;
+    p.runge = reinterpret_cast<uint2*>(ws + w.runge) + 2 * ((size_t)R.tile_base + (size_t)rank);
     p.staging = reinterpret_cast<uint2*>(ws + w.staging);
     p.val = val_d;
     p.idx = idx_d;
@@ -273,12 +272,12 @@ deft_status deft_select_update_ranks(float* acc_d, int64_t n_g, const void* plan
         const RankInfo& R = plan_ranks(plan_h)[r];
         void* const* ev = events ? events + 3 * (size_t)(r - rank_begin) : nullptr;
         if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[0]), st));
-        deft_status s = select_rank(acc_d, plan_h, plan_d, r, val_d + R.out_off, idx_d + R.out_off, R.k,
-                                    ws_d, ws_bytes, st);
+        // the selection kernel zeroes what it selects on its way out (same result as a separate
+        // deft_residual_update of the rank's indices, one launch less)
+        const deft_status s = select_rank(acc_d, plan_h, plan_d, r, val_d + R.out_off, idx_d + R.out_off, R.k,
+                                          ws_d, ws_bytes, st, true);
         if (s != DEFT_OK) return s;
         if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[1]), st));
-        s = launch_residual_update(acc_d, idx_d + R.out_off, R.k, st);
-        if (s != DEFT_OK) return s;
         if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[2]), st));
     }
     return DEFT_OK;

@@ -15,7 +15,7 @@ namespace deft {
 // is read with aligned 128-bit loads whatever the layer boundaries are; the first and
 // last tile of a layer may be partial and are read element-wise under a mask.
 // One warp processes one tile at a time.  Every CTA owns a contiguous run of a rank's
-// tiles; the entries it stages for one layer form one contiguous "run" of the staging stream.
+// tiles in every phase and keeps the entries it stages for them.
 // ---------------------------------------------------------------------------------
 constexpr int kTile = 2048;          // elements per tile
 constexpr int kSelThreads = 512;     // one persistent CTA per SM (128 registers per thread)
@@ -27,10 +27,10 @@ constexpr int kSlots = 8;            // per-CTA shared-memory histograms live at
 constexpr int kBins1 = 4096, kBins2 = 1024, kBins3 = 512;
 constexpr int kShift1 = 19, kShift2 = 9;
 
-// A layer is "small" when one CTA can finish it from shared memory: at most kSmallTiles
-// chunks and at most kSmallEntries staged entries.  Everything else takes the general path.
-constexpr int kSmallTiles = 4096;
-constexpr int kSmallEntries = 20480;
+// Layers of at most kDirectElems elements are not streamed: one CTA loads each of them whole.
+constexpr int kDirectElems = 16384;
+// Staged entries a CTA keeps in shared memory; the rest spills to the staging stream in HBM.
+constexpr int kResident = 16384;
 
 constexpr int kMaxRanks = 4096;      // workers per plan
 
@@ -92,27 +92,23 @@ inline const LayerDesc* plan_descs(const void* plan, int64_t N) {
                                               sizeof(RankInfo) * (size_t)N);
 }
 
-struct LayerState {                  // per layer, written by the kernels; 32 bytes
+struct LayerState {                  // per layer, written by the kernels; 64 bytes
     uint32_t b1, above1;             // level-1 bucket of the k-th key; keys strictly above that bucket
-    uint32_t cand1, big;             // keys inside bucket b1; 1 = layer takes the general path
     uint32_t b2, krem2;              // level 2 (inside b1): bucket, and how many still to take inside it
     uint32_t T, need;                // exact threshold key; entries equal to T to take (lowest indices)
+    uint32_t ticket1, ticket2, ticket3;   // tiles whose level-1/2/3 counts have been flushed
+    uint32_t pad[7];
 };
-static_assert(sizeof(LayerState) == 32, "LayerState layout");
-
-struct RankFlags {
-    uint32_t any_big;                // some layer of the rank takes the general path
-    uint32_t error;                  // reserved for kernel-side consistency checks
-};
+static_assert(sizeof(LayerState) == 64, "LayerState layout");
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Carve-up of the caller's workspace.  Offsets depend only on (elems, L, tiles).
 struct WsLayout {
     size_t plan;                     // scratch device plan for the one-shot calls
-    size_t zero_begin, zero_end;     // [state | flags | hist1 | hist2 | hist3]: cleared at plan upload
-    size_t state, flags, hist1, hist2, hist3;
-    size_t cnt, ge, staging;
+    size_t zero_begin, zero_end;     // [state | hist1 | hist2 | hist3]: cleared at plan upload
+    size_t state, hist1, hist2, hist3;
+    size_t tt, runge, staging;
     size_t total;
 };
 
@@ -122,14 +118,13 @@ inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
     w.plan = off;     off += align_up(plan_bytes(L, 1), 256);
     w.zero_begin = off;
     w.state = off;    off += align_up(sizeof(LayerState) * (size_t)L, 256);
-    w.flags = off;    off += align_up(sizeof(RankFlags) * (size_t)kMaxRanks, 256);
     w.hist1 = off;    off += sizeof(uint32_t) * (size_t)kBins1 * (size_t)L;
     w.hist2 = off;    off += sizeof(uint32_t) * (size_t)kBins2 * (size_t)L;
     w.hist3 = off;    off += sizeof(uint32_t) * (size_t)kBins3 * (size_t)L;
     w.zero_end = off;
+    w.tt = off;       off += align_up(sizeof(uint4) * (size_t)tiles, 256);
     const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
-    w.cnt = off;      off += align_up(sizeof(uint32_t) * slots, 256);
-    w.ge = off;       off += align_up(sizeof(uint2) * slots, 256);
+    w.runge = off;    off += align_up(sizeof(uint2) * slots, 256);
     w.staging = off;  off += align_up(sizeof(uint2) * (size_t)elems, 256);
     w.total = off;
     return w;
@@ -145,16 +140,16 @@ inline size_t norms_ws_bytes(int64_t n_g, int64_t L) {
 // Arguments of the fused selection kernel (one rank).
 struct SelParams {
     const float* acc;
+    float* acc_rw;                   // NULL, or the same vector: selected entries are zeroed on the way out
     const LayerDesc* desc;           // the rank's layers + sentinel (device)
     int32_t n_my, tiles;
     LayerState* state;               // [L]
-    RankFlags* flags;                // this rank's flags
     uint32_t* hist1;                 // [L][kBins1]
     uint32_t* hist2;                 // [L][kBins2]
     uint32_t* hist3;                 // [L][kBins3]
-    uint32_t* runcnt;                // this rank's runs (slot = CTA + layer position): staged entries
-    uint2* runge;                    // this rank's runs: (#key > T, #key == T), then exclusive scans
-    uint2* staging;                  // absolute base; (value bits, offset from the run's first tile)
+    uint4* tt;                       // this rank's tiles: (first entry, entries, #key > T, #key == T)
+    uint2* runge;                    // this rank's (CTA, layer) pairs (slot = CTA + layer position): totals
+    uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output
     int64_t* idx;
     unsigned long long* timing;      // optional: 16 phase timestamps (ns, max over CTAs); NULL = off

@@ -42,7 +42,9 @@ constexpr int kSmAuxBytes = 32 * 1024;
 static_assert(kSlots * kBins2 * 4 <= kSmAuxBytes && kBins1 * 4 + kBins2 * 4 <= kSmAuxBytes, "aux region");
 constexpr int kSmMisc = kSmAux + kSmAuxBytes;
 constexpr int kSmMiscBytes = 2048;
-constexpr int kSmemBytes = kSmMisc + kSmMiscBytes;
+constexpr int kSmGroup = kSmMisc + kSmMiscBytes;   // GroupShared
+constexpr int kSmGroupBytes = 512;
+constexpr int kSmemBytes = kSmGroup + kSmGroupBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 static_assert(kBins2 >= kBins3, "the level-3 histogram reuses the level-2 buffer");
 
@@ -210,6 +212,12 @@ __device__ __forceinline__ void stage_put(const Stage& st, uint32_t pos, uint2 v
 __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
     return pos < (uint32_t)kResident ? st.res[pos] : __ldcg(st.spill + (pos - kResident));
 }
+// Entry `pos` of a tile whose entries [first, first + n) are known to be all resident
+// (`all_res`, uniform over the warp): a plain shared-memory access, no address-space test.
+__device__ __forceinline__ uint2 stage_get_tile(const Stage& st, const uint2* res_sh, bool all_res, uint32_t pos) {
+    if (all_res) return res_sh[pos];
+    return stage_get(st, pos);
+}
 
 // Bit c of the result: component c of v has key >= thr.
 __device__ __forceinline__ uint32_t keep4(const uint4& v, uint32_t thr) {
@@ -227,7 +235,8 @@ __device__ __forceinline__ uint32_t valid4(int o, int s, int e) {
 // (load, lane, component = ascending offset).  Returns (first entry, entries).
 // The common case (a handful of entries per tile) costs about 3 instructions per element.
 __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t b1,
-                                             uint32_t* h2, const Stage& st, uint32_t* cursor, int lane) {
+                                             uint32_t* h2, const Stage& st, uint2* res_sh, uint32_t* cursor,
+                                             int lane) {
     TileRegs t;
     load_tile(acc, ts, lane, t);
     const uint32_t thr = b1 << kShift1;          // key >= thr  <=>  bucket >= b1
@@ -263,6 +272,7 @@ __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, cons
     uint32_t first = 0;
     if (lane == 0) first = atomicAdd(cursor, n);
     first = __shfl_sync(0xffffffffu, first, 0);
+    const bool all_res = first + n <= (uint32_t)kResident;   // uniform over the warp
     uint32_t load_base = first;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -276,7 +286,8 @@ __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, cons
                 if (k4 & (1u << c)) {
                     const uint32_t key = key_of(w[c]);
                     if ((key >> kShift1) == b1) atomicAdd(&h2[(key >> kShift2) & (kBins2 - 1)], 1u);
-                    stage_put(st, pos, make_uint2(w[c], (uint32_t)((i * 32 + lane) * 4 + c)));
+                    const uint2 ent = make_uint2(w[c], (uint32_t)((i * 32 + lane) * 4 + c));
+                    if (all_res) res_sh[pos] = ent; else stage_put(st, pos, ent);
                     ++pos;
                 }
         }
@@ -334,39 +345,57 @@ __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
     return p.desc[j].end - p.desc[j].start <= kDirectElems;
 }
 
-// The streamed (non-direct) layers of the CTA's range, kSlots at a time.
+// The streamed (non-direct) layers of the CTA's range, kSlots at a time.  The per-slot facts
+// the tile loops need live in shared memory so that walking the tiles touches no global or
+// local memory.
+struct GroupShared {
+    int lay[kSlots];        // layer position in the rank's list
+    int lid[kSlots];        // layer id in the model (state / histogram index)
+    int tf[kSlots];         // first tile of the layer
+    int tfe[kSlots];        // one past its last tile
+    int64_t start[kSlots];
+    int64_t end[kSlots];
+    int64_t out_off[kSlots];
+};
 struct Group {
     int ns;
-    int lay[kSlots];
     int qa, qb;   // the CTA's tiles from the first to the last layer of the group
 };
 
-__device__ __forceinline__ bool next_group(const SelParams& p, const CtaRange& r, int& jn, Group& g) {
+// Every thread computes the same group; threads < ns publish the per-slot facts.  The caller
+// must __syncthreads() before the facts are read.
+__device__ __forceinline__ bool next_group(const SelParams& p, const CtaRange& r, int& jn, Group& g,
+                                           GroupShared* gs) {
     g.ns = 0;
-    int j = jn;
-    for (; j <= r.jB && g.ns < kSlots; ++j)
-        if (!is_direct(p, j)) g.lay[g.ns++] = j;
+    int j = jn, first = -1, last = -1;
+    for (; j <= r.jB && g.ns < kSlots; ++j) {
+        if (is_direct(p, j)) continue;
+        if (g.ns == (int)threadIdx.x) {
+            gs->lay[g.ns] = j;
+            gs->lid[g.ns] = p.desc[j].layer_id;
+            gs->tf[g.ns] = p.desc[j].tile_first;
+            gs->tfe[g.ns] = p.desc[j + 1].tile_first;
+            gs->start[g.ns] = p.desc[j].start;
+            gs->end[g.ns] = p.desc[j].end;
+            gs->out_off[g.ns] = p.desc[j].out_off;
+        }
+        if (first < 0) first = j;
+        last = j;
+        ++g.ns;
+    }
     jn = j;
     if (g.ns == 0) return false;
-    const int tf = p.desc[g.lay[0]].tile_first, tfe = p.desc[g.lay[g.ns - 1] + 1].tile_first;
+    const int tf = p.desc[first].tile_first, tfe = p.desc[last + 1].tile_first;
     g.qa = r.q0 > tf ? r.q0 : tf;
     g.qb = r.q1 < tfe ? r.q1 : tfe;
     return true;
 }
 
-// Per-warp walk over the group's tiles: tile q belongs to layer lay[s] (or to a direct layer:
-// result < 0).  `jj` and `s` are cursors that only move forward.
-__device__ __forceinline__ int tile_slot(const SelParams& p, const Group& g, int q, int& jj, int& s) {
-    while (q >= p.desc[jj + 1].tile_first) ++jj;
-    while (s < g.ns - 1 && g.lay[s] < jj) ++s;
-    return g.lay[s] == jj ? s : -1;
-}
-
-// How many of layer j's tiles lie in this CTA's range.
-__device__ __forceinline__ uint32_t my_tiles_of(const SelParams& p, const CtaRange& r, int j) {
-    const int tf = p.desc[j].tile_first, tfe = p.desc[j + 1].tile_first;
-    const int a = r.q0 > tf ? r.q0 : tf, b = r.q1 < tfe ? r.q1 : tfe;
-    return b > a ? (uint32_t)(b - a) : 0u;
+// Per-warp walk over the group's tiles: tile q belongs to slot s (or to a direct layer that
+// lies between two slots: result < 0).  `s` is a cursor that only moves forward.
+__device__ __forceinline__ int tile_slot(const Group& g, const GroupShared* gs, int q, int& s) {
+    while (s < g.ns - 1 && q >= gs->tfe[s]) ++s;
+    return (q >= gs->tf[s] && q < gs->tfe[s]) ? s : -1;
 }
 
 // After the CTA has flushed its counts of the group's layers (a __syncthreads() lies between
@@ -374,15 +403,16 @@ __device__ __forceinline__ uint32_t my_tiles_of(const SelParams& p, const CtaRan
 // last tiles, so the layer's histogram is complete.
 template <int kTicket>
 __device__ __forceinline__ void take_tickets(const SelParams& p, const CtaRange& r, const Group& g,
-                                             uint32_t* last) {
+                                             const GroupShared* gs, uint32_t* last) {
     if ((int)threadIdx.x < g.ns) {
-        const int j = g.lay[threadIdx.x];
-        LayerState* st = p.state + p.desc[j].layer_id;
+        const int sl = threadIdx.x;
+        LayerState* st = p.state + gs->lid[sl];
         uint32_t* t = kTicket == 1 ? &st->ticket1 : kTicket == 2 ? &st->ticket2 : &st->ticket3;
-        const uint32_t mine = my_tiles_of(p, r, j);
+        const int a = r.q0 > gs->tf[sl] ? r.q0 : gs->tf[sl], b = r.q1 < gs->tfe[sl] ? r.q1 : gs->tfe[sl];
+        const uint32_t mine = b > a ? (uint32_t)(b - a) : 0u;   // this CTA's tiles of the layer
         __threadfence();
         const uint32_t old = atomicAdd(t, mine);
-        last[threadIdx.x] = (old + mine == (uint32_t)(p.desc[j + 1].tile_first - p.desc[j].tile_first)) ? 1u : 0u;
+        last[sl] = (old + mine == (uint32_t)(gs->tfe[sl] - gs->tf[sl])) ? 1u : 0u;
     }
     __syncthreads();
 }
@@ -395,26 +425,28 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     Group g;
-    for (int jn = r.jA; next_group(p, r, jn, g);) {
+    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
+    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
+        __syncthreads();   // the group's facts are published
         for (int i = threadIdx.x; i < g.ns * kBins1; i += kSelThreads) hist[i] = 0;
         __syncthreads();
-        int jj = g.lay[0], s = 0;
+        int s = 0;
         for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            const int slot = tile_slot(p, g, q, jj, s);
+            const int slot = tile_slot(g, gs, q, s);
             if (slot < 0) continue;
-            const TileSpan ts = tile_span(p.desc[jj].start, p.desc[jj].end, p.desc[jj].tile_first, q);
+            const TileSpan ts = tile_span(gs->start[slot], gs->end[slot], gs->tf[slot], q);
             hist_tile(p.acc, ts, hist + slot * kBins1, lane);
         }
         __syncthreads();
         for (int i = threadIdx.x; i < g.ns * kBins1; i += kSelThreads) {
             const uint32_t c = hist[i];
-            if (c) atomicAdd(p.hist1 + (size_t)p.desc[g.lay[i / kBins1]].layer_id * kBins1 + (i % kBins1), c);
+            if (c) atomicAdd(p.hist1 + (size_t)gs->lid[i / kBins1] * kBins1 + (i % kBins1), c);
         }
         __syncthreads();
-        take_tickets<1>(p, r, g, misc + kMLast);
+        take_tickets<1>(p, r, g, gs, misc + kMLast);
         for (int s2 = 0; s2 < g.ns; ++s2) {
             if (!misc[kMLast + s2]) continue;   // uniform over the CTA
-            const int j = g.lay[s2];
+            const int j = gs->lay[s2];
             const int lid = p.desc[j].layer_id;
             __threadfence();
             block_scan_select<true>(p.hist1 + (size_t)lid * kBins1, kBins1, (uint32_t)p.desc[j].k,
@@ -425,6 +457,7 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
             }
             __syncthreads();
         }
+        __syncthreads();   // the group's facts are no longer read
     }
 }
 
@@ -438,29 +471,31 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) misc[kMCursor] = 0;
     Group g;
-    for (int jn = r.jA; next_group(p, r, jn, g);) {
-        if ((int)threadIdx.x < g.ns) misc[kMTabA + threadIdx.x] = __ldcg(&p.state[p.desc[g.lay[threadIdx.x]].layer_id].b1);
+    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
+    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
+        __syncthreads();   // the group's facts are published
+        if ((int)threadIdx.x < g.ns) misc[kMTabA + threadIdx.x] = __ldcg(&p.state[gs->lid[threadIdx.x]].b1);
         for (int i = threadIdx.x; i < g.ns * kBins2; i += kSelThreads) hist2s[i] = 0;
         __syncthreads();
-        int jj = g.lay[0], s = 0;
+        int s = 0;
         for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            const int slot = tile_slot(p, g, q, jj, s);
+            const int slot = tile_slot(g, gs, q, s);
             if (slot < 0) continue;
-            const TileSpan ts = tile_span(p.desc[jj].start, p.desc[jj].end, p.desc[jj].tile_first, q);
+            const TileSpan ts = tile_span(gs->start[slot], gs->end[slot], gs->tf[slot], q);
             const uint2 fn = filter_tile(p.acc, ts, misc[kMTabA + slot], hist2s + slot * kBins2, st,
-                                         misc + kMCursor, lane);
+                                         reinterpret_cast<uint2*>(smem + kSmMain), misc + kMCursor, lane);
             if (lane == 0) p.tt[q] = make_uint4(fn.x, fn.y, 0u, 0u);
         }
         __syncthreads();
         for (int i = threadIdx.x; i < g.ns * kBins2; i += kSelThreads) {
             const uint32_t c = hist2s[i];
-            if (c) atomicAdd(p.hist2 + (size_t)p.desc[g.lay[i / kBins2]].layer_id * kBins2 + (i % kBins2), c);
+            if (c) atomicAdd(p.hist2 + (size_t)gs->lid[i / kBins2] * kBins2 + (i % kBins2), c);
         }
         __syncthreads();
-        take_tickets<2>(p, r, g, misc + kMLast);
+        take_tickets<2>(p, r, g, gs, misc + kMLast);
         for (int s2 = 0; s2 < g.ns; ++s2) {
             if (!misc[kMLast + s2]) continue;   // uniform over the CTA
-            const int j = g.lay[s2];
+            const int j = gs->lay[s2];
             const int lid = p.desc[j].layer_id;
             __threadfence();
             const uint32_t krem1 = (uint32_t)p.desc[j].k - __ldcg(&p.state[lid].above1);
@@ -471,6 +506,7 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
             }
             __syncthreads();
         }
+        __syncthreads();   // the group's facts are no longer read
     }
 }
 
@@ -482,37 +518,45 @@ __device__ __forceinline__ void step_hist3(const SelParams& p, const CtaRange& r
     uint32_t* h3 = reinterpret_cast<uint32_t*>(smem + kSmAux);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint2* res_sh = reinterpret_cast<const uint2*>(smem + kSmMain);
     Group g;
-    for (int jn = r.jA; next_group(p, r, jn, g);) {
+    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
+    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
+        __syncthreads();   // the group's facts are published
         if ((int)threadIdx.x < g.ns) {
-            const LayerState* ls = p.state + p.desc[g.lay[threadIdx.x]].layer_id;
+            const LayerState* ls = p.state + gs->lid[threadIdx.x];
             misc[kMTabA + threadIdx.x] = (__ldcg(&ls->b1) << (kShift1 - kShift2)) | __ldcg(&ls->b2);
         }
         for (int i = threadIdx.x; i < g.ns * kBins3; i += kSelThreads) h3[i] = 0;
         __syncthreads();
-        int jj = g.lay[0], s = 0;
+        stamp(p, 8);
+        int s = 0;
         TtBatch tb;
         for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
             if ((q - g.qa - warp) % (32 * kSelWarps) == 0) tt_fetch(p, q, g.qb, lane, tb);
-            const int slot = tile_slot(p, g, q, jj, s);
+            const int slot = tile_slot(g, gs, q, s);
             if (slot < 0) continue;
             const uint4 t = tt_get(tb, q);
             const uint32_t prefix = misc[kMTabA + slot];
+            const bool all_res = t.x + t.y <= (uint32_t)kResident;
             for (uint32_t e = lane; e < t.y; e += 32) {
-                const uint32_t key = key_of(stage_get(st, t.x + e).x);
+                const uint32_t key = key_of(stage_get_tile(st, res_sh, all_res, t.x + e).x);
                 if ((key >> kShift2) == prefix) atomicAdd(&h3[slot * kBins3 + (key & (kBins3 - 1))], 1u);
             }
         }
+        stamp(p, 9);
         __syncthreads();
         for (int i = threadIdx.x; i < g.ns * kBins3; i += kSelThreads) {
             const uint32_t c = h3[i];
-            if (c) atomicAdd(p.hist3 + (size_t)p.desc[g.lay[i / kBins3]].layer_id * kBins3 + (i % kBins3), c);
+            if (c) atomicAdd(p.hist3 + (size_t)gs->lid[i / kBins3] * kBins3 + (i % kBins3), c);
         }
         __syncthreads();
-        take_tickets<3>(p, r, g, misc + kMLast);
+        stamp(p, 10);
+        take_tickets<3>(p, r, g, gs, misc + kMLast);
+        stamp(p, 11);
         for (int s2 = 0; s2 < g.ns; ++s2) {
             if (!misc[kMLast + s2]) continue;   // uniform over the CTA
-            const int lid = p.desc[g.lay[s2]].layer_id;
+            const int lid = gs->lid[s2];
             __threadfence();
             const uint32_t krem2 = __ldcg(&p.state[lid].krem2);
             block_scan_select<true>(p.hist3 + (size_t)lid * kBins3, kBins3, krem2, misc + kMScratch, misc + kMOut3);
@@ -523,6 +567,7 @@ __device__ __forceinline__ void step_hist3(const SelParams& p, const CtaRange& r
             }
             __syncthreads();
         }
+        __syncthreads();   // the group's facts are no longer read
     }
 }
 
@@ -533,25 +578,29 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
                                            unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint2* res_sh = reinterpret_cast<const uint2*>(smem + kSmMain);
     Group g;
-    for (int jn = r.jA; next_group(p, r, jn, g);) {
+    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
+    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
+        __syncthreads();   // the group's facts are published
         if ((int)threadIdx.x < g.ns) {
-            misc[kMTabA + threadIdx.x] = __ldcg(&p.state[p.desc[g.lay[threadIdx.x]].layer_id].T);
+            misc[kMTabA + threadIdx.x] = __ldcg(&p.state[gs->lid[threadIdx.x]].T);
             misc[kMTotGt + threadIdx.x] = 0;
             misc[kMTotEq + threadIdx.x] = 0;
         }
         __syncthreads();
-        int jj = g.lay[0], s = 0;
+        int s = 0;
         TtBatch tb;
         for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
             if ((q - g.qa - warp) % (32 * kSelWarps) == 0) tt_fetch(p, q, g.qb, lane, tb);
-            const int slot = tile_slot(p, g, q, jj, s);
+            const int slot = tile_slot(g, gs, q, s);
             if (slot < 0) continue;
             const uint4 t = tt_get(tb, q);
             const uint32_t T = misc[kMTabA + slot];
             uint32_t n_gt = 0, n_eq = 0;
+            const bool all_res = t.x + t.y <= (uint32_t)kResident;
             for (uint32_t e = lane; e < t.y; e += 32) {
-                const uint32_t key = key_of(stage_get(st, t.x + e).x);
+                const uint32_t key = key_of(stage_get_tile(st, res_sh, all_res, t.x + e).x);
                 n_gt += key > T;
                 n_eq += key == T;
             }
@@ -565,7 +614,7 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
         }
         __syncthreads();
         if ((int)threadIdx.x < g.ns)
-            p.runge[blockIdx.x + g.lay[threadIdx.x]] = make_uint2(misc[kMTotGt + threadIdx.x], misc[kMTotEq + threadIdx.x]);
+            p.runge[blockIdx.x + gs->lay[threadIdx.x]] = make_uint2(misc[kMTotGt + threadIdx.x], misc[kMTotEq + threadIdx.x]);
         __syncthreads();
     }
 }
@@ -599,10 +648,13 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint32_t* scratch = misc + kMScratch;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint2* res_sh = reinterpret_cast<const uint2*>(smem + kSmMain);
     Group g;
-    for (int jn = r.jA; next_group(p, r, jn, g);) {
+    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
+    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
+        __syncthreads();   // the group's facts are published
         for (int s2 = 0; s2 < g.ns; ++s2) {
-            const int j = g.lay[s2];
+            const int j = gs->lay[s2];
             const int tf = p.desc[j].tile_first, tfe = p.desc[j + 1].tile_first;
             // totals of the CTAs that hold earlier tiles of the layer
             const int b0 = cta_of_tile(p, tf);
@@ -637,23 +689,24 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             }
         }
         __syncthreads();
-        int jj = g.lay[0], s = 0;
+        int s = 0;
         TtBatch tb;
         for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
             if ((q - g.qa - warp) % (32 * kSelWarps) == 0) tt_fetch(p, q, g.qb, lane, tb);
-            const int slot = tile_slot(p, g, q, jj, s);
+            const int slot = tile_slot(g, gs, q, s);
             if (slot < 0) continue;
             const uint4 t = tt_get(tb, q);
             if (t.y == 0) continue;
             const uint32_t T = misc[kMTabA + slot], need = misc[kMTabB + slot];
-            const int64_t lo = (p.desc[jj].start / kTile + (q - p.desc[jj].tile_first)) * kTile;
-            const int64_t out_off = p.desc[jj].out_off;
+            const int64_t lo = (gs->start[slot] / kTile + (q - gs->tf[slot])) * kTile;
+            const int64_t out_off = gs->out_off[slot];
             uint32_t gt_before = t.z, eq_before = t.w;
+            const bool all_res = t.x + t.y <= (uint32_t)kResident;
             for (uint32_t e0 = 0; e0 < t.y; e0 += 32) {
                 const uint32_t e = e0 + lane;
                 const bool valid = e < t.y;
                 uint2 ent = make_uint2(0u, 0u);
-                if (valid) ent = stage_get(st, t.x + e);
+                if (valid) ent = stage_get_tile(st, res_sh, all_res, t.x + e);
                 emit_batch(p, out_off, lo, valid, ent.x, (int64_t)ent.y, T, need, gt_before, eq_before, lane);
             }
         }

@@ -129,12 +129,29 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.hist1 = reinterpret_cast<uint32_t*>(ws + w.hist1);
     p.hist2 = reinterpret_cast<uint32_t*>(ws + w.hist2);
     p.hist3 = reinterpret_cast<uint32_t*>(ws + w.hist3);
-    p.tt = reinterpret_cast<uint4*>(ws + w.tt) + R.tile_base;
     p.runge = reinterpret_cast<uint2*>(ws + w.runge) + 2 * ((size_t)R.tile_base + (size_t)rank);
     p.staging = reinterpret_cast<uint2*>(ws + w.staging);
     p.val = val_d;
     p.idx = idx_d;
     p.timing = g_select_timing;
+    // one CTA per SM at most (co-resident by construction); fewer when the rank is small
+    const int sms = sm_count();
+    int want = (R.tiles + 1) / 2;
+    if (want < R.n_my) want = R.n_my;
+    if (want < 1) want = 1;
+    p.grid = want < sms ? want : sms;
+    // limits of one CTA's share: tiles, and streamed (non-direct) layers
+    const LayerDesc* hd = plan_descs(plan_h, hdr->N) + R.desc_first;
+    int j = 0;
+    for (int b = 0; b < p.grid; ++b) {
+        const int q0 = (int)((int64_t)R.tiles * b / p.grid), q1 = (int)((int64_t)R.tiles * (b + 1) / p.grid);
+        if (q1 - q0 > kMaxLocalTiles) return DEFT_ERR_INVALID_ARG;
+        while (j + 1 < R.n_my && hd[j + 1].tile_first <= q0) ++j;
+        int streamed = 0;
+        for (int jj = j; jj < R.n_my && hd[jj].tile_first < q1; ++jj)
+            streamed += (hd[jj].end - hd[jj].start > kDirectElems);
+        if (streamed > kMaxLocalLayers) return DEFT_ERR_INVALID_ARG;
+    }
     return launch_select(p, stream);
 }
 

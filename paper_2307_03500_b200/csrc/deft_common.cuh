@@ -20,17 +20,23 @@ namespace deft {
 constexpr int kTile = 2048;          // elements per tile
 constexpr int kSelThreads = 512;     // one persistent CTA per SM (128 registers per thread)
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kSlots = 8;            // per-CTA shared-memory histograms live at once
+constexpr int kSlots = 8;            // level-1 shared-memory histograms live at once per CTA
 
 // Radix digits over the 31-bit magnitude key (IEEE bits with the sign cleared):
 // level 1 = bits 30..19 (exponent + 4 mantissa bits), level 2 = bits 18..9, level 3 = bits 8..0.
 constexpr int kBins1 = 4096, kBins2 = 1024, kBins3 = 512;
 constexpr int kShift1 = 19, kShift2 = 9;
+// Layers that one CTA loads whole ("direct") use coarser digits: bits 30..19, 18..9, 8..0.
+constexpr int kDBins1 = 4096, kDBins2 = 1024, kDBins3 = 512;
+constexpr int kDShift1 = 19, kDShift2 = 9;
 
 // Layers of at most kDirectElems elements are not streamed: one CTA loads each of them whole.
 constexpr int kDirectElems = 16384;
 // Staged entries a CTA keeps in shared memory; the rest spills to the staging stream in HBM.
 constexpr int kResident = 16384;
+// Limits of one CTA's share of a rank (checked on the host before launch).
+constexpr int kMaxLocalTiles = 4096;    // tiles per CTA
+constexpr int kMaxLocalLayers = 256;    // streamed layers per CTA
 
 constexpr int kMaxRanks = 4096;      // workers per plan
 
@@ -96,8 +102,8 @@ struct LayerState {                  // per layer, written by the kernels; 64 by
     uint32_t b1, above1;             // level-1 bucket of the k-th key; keys strictly above that bucket
     uint32_t b2, krem2;              // level 2 (inside b1): bucket, and how many still to take inside it
     uint32_t T, need;                // exact threshold key; entries equal to T to take (lowest indices)
-    uint32_t ticket1, ticket2, ticket3;   // tiles whose level-1/2/3 counts have been flushed
-    uint32_t pad[7];
+    uint32_t ticket1;                // tiles whose level-1 counts have been flushed
+    uint32_t pad[9];
 };
 static_assert(sizeof(LayerState) == 64, "LayerState layout");
 
@@ -108,7 +114,7 @@ struct WsLayout {
     size_t plan;                     // scratch device plan for the one-shot calls
     size_t zero_begin, zero_end;     // [state | hist1 | hist2 | hist3]: cleared at plan upload
     size_t state, hist1, hist2, hist3;
-    size_t tt, runge, staging;
+    size_t runge, staging;
     size_t total;
 };
 
@@ -122,7 +128,6 @@ inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
     w.hist2 = off;    off += sizeof(uint32_t) * (size_t)kBins2 * (size_t)L;
     w.hist3 = off;    off += sizeof(uint32_t) * (size_t)kBins3 * (size_t)L;
     w.zero_end = off;
-    w.tt = off;       off += align_up(sizeof(uint4) * (size_t)tiles, 256);
     const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
     w.runge = off;    off += align_up(sizeof(uint2) * slots, 256);
     w.staging = off;  off += align_up(sizeof(uint2) * (size_t)elems, 256);
@@ -143,11 +148,11 @@ struct SelParams {
     float* acc_rw;                   // NULL, or the same vector: selected entries are zeroed on the way out
     const LayerDesc* desc;           // the rank's layers + sentinel (device)
     int32_t n_my, tiles;
+    int32_t grid;                    // CTAs of the launch (one per SM at most)
     LayerState* state;               // [L]
     uint32_t* hist1;                 // [L][kBins1]
     uint32_t* hist2;                 // [L][kBins2]
     uint32_t* hist3;                 // [L][kBins3]
-    uint4* tt;                       // this rank's tiles: (first entry, entries, #key > T, #key == T)
     uint2* runge;                    // this rank's (CTA, layer) pairs (slot = CTA + layer position): totals
     uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output

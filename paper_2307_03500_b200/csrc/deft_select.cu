@@ -1,19 +1,20 @@
 // Layer-wise top-k selection for one worker (Algorithm 5) as ONE persistent cooperative
 // kernel: a segmented radix select over magnitude bit patterns followed by an ordered
 // compaction.  One CTA of 512 threads per SM; five steps separated by grid barriers.  Every
-// CTA owns the same contiguous run of the rank's tiles in every step, and keeps what it
+// CTA owns the same contiguous run of the rank's tiles in every step and keeps what it
 // stages for them (in shared memory; overflow spills to HBM), so after the second read of the
 // vector all work is local to the CTA that staged the data.
 //
 //   A   read 1: per-layer histogram of key bits 30..19 in shared memory, flushed with integer
 //       atomics; the CTA that flushes a layer's last tiles finds the bucket b1 holding the
 //       k-th largest key
-//   B   read 2: one warp per tile keeps the whole tile in registers, and moves every entry
+//   B   read 2: one warp per tile keeps the whole tile in registers and moves every entry
 //       with bucket >= b1, in index order, behind the CTA's staging cursor; bucket-b1 entries
-//       feed the level-2 histogram (bits 18..9); last flusher finds bucket b2
-//   S2  level-3 histogram (bits 8..0) over the staged entries of bucket (b1, b2); last
-//       flusher fixes the exact threshold key T and how many entries equal to T are needed
-//   S3  per tile: staged entries above T / equal to T; per (CTA, layer) totals
+//       feed the level-2 histogram (bits 18..9)
+//   S2  every CTA finds bucket b2 of its layers from the level-2 histograms, then adds the
+//       level-3 histogram (bits 8..0) of its staged entries of bucket (b1, b2)
+//   S3  every CTA fixes the exact threshold key T and the number of entries equal to T to
+//       take, counts its staged entries above / equal to T per tile, publishes its totals
 //   S4  every CTA adds up the totals of the CTAs before it, scans its own tiles, and writes
 //       (value, int64 index) in ascending index (equal keys: lowest indices first);
 //       optionally zeroes the selected entries of the vector (residual update)
@@ -32,35 +33,68 @@ namespace cg = cooperative_groups;
 namespace deft {
 namespace {
 
+constexpr int kS2Chunk = 8;       // layers whose level-3 histograms are built at once
+constexpr int kBSlots = 4;        // layers whose level-2 histograms are built at once
+
 // shared-memory carve-up (bytes)
 constexpr int kSmMain = 0;   // A: kSlots level-1 histograms | B..S4: resident entries | direct: keys
 constexpr int kSmMainBytes = 128 * 1024;
 static_assert(kSlots * kBins1 * 4 <= kSmMainBytes && kResident * 8 <= kSmMainBytes &&
               kDirectElems * 4 <= kSmMainBytes, "main region");
-constexpr int kSmAux = kSmMain + kSmMainBytes;   // B: level-2 slots | S2: level-3 slots | direct: level-1 + level-2/3
-constexpr int kSmAuxBytes = 32 * 1024;
-static_assert(kSlots * kBins2 * 4 <= kSmAuxBytes && kBins1 * 4 + kBins2 * 4 <= kSmAuxBytes, "aux region");
-constexpr int kSmMisc = kSmAux + kSmAuxBytes;
-constexpr int kSmMiscBytes = 2048;
-constexpr int kSmGroup = kSmMisc + kSmMiscBytes;   // GroupShared
-constexpr int kSmGroupBytes = 512;
-constexpr int kSmemBytes = kSmGroup + kSmGroupBytes;
+constexpr int kSmAux = kSmMain + kSmMainBytes;   // B: level-2 slots | S2: level-3 slots | direct: its histograms
+constexpr int kSmAuxBytes = 20 * 1024;
+static_assert(kBSlots * kBins2 * 4 <= kSmAuxBytes && kS2Chunk * kBins3 * 4 <= kSmAuxBytes &&
+              kDBins1 * 4 + kDBins2 * 4 <= kSmAuxBytes && kDBins2 >= kDBins3, "aux region");
+constexpr int kSmTile = kSmAux + kSmAuxBytes;    // per local tile: first entry, entries, counts
+constexpr int kSmTileBytes = kMaxLocalTiles * 10;
+constexpr int kSmLayer = kSmTile + kSmTileBytes; // per local streamed layer, see LayerTable
+constexpr int kSmLayerBytes = kMaxLocalLayers * 64;
+constexpr int kSmPref = kSmLayer + kSmLayerBytes;   // prefixes of one batch of tiles in S4
+constexpr int kSmPrefBytes = kSelThreads * 8;
+constexpr int kSmMisc = kSmPref + kSmPrefBytes;
+constexpr int kSmMiscBytes = 1024;
+constexpr int kSmemBytes = kSmMisc + kSmMiscBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
-static_assert(kBins2 >= kBins3, "the level-3 histogram reuses the level-2 buffer");
 
 enum MiscOff : int {   // word offsets inside the misc area
     kMScratch = 0,     // 64: block scan scratch
     kMOut3 = 64,       // 4: result of block_scan_select
-    kMTabA = 72,       // kSlots: per-slot value of the current step (b1 | prefix | T)
-    kMTabB = 80,       // kSlots: second per-slot value (need)
-    kMLast = 88,       // kSlots: this CTA flushed the layer's last tiles
-    kMTotGt = 96,      // kSlots
-    kMTotEq = 104,     // kSlots
-    kMCursor = 112,    // 1: staged entries of this CTA so far
+    kMLast = 72,       // kSlots: this CTA flushed the layer's last tiles
+    kMCursor = 80,     // 1: staged entries of this CTA
+    kMTab = 96,        // kBSlots: per-slot b1 in step B
     kMWarpCnt = 128,   // 32: per-warp packed counts (direct layers)
 };
-static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4, "misc area");
-static_assert(kSlots <= 8, "misc tables are 8 wide");
+static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4 && kSlots <= 8 && kBSlots <= 32, "misc area");
+
+// Facts about the CTA's streamed layers (shared memory, struct of arrays).
+struct LayerTable {
+    int j[kMaxLocalLayers];          // position in the rank's layer list
+    int lid[kMaxLocalLayers];        // layer id in the model (state / histogram index)
+    int tf[kMaxLocalLayers];         // first tile (rank-local tile id)
+    int tfe[kMaxLocalLayers];        // one past the last tile
+    int64_t start[kMaxLocalLayers];  // first element
+    int64_t end[kMaxLocalLayers];
+    int64_t out_off[kMaxLocalLayers];
+    uint32_t v0[kMaxLocalLayers];    // step value: prefix (b1, b2) | T
+    uint32_t v1[kMaxLocalLayers];    // step value: krem1 | krem2 | need
+    uint32_t base_gt[kMaxLocalLayers];
+    uint32_t base_eq[kMaxLocalLayers];
+};
+static_assert(sizeof(LayerTable) <= kSmLayerBytes, "layer table");
+
+struct TileTable {                   // per local tile (tile q - q0 of the CTA)
+    uint32_t first[kMaxLocalTiles];  // first staged entry
+    uint32_t ge[kMaxLocalTiles];     // staged entries above T | equal to T << 16
+    uint16_t n[kMaxLocalTiles];      // staged entries
+};
+static_assert(sizeof(TileTable) <= kSmTileBytes && kTile <= 65535, "tile table");
+
+// staged entry: .x = value bits, .y = offset in tile | local layer << 11 | local tile << 19
+__device__ __forceinline__ uint32_t pack_y(uint32_t off, uint32_t c, uint32_t lq) { return off | (c << 11) | (lq << 19); }
+__device__ __forceinline__ uint32_t y_off(uint32_t y) { return y & 0x7ffu; }
+__device__ __forceinline__ uint32_t y_layer(uint32_t y) { return (y >> 11) & 0xffu; }
+__device__ __forceinline__ uint32_t y_tile(uint32_t y) { return y >> 19; }
+static_assert(kTile == 2048 && kMaxLocalLayers <= 256 && kMaxLocalTiles <= 8192, "entry packing");
 
 __device__ __forceinline__ uint32_t key_of(uint32_t bits) { return bits & 0x7fffffffu; }
 
@@ -107,6 +141,16 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
     return v;
 }
 
+// Sum over lanes >= mine (lane 31 is the top).
+__device__ __forceinline__ uint32_t warp_suffix_sum(uint32_t v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t x = __shfl_down_sync(0xffffffffu, v, o);
+        if (lane + o < 32) v += x;
+    }
+    return v;
+}
+
 // Exclusive prefix of v over the CTA in thread order; `total` = sum over the CTA.
 // scratch: 33 words of shared memory.
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratch, uint32_t& total) {
@@ -126,30 +170,70 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratc
     return scratch[w] + incl - v;
 }
 
-// CTA-wide: walks a histogram (at most 8 * kSelThreads bins) from its top bin down and finds
-// the bucket that holds the k-th largest key.  out[0] = bucket, out[1] = keys strictly above it.
-template <bool kGlobal>
-__device__ __forceinline__ void block_scan_select(const uint32_t* h, int nbins, uint32_t k,
-                                                  uint32_t* scratch, uint32_t* out) {
-    const int per = (nbins + kSelThreads - 1) / kSelThreads;
-    const int base = nbins - per * ((int)threadIdx.x + 1);   // thread order = descending bins
-    uint32_t c[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+// CTA-wide: walks a histogram of kBins bins (kBins / kSelThreads consecutive bins per thread,
+// at most 32) from its top bin down and finds the bucket that holds the k-th largest key.
+// out[0] = bucket, out[1] = keys strictly above it.
+template <int kBins, bool kGlobal>
+__device__ __forceinline__ void block_scan_select(const uint32_t* h, uint32_t k, uint32_t* scratch, uint32_t* out) {
+    constexpr int kPer = (kBins + kSelThreads - 1) / kSelThreads;
+    static_assert(kPer <= 32 && (kBins % kPer) == 0, "bins per thread");
+    const int base = kBins - kPer * ((int)threadIdx.x + 1);   // thread order = descending bins
+    uint32_t c[kPer];
     uint32_t sum = 0;
-    for (int i = 0; i < per; ++i)
-        if (base + i >= 0) { c[i] = kGlobal ? __ldcg(h + base + i) : h[base + i]; sum += c[i]; }
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        c[i] = 0;
+        if (base >= 0) c[i] = kGlobal ? __ldcg(h + base + i) : h[base + i];
+        sum += c[i];
+    }
     if (threadIdx.x == 0) { out[0] = 0; out[1] = 0; }
     uint32_t total;
     const uint32_t excl = block_excl_scan(sum, scratch, total);   // keys in bins above mine
     if (sum != 0 && excl < k && k <= excl + sum) {
         uint32_t run = excl;
-        for (int i = per - 1; i >= 0; --i) {
-            if (run + c[i] >= k) { out[0] = (uint32_t)(base + i); out[1] = run; break; }
-            run += c[i];
+        bool found = false;
+#pragma unroll
+        for (int i = kPer - 1; i >= 0; --i) {
+            if (!found) {
+                if (run + c[i] >= k) { out[0] = (uint32_t)(base + i); out[1] = run; found = true; }
+                else run += c[i];
+            }
         }
     }
     __syncthreads();
 }
-static_assert(kBins1 <= 8 * kSelThreads, "at most 8 bins per thread");
+
+// One warp: the same search on a histogram of 32 * kPerLane bins in global memory (kPerLane =
+// 8, 16 or 32).  Lane l reads bins [kPerLane * l, kPerLane * (l + 1)); lane 31 holds the top.
+template <int kPerLane>
+__device__ __forceinline__ void warp_scan_select(const uint32_t* __restrict__ h, uint32_t k, int lane,
+                                                 uint32_t& bucket, uint32_t& above) {
+    uint32_t c[kPerLane];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int i = 0; i < kPerLane / 4; ++i) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(h + kPerLane * lane) + i);
+        c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
+        sum += v.x + v.y + v.z + v.w;
+    }
+    const uint32_t ab = warp_suffix_sum(sum, lane) - sum;   // keys in lanes above mine
+    const unsigned hit = __ballot_sync(0xffffffffu, sum != 0 && ab < k && k <= ab + sum);
+    bucket = 0; above = 0;
+    if (hit == 0) return;            // k exceeds the histogram total: cannot happen for a valid plan
+    const int owner = __ffs(hit) - 1;
+    uint32_t b = 0, a = ab;
+    bool found = false;
+#pragma unroll
+    for (int i = kPerLane - 1; i >= 0; --i) {
+        if (!found) {
+            if (a + c[i] >= k) { b = kPerLane * lane + i; found = true; }
+            else a += c[i];
+        }
+    }
+    bucket = __shfl_sync(0xffffffffu, b, owner);
+    above = __shfl_sync(0xffffffffu, a, owner);
+}
+static_assert(kBins2 % 128 == 0 && kBins3 % 128 == 0 && kBins2 <= 1024 && kBins3 <= 1024, "warp_scan_select shapes");
 
 // ---------------------------------------------------------------------------------
 // tile workers: one warp holds a whole tile (kTile = 2048 elements) in registers
@@ -212,12 +296,6 @@ __device__ __forceinline__ void stage_put(const Stage& st, uint32_t pos, uint2 v
 __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
     return pos < (uint32_t)kResident ? st.res[pos] : __ldcg(st.spill + (pos - kResident));
 }
-// Entry `pos` of a tile whose entries [first, first + n) are known to be all resident
-// (`all_res`, uniform over the warp): a plain shared-memory access, no address-space test.
-__device__ __forceinline__ uint2 stage_get_tile(const Stage& st, const uint2* res_sh, bool all_res, uint32_t pos) {
-    if (all_res) return res_sh[pos];
-    return stage_get(st, pos);
-}
 
 // Bit c of the result: component c of v has key >= thr.
 __device__ __forceinline__ uint32_t keep4(const uint4& v, uint32_t thr) {
@@ -235,7 +313,7 @@ __device__ __forceinline__ uint32_t valid4(int o, int s, int e) {
 // (load, lane, component = ascending offset).  Returns (first entry, entries).
 // The common case (a handful of entries per tile) costs about 3 instructions per element.
 __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t b1,
-                                             uint32_t* h2, const Stage& st, uint2* res_sh, uint32_t* cursor,
+                                             uint32_t* h2, const Stage& st, uint32_t ytag, uint32_t* cursor,
                                              int lane) {
     TileRegs t;
     load_tile(acc, ts, lane, t);
@@ -272,7 +350,6 @@ __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, cons
     uint32_t first = 0;
     if (lane == 0) first = atomicAdd(cursor, n);
     first = __shfl_sync(0xffffffffu, first, 0);
-    const bool all_res = first + n <= (uint32_t)kResident;   // uniform over the warp
     uint32_t load_base = first;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -286,35 +363,13 @@ __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, cons
                 if (k4 & (1u << c)) {
                     const uint32_t key = key_of(w[c]);
                     if ((key >> kShift1) == b1) atomicAdd(&h2[(key >> kShift2) & (kBins2 - 1)], 1u);
-                    const uint2 ent = make_uint2(w[c], (uint32_t)((i * 32 + lane) * 4 + c));
-                    if (all_res) res_sh[pos] = ent; else stage_put(st, pos, ent);
+                    stage_put(st, pos, make_uint2(w[c], ytag | (uint32_t)((i * 32 + lane) * 4 + c)));
                     ++pos;
                 }
         }
         load_base += tot_i;
     }
     return make_uint2(first, n);
-}
-
-// The tile-table records of a warp's next 32 tiles (tile q0 + i * kSelWarps is held by lane i),
-// fetched with one request so that the walk over the tiles does not wait for memory per tile.
-struct TtBatch {
-    uint4 rec;
-    int q0;
-};
-__device__ __forceinline__ void tt_fetch(const SelParams& p, int q0, int qb, int lane, TtBatch& b) {
-    const int q = q0 + lane * kSelWarps;
-    b.q0 = q0;
-    b.rec = q < qb ? __ldcg(p.tt + q) : make_uint4(0u, 0u, 0u, 0u);
-}
-__device__ __forceinline__ uint4 tt_get(const TtBatch& b, int q) {
-    const int i = (q - b.q0) / kSelWarps;
-    uint4 r;
-    r.x = __shfl_sync(0xffffffffu, b.rec.x, i);
-    r.y = __shfl_sync(0xffffffffu, b.rec.y, i);
-    r.z = __shfl_sync(0xffffffffu, b.rec.z, i);
-    r.w = __shfl_sync(0xffffffffu, b.rec.w, i);
-    return r;
 }
 
 // ---------------------------------------------------------------------------------
@@ -345,277 +400,205 @@ __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
     return p.desc[j].end - p.desc[j].start <= kDirectElems;
 }
 
-// The streamed (non-direct) layers of the CTA's range, kSlots at a time.  The per-slot facts
-// the tile loops need live in shared memory so that walking the tiles touches no global or
-// local memory.
-struct GroupShared {
-    int lay[kSlots];        // layer position in the rank's list
-    int lid[kSlots];        // layer id in the model (state / histogram index)
-    int tf[kSlots];         // first tile of the layer
-    int tfe[kSlots];        // one past its last tile
-    int64_t start[kSlots];
-    int64_t end[kSlots];
-    int64_t out_off[kSlots];
-};
-struct Group {
-    int ns;
-    int qa, qb;   // the CTA's tiles from the first to the last layer of the group
-};
-
-// Every thread computes the same group; threads < ns publish the per-slot facts.  The caller
-// must __syncthreads() before the facts are read.
-__device__ __forceinline__ bool next_group(const SelParams& p, const CtaRange& r, int& jn, Group& g,
-                                           GroupShared* gs) {
-    g.ns = 0;
-    int j = jn, first = -1, last = -1;
-    for (; j <= r.jB && g.ns < kSlots; ++j) {
-        if (is_direct(p, j)) continue;
-        if (g.ns == (int)threadIdx.x) {
-            gs->lay[g.ns] = j;
-            gs->lid[g.ns] = p.desc[j].layer_id;
-            gs->tf[g.ns] = p.desc[j].tile_first;
-            gs->tfe[g.ns] = p.desc[j + 1].tile_first;
-            gs->start[g.ns] = p.desc[j].start;
-            gs->end[g.ns] = p.desc[j].end;
-            gs->out_off[g.ns] = p.desc[j].out_off;
+// Fills the table of the CTA's streamed layers; returns how many there are (at most
+// kMaxLocalLayers: checked on the host).
+__device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRange& r, LayerTable* lt,
+                                                 uint32_t* scratch) {
+    int nl = 0;
+    for (int j0 = r.jA; j0 <= r.jB; j0 += kSelThreads) {
+        const int j = j0 + (int)threadIdx.x;
+        const bool streamed = j <= r.jB && !is_direct(p, j);
+        uint32_t tot;
+        const int c = nl + (int)block_excl_scan(streamed ? 1u : 0u, scratch, tot);
+        if (streamed && c < kMaxLocalLayers) {
+            lt->j[c] = j;
+            lt->lid[c] = p.desc[j].layer_id;
+            lt->tf[c] = p.desc[j].tile_first;
+            lt->tfe[c] = p.desc[j + 1].tile_first;
+            lt->start[c] = p.desc[j].start;
+            lt->end[c] = p.desc[j].end;
+            lt->out_off[c] = p.desc[j].out_off;
         }
-        if (first < 0) first = j;
-        last = j;
-        ++g.ns;
-    }
-    jn = j;
-    if (g.ns == 0) return false;
-    const int tf = p.desc[first].tile_first, tfe = p.desc[last + 1].tile_first;
-    g.qa = r.q0 > tf ? r.q0 : tf;
-    g.qb = r.q1 < tfe ? r.q1 : tfe;
-    return true;
-}
-
-// Per-warp walk over the group's tiles: tile q belongs to slot s (or to a direct layer that
-// lies between two slots: result < 0).  `s` is a cursor that only moves forward.
-__device__ __forceinline__ int tile_slot(const Group& g, const GroupShared* gs, int q, int& s) {
-    while (s < g.ns - 1 && q >= gs->tfe[s]) ++s;
-    return (q >= gs->tf[s] && q < gs->tfe[s]) ? s : -1;
-}
-
-// After the CTA has flushed its counts of the group's layers (a __syncthreads() lies between
-// the flush and this call): take a ticket per layer; last[s] = this CTA flushed the layer's
-// last tiles, so the layer's histogram is complete.
-template <int kTicket>
-__device__ __forceinline__ void take_tickets(const SelParams& p, const CtaRange& r, const Group& g,
-                                             const GroupShared* gs, uint32_t* last) {
-    if ((int)threadIdx.x < g.ns) {
-        const int sl = threadIdx.x;
-        LayerState* st = p.state + gs->lid[sl];
-        uint32_t* t = kTicket == 1 ? &st->ticket1 : kTicket == 2 ? &st->ticket2 : &st->ticket3;
-        const int a = r.q0 > gs->tf[sl] ? r.q0 : gs->tf[sl], b = r.q1 < gs->tfe[sl] ? r.q1 : gs->tfe[sl];
-        const uint32_t mine = b > a ? (uint32_t)(b - a) : 0u;   // this CTA's tiles of the layer
-        __threadfence();
-        const uint32_t old = atomicAdd(t, mine);
-        last[sl] = (old + mine == (uint32_t)(gs->tfe[sl] - gs->tf[sl])) ? 1u : 0u;
+        nl += (int)tot;
     }
     __syncthreads();
+    return nl < kMaxLocalLayers ? nl : kMaxLocalLayers;
+}
+
+// Per-warp walk over tiles in ascending order: tile q belongs to local layer c (or to a direct
+// layer lying between two streamed ones: result < 0).  `c` is a cursor that only moves forward.
+__device__ __forceinline__ int tile_layer(const LayerTable* lt, int nl, int q, int& c) {
+    while (c < nl - 1 && q >= lt->tfe[c]) ++c;
+    return (q >= lt->tf[c] && q < lt->tfe[c]) ? c : -1;
 }
 
 // ---------------------------------------------------------------------------------
-// step A: level-1 histograms
+// step A: level-1 histograms, kSlots layers at a time
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r, unsigned char* smem) {
+__device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r, const LayerTable* lt, int nl,
+                                           unsigned char* smem) {
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem + kSmMain);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    Group g;
-    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
-    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
-        __syncthreads();   // the group's facts are published
-        for (int i = threadIdx.x; i < g.ns * kBins1; i += kSelThreads) hist[i] = 0;
+    for (int c0 = 0; c0 < nl; c0 += kSlots) {
+        const int ns = nl - c0 < kSlots ? nl - c0 : kSlots;
+        for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) hist[i] = 0;
         __syncthreads();
-        int s = 0;
-        for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            const int slot = tile_slot(g, gs, q, s);
-            if (slot < 0) continue;
-            const TileSpan ts = tile_span(gs->start[slot], gs->end[slot], gs->tf[slot], q);
-            hist_tile(p.acc, ts, hist + slot * kBins1, lane);
+        const int qa = r.q0 > lt->tf[c0] ? r.q0 : lt->tf[c0];
+        const int qb = r.q1 < lt->tfe[c0 + ns - 1] ? r.q1 : lt->tfe[c0 + ns - 1];
+        int c = c0;
+        for (int q = qa + warp; q < qb; q += kSelWarps) {
+            const int cl = tile_layer(lt, c0 + ns, q, c);
+            if (cl < 0) continue;
+            const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
+            hist_tile(p.acc, ts, hist + (cl - c0) * kBins1, lane);
         }
         __syncthreads();
-        for (int i = threadIdx.x; i < g.ns * kBins1; i += kSelThreads) {
-            const uint32_t c = hist[i];
-            if (c) atomicAdd(p.hist1 + (size_t)gs->lid[i / kBins1] * kBins1 + (i % kBins1), c);
+        for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) {
+            const uint32_t cnt = hist[i];
+            if (cnt) atomicAdd(p.hist1 + (size_t)lt->lid[c0 + i / kBins1] * kBins1 + (i % kBins1), cnt);
         }
         __syncthreads();
-        take_tickets<1>(p, r, g, gs, misc + kMLast);
-        for (int s2 = 0; s2 < g.ns; ++s2) {
-            if (!misc[kMLast + s2]) continue;   // uniform over the CTA
-            const int j = gs->lay[s2];
-            const int lid = p.desc[j].layer_id;
+        // ticket per layer: the CTA that flushes a layer's last tiles sees the complete histogram
+        if ((int)threadIdx.x < ns) {
+            const int cl = c0 + threadIdx.x;
+            const int a = r.q0 > lt->tf[cl] ? r.q0 : lt->tf[cl], b = r.q1 < lt->tfe[cl] ? r.q1 : lt->tfe[cl];
+            const uint32_t mine = b > a ? (uint32_t)(b - a) : 0u;
             __threadfence();
-            block_scan_select<true>(p.hist1 + (size_t)lid * kBins1, kBins1, (uint32_t)p.desc[j].k,
-                                    misc + kMScratch, misc + kMOut3);
+            const uint32_t old = atomicAdd(&p.state[lt->lid[cl]].ticket1, mine);
+            misc[kMLast + threadIdx.x] = (old + mine == (uint32_t)(lt->tfe[cl] - lt->tf[cl])) ? 1u : 0u;
+        }
+        __syncthreads();
+        for (int s = 0; s < ns; ++s) {
+            if (!misc[kMLast + s]) continue;   // uniform over the CTA
+            const int cl = c0 + s;
+            const int lid = lt->lid[cl];
+            __threadfence();
+            block_scan_select<kBins1, true>(p.hist1 + (size_t)lid * kBins1, (uint32_t)p.desc[lt->j[cl]].k,
+                                            misc + kMScratch, misc + kMOut3);
             if (threadIdx.x == 0) {
                 p.state[lid].b1 = misc[kMOut3];
                 p.state[lid].above1 = misc[kMOut3 + 1];
             }
             __syncthreads();
         }
-        __syncthreads();   // the group's facts are no longer read
+        __syncthreads();
     }
 }
 
 // ---------------------------------------------------------------------------------
-// step B: staging pass + level-2 histograms
+// step B: staging pass + level-2 histograms, kBSlots layers at a time
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& r, const Stage& st,
-                                            unsigned char* smem) {
+__device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
+                                            TileTable* tt, const Stage& st, unsigned char* smem) {
     uint32_t* hist2s = reinterpret_cast<uint32_t*>(smem + kSmAux);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) misc[kMCursor] = 0;
-    Group g;
-    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
-    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
-        __syncthreads();   // the group's facts are published
-        if ((int)threadIdx.x < g.ns) misc[kMTabA + threadIdx.x] = __ldcg(&p.state[gs->lid[threadIdx.x]].b1);
-        for (int i = threadIdx.x; i < g.ns * kBins2; i += kSelThreads) hist2s[i] = 0;
+    for (int c0 = 0; c0 < nl; c0 += kBSlots) {
+        const int ns = nl - c0 < kBSlots ? nl - c0 : kBSlots;
+        if ((int)threadIdx.x < ns) {
+            const LayerState* ls = p.state + lt->lid[c0 + threadIdx.x];
+            misc[kMTab + threadIdx.x] = __ldcg(&ls->b1);
+            lt->v1[c0 + threadIdx.x] = (uint32_t)p.desc[lt->j[c0 + threadIdx.x]].k - __ldcg(&ls->above1);   // krem1
+        }
+        for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) hist2s[i] = 0;
         __syncthreads();
-        int s = 0;
-        for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            const int slot = tile_slot(g, gs, q, s);
-            if (slot < 0) continue;
-            const TileSpan ts = tile_span(gs->start[slot], gs->end[slot], gs->tf[slot], q);
-            const uint2 fn = filter_tile(p.acc, ts, misc[kMTabA + slot], hist2s + slot * kBins2, st,
-                                         reinterpret_cast<uint2*>(smem + kSmMain), misc + kMCursor, lane);
-            if (lane == 0) p.tt[q] = make_uint4(fn.x, fn.y, 0u, 0u);
+        const int qa = r.q0 > lt->tf[c0] ? r.q0 : lt->tf[c0];
+        const int qb = r.q1 < lt->tfe[c0 + ns - 1] ? r.q1 : lt->tfe[c0 + ns - 1];
+        int c = c0;
+        for (int q = qa + warp; q < qb; q += kSelWarps) {
+            const int cl = tile_layer(lt, c0 + ns, q, c);
+            if (cl < 0) continue;
+            const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
+            const uint32_t lq = (uint32_t)(q - r.q0);
+            const uint2 fn = filter_tile(p.acc, ts, misc[kMTab + cl - c0], hist2s + (cl - c0) * kBins2, st,
+                                         pack_y(0u, (uint32_t)cl, lq), misc + kMCursor, lane);
+            if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
         }
         __syncthreads();
-        for (int i = threadIdx.x; i < g.ns * kBins2; i += kSelThreads) {
-            const uint32_t c = hist2s[i];
-            if (c) atomicAdd(p.hist2 + (size_t)gs->lid[i / kBins2] * kBins2 + (i % kBins2), c);
+        for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) {
+            const uint32_t cnt = hist2s[i];
+            if (cnt) atomicAdd(p.hist2 + (size_t)lt->lid[c0 + i / kBins2] * kBins2 + (i % kBins2), cnt);
         }
         __syncthreads();
-        take_tickets<2>(p, r, g, gs, misc + kMLast);
-        for (int s2 = 0; s2 < g.ns; ++s2) {
-            if (!misc[kMLast + s2]) continue;   // uniform over the CTA
-            const int j = gs->lay[s2];
-            const int lid = p.desc[j].layer_id;
-            __threadfence();
-            const uint32_t krem1 = (uint32_t)p.desc[j].k - __ldcg(&p.state[lid].above1);
-            block_scan_select<true>(p.hist2 + (size_t)lid * kBins2, kBins2, krem1, misc + kMScratch, misc + kMOut3);
-            if (threadIdx.x == 0) {
-                p.state[lid].b2 = misc[kMOut3];
-                p.state[lid].krem2 = krem1 - misc[kMOut3 + 1];
-            }
-            __syncthreads();
-        }
-        __syncthreads();   // the group's facts are no longer read
     }
 }
 
 // ---------------------------------------------------------------------------------
-// step S2: level-3 histograms over the staged entries of bucket (b1, b2)
+// step S2: bucket b2 of every local layer, then the level-3 histograms of the staged entries
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_hist3(const SelParams& p, const CtaRange& r, const Stage& st,
+__device__ __forceinline__ void step_hist3(const SelParams& p, LayerTable* lt, int nl, const Stage& st,
                                            unsigned char* smem) {
     uint32_t* h3 = reinterpret_cast<uint32_t*>(smem + kSmAux);
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
+    const uint32_t* misc = reinterpret_cast<const uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint2* res_sh = reinterpret_cast<const uint2*>(smem + kSmMain);
-    Group g;
-    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
-    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
-        __syncthreads();   // the group's facts are published
-        if ((int)threadIdx.x < g.ns) {
-            const LayerState* ls = p.state + gs->lid[threadIdx.x];
-            misc[kMTabA + threadIdx.x] = (__ldcg(&ls->b1) << (kShift1 - kShift2)) | __ldcg(&ls->b2);
+    const uint32_t total = misc[kMCursor];
+    if (p.timing && threadIdx.x == 0) { atomicMax(p.timing + 14, (unsigned long long)total); atomicAdd(p.timing + 15, (unsigned long long)total); }
+    for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer
+        const int lid = lt->lid[c];
+        uint32_t b2, above2;
+        warp_scan_select<kBins2 / 32>(p.hist2 + (size_t)lid * kBins2, lt->v1[c], lane, b2, above2);
+        const uint32_t b1 = __ldcg(&p.state[lid].b1);
+        __syncwarp();
+        if (lane == 0) {
+            lt->v0[c] = (b1 << (kShift1 - kShift2)) | b2;   // key >> kShift2 of the candidates
+            lt->v1[c] = lt->v1[c] - above2;                 // krem2
         }
-        for (int i = threadIdx.x; i < g.ns * kBins3; i += kSelThreads) h3[i] = 0;
+    }
+    for (int c0 = 0; c0 < nl; c0 += kS2Chunk) {
+        const int ns = nl - c0 < kS2Chunk ? nl - c0 : kS2Chunk;
+        for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) h3[i] = 0;
         __syncthreads();
-        stamp(p, 8);
-        int s = 0;
-        TtBatch tb;
-        for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            if ((q - g.qa - warp) % (32 * kSelWarps) == 0) tt_fetch(p, q, g.qb, lane, tb);
-            const int slot = tile_slot(g, gs, q, s);
-            if (slot < 0) continue;
-            const uint4 t = tt_get(tb, q);
-            const uint32_t prefix = misc[kMTabA + slot];
-            const bool all_res = t.x + t.y <= (uint32_t)kResident;
-            for (uint32_t e = lane; e < t.y; e += 32) {
-                const uint32_t key = key_of(stage_get_tile(st, res_sh, all_res, t.x + e).x);
-                if ((key >> kShift2) == prefix) atomicAdd(&h3[slot * kBins3 + (key & (kBins3 - 1))], 1u);
-            }
-        }
-        stamp(p, 9);
-        __syncthreads();
-        for (int i = threadIdx.x; i < g.ns * kBins3; i += kSelThreads) {
-            const uint32_t c = h3[i];
-            if (c) atomicAdd(p.hist3 + (size_t)gs->lid[i / kBins3] * kBins3 + (i % kBins3), c);
+        for (uint32_t pos = threadIdx.x; pos < total; pos += kSelThreads) {
+            const uint2 ent = stage_get(st, pos);
+            const int c = (int)y_layer(ent.y);
+            const uint32_t key = key_of(ent.x);
+            if (c >= c0 && c < c0 + ns && (key >> kShift2) == lt->v0[c])
+                atomicAdd(&h3[(c - c0) * kBins3 + (key & (kBins3 - 1))], 1u);
         }
         __syncthreads();
-        stamp(p, 10);
-        take_tickets<3>(p, r, g, gs, misc + kMLast);
-        stamp(p, 11);
-        for (int s2 = 0; s2 < g.ns; ++s2) {
-            if (!misc[kMLast + s2]) continue;   // uniform over the CTA
-            const int lid = gs->lid[s2];
-            __threadfence();
-            const uint32_t krem2 = __ldcg(&p.state[lid].krem2);
-            block_scan_select<true>(p.hist3 + (size_t)lid * kBins3, kBins3, krem2, misc + kMScratch, misc + kMOut3);
-            if (threadIdx.x == 0) {
-                const uint32_t b1 = __ldcg(&p.state[lid].b1), b2 = __ldcg(&p.state[lid].b2);
-                p.state[lid].T = (b1 << kShift1) | (b2 << kShift2) | misc[kMOut3];
-                p.state[lid].need = krem2 - misc[kMOut3 + 1];
-            }
-            __syncthreads();
+        for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) {
+            const uint32_t cnt = h3[i];
+            if (cnt) atomicAdd(p.hist3 + (size_t)lt->lid[c0 + i / kBins3] * kBins3 + (i % kBins3), cnt);
         }
-        __syncthreads();   // the group's facts are no longer read
+        __syncthreads();
     }
 }
 
 // ---------------------------------------------------------------------------------
-// step S3: per tile and per (CTA, layer): staged entries above T / equal to T
+// step S3: threshold T of every local layer, counts per tile, totals per (CTA, layer)
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r, const Stage& st,
-                                           unsigned char* smem) {
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
+__device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
+                                           TileTable* tt, const Stage& st, unsigned char* smem) {
+    const uint32_t* misc = reinterpret_cast<const uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint2* res_sh = reinterpret_cast<const uint2*>(smem + kSmMain);
-    Group g;
-    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
-    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
-        __syncthreads();   // the group's facts are published
-        if ((int)threadIdx.x < g.ns) {
-            misc[kMTabA + threadIdx.x] = __ldcg(&p.state[gs->lid[threadIdx.x]].T);
-            misc[kMTotGt + threadIdx.x] = 0;
-            misc[kMTotEq + threadIdx.x] = 0;
+    const uint32_t total = misc[kMCursor];
+    for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer
+        uint32_t b3, above3;
+        warp_scan_select<kBins3 / 32>(p.hist3 + (size_t)lt->lid[c] * kBins3, lt->v1[c], lane, b3, above3);
+        __syncwarp();
+        if (lane == 0) {
+            lt->v0[c] = (lt->v0[c] << kShift2) | b3;   // T
+            lt->v1[c] = lt->v1[c] - above3;            // need
         }
-        __syncthreads();
-        int s = 0;
-        TtBatch tb;
-        for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            if ((q - g.qa - warp) % (32 * kSelWarps) == 0) tt_fetch(p, q, g.qb, lane, tb);
-            const int slot = tile_slot(g, gs, q, s);
-            if (slot < 0) continue;
-            const uint4 t = tt_get(tb, q);
-            const uint32_t T = misc[kMTabA + slot];
-            uint32_t n_gt = 0, n_eq = 0;
-            const bool all_res = t.x + t.y <= (uint32_t)kResident;
-            for (uint32_t e = lane; e < t.y; e += 32) {
-                const uint32_t key = key_of(stage_get_tile(st, res_sh, all_res, t.x + e).x);
-                n_gt += key > T;
-                n_eq += key == T;
-            }
-            n_gt = __reduce_add_sync(0xffffffffu, n_gt);
-            n_eq = __reduce_add_sync(0xffffffffu, n_eq);
-            if (lane == 0) {
-                p.tt[q] = make_uint4(t.x, t.y, n_gt, n_eq);
-                atomicAdd(&misc[kMTotGt + slot], n_gt);
-                atomicAdd(&misc[kMTotEq + slot], n_eq);
-            }
-        }
-        __syncthreads();
-        if ((int)threadIdx.x < g.ns)
-            p.runge[blockIdx.x + gs->lay[threadIdx.x]] = make_uint2(misc[kMTotGt + threadIdx.x], misc[kMTotEq + threadIdx.x]);
-        __syncthreads();
+    }
+    for (int i = threadIdx.x; i < r.q1 - r.q0; i += kSelThreads) tt->ge[i] = 0;
+    __syncthreads();
+    for (uint32_t pos = threadIdx.x; pos < total; pos += kSelThreads) {
+        const uint2 ent = stage_get(st, pos);
+        const uint32_t key = key_of(ent.x), T = lt->v0[y_layer(ent.y)];
+        if (key > T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u);
+        else if (key == T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u << 16);
+    }
+    __syncthreads();
+    for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of its tiles here
+        const int a = (r.q0 > lt->tf[c] ? r.q0 : lt->tf[c]) - r.q0, b = (r.q1 < lt->tfe[c] ? r.q1 : lt->tfe[c]) - r.q0;
+        uint32_t gt = 0, eq = 0;
+        for (int i = a + lane; i < b; i += 32) { const uint32_t v = tt->ge[i]; gt += v & 0xffffu; eq += v >> 16; }
+        gt = __reduce_add_sync(0xffffffffu, gt);
+        eq = __reduce_add_sync(0xffffffffu, eq);
+        if (lane == 0) p.runge[blockIdx.x + lt->j[c]] = make_uint2(gt, eq);
     }
 }
 
@@ -624,11 +607,11 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
 __device__ __forceinline__ void emit_batch(const SelParams& p, int64_t out_off, int64_t elem0, bool valid,
                                            uint32_t bits, int64_t off, uint32_t T, uint32_t need,
                                            uint32_t& gt_before, uint32_t& eq_before, int lane) {
-    const uint32_t lt = (1u << lane) - 1u;
+    const uint32_t lt_mask = (1u << lane) - 1u;
     const uint32_t key = key_of(bits);
     const bool gt = valid && key > T, eq = valid && key == T;
     const unsigned gt_b = __ballot_sync(0xffffffffu, gt), eq_b = __ballot_sync(0xffffffffu, eq);
-    const uint32_t my_gt = gt_before + __popc(gt_b & lt), my_eq = eq_before + __popc(eq_b & lt);
+    const uint32_t my_gt = gt_before + __popc(gt_b & lt_mask), my_eq = eq_before + __popc(eq_b & lt_mask);
     if (gt || (eq && my_eq < need)) {
         // selected entries before me: every larger key, and the first `need` equal ones
         const int64_t pos = out_off + my_gt + (my_eq < need ? my_eq : need);
@@ -641,86 +624,73 @@ __device__ __forceinline__ void emit_batch(const SelParams& p, int64_t out_off, 
 }
 
 // ---------------------------------------------------------------------------------
-// step S4: prefix over the CTAs before this one, scan of the own tiles, ordered write
+// step S4: totals of the CTAs before this one, scan of the own tiles, ordered write
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r, const Stage& st,
-                                          unsigned char* smem) {
+__device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
+                                          const TileTable* tt, const Stage& st, unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
+    uint2* pref = reinterpret_cast<uint2*>(smem + kSmPref);
     uint32_t* scratch = misc + kMScratch;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint2* res_sh = reinterpret_cast<const uint2*>(smem + kSmMain);
-    Group g;
-    GroupShared* gs = reinterpret_cast<GroupShared*>(smem + kSmGroup);
-    for (int jn = r.jA; next_group(p, r, jn, g, gs);) {
-        __syncthreads();   // the group's facts are published
-        for (int s2 = 0; s2 < g.ns; ++s2) {
-            const int j = gs->lay[s2];
-            const int tf = p.desc[j].tile_first, tfe = p.desc[j + 1].tile_first;
-            // totals of the CTAs that hold earlier tiles of the layer
-            const int b0 = cta_of_tile(p, tf);
-            uint32_t v_gt = 0, v_eq = 0;
-            for (int b = b0 + (int)threadIdx.x; b < (int)blockIdx.x; b += kSelThreads) {
-                if (cta_q0(p, b) < cta_q0(p, b + 1)) {
-                    const uint2 c = __ldcg(p.runge + b + j);
-                    v_gt += c.x;
-                    v_eq += c.y;
+    for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of earlier CTAs
+        const int j = lt->j[c];
+        uint32_t gt = 0, eq = 0;
+        for (int b = cta_of_tile(p, lt->tf[c]) + lane; b < (int)blockIdx.x; b += 32) {
+            if (cta_q0(p, b) < cta_q0(p, b + 1)) {
+                const uint2 v = __ldcg(p.runge + b + j);
+                gt += v.x;
+                eq += v.y;
+            }
+        }
+        gt = __reduce_add_sync(0xffffffffu, gt);
+        eq = __reduce_add_sync(0xffffffffu, eq);
+        if (lane == 0) { lt->base_gt[c] = gt; lt->base_eq[c] = eq; }
+    }
+    __syncthreads();
+    for (int c = 0; c < nl; ++c) {
+        const int ta = (r.q0 > lt->tf[c] ? r.q0 : lt->tf[c]) - r.q0, tb = (r.q1 < lt->tfe[c] ? r.q1 : lt->tfe[c]) - r.q0;
+        const uint32_t T = lt->v0[c], need = lt->v1[c];
+        const int64_t start = lt->start[c], out_off = lt->out_off[c];
+        const int tf = lt->tf[c];
+        uint32_t base_gt = lt->base_gt[c], base_eq = lt->base_eq[c];
+        for (int t0 = ta; t0 < tb; t0 += kSelThreads) {   // batches of kSelThreads tiles
+            const int i = t0 + (int)threadIdx.x;
+            const uint32_t v = i < tb ? tt->ge[i] : 0u;
+            uint32_t tot_gt, tot_eq;
+            const uint32_t e_gt = block_excl_scan(v & 0xffffu, scratch, tot_gt);
+            const uint32_t e_eq = block_excl_scan(v >> 16, scratch, tot_eq);
+            pref[threadIdx.x] = make_uint2(base_gt + e_gt, base_eq + e_eq);
+            __syncthreads();
+            const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
+            for (int lq = t0 + warp; lq < tend; lq += kSelWarps) {
+                const uint32_t n = tt->n[lq];
+                if (n == 0) continue;
+                const uint32_t first = tt->first[lq];
+                const int64_t lo = (start / kTile + (r.q0 + lq - tf)) * kTile;
+                uint32_t gt_before = pref[lq - t0].x, eq_before = pref[lq - t0].y;
+                for (uint32_t e0 = 0; e0 < n; e0 += 32) {
+                    const uint32_t e = e0 + lane;
+                    const bool valid = e < n;
+                    uint2 ent = make_uint2(0u, 0u);
+                    if (valid) ent = stage_get(st, first + e);
+                    emit_batch(p, out_off, lo, valid, ent.x, (int64_t)y_off(ent.y), T, need, gt_before, eq_before, lane);
                 }
             }
-            uint32_t base_gt, base_eq;
-            block_excl_scan(v_gt, scratch, base_gt);
-            block_excl_scan(v_eq, scratch, base_eq);
-            // exclusive scan over this CTA's tiles of the layer, written back over the counts
-            const int ta = r.q0 > tf ? r.q0 : tf, tb = r.q1 < tfe ? r.q1 : tfe;
-            for (int t0 = ta; t0 < tb; t0 += kSelThreads) {
-                const int q = t0 + (int)threadIdx.x;
-                uint4 t = make_uint4(0u, 0u, 0u, 0u);
-                if (q < tb) t = __ldcg(p.tt + q);
-                uint32_t tot_gt, tot_eq;
-                const uint32_t e_gt = block_excl_scan(t.z, scratch, tot_gt);
-                const uint32_t e_eq = block_excl_scan(t.w, scratch, tot_eq);
-                if (q < tb) p.tt[q] = make_uint4(t.x, t.y, base_gt + e_gt, base_eq + e_eq);
-                base_gt += tot_gt;
-                base_eq += tot_eq;
-            }
-            if (threadIdx.x == 0) {
-                const LayerState* ls = p.state + p.desc[j].layer_id;
-                misc[kMTabA + s2] = __ldcg(&ls->T);
-                misc[kMTabB + s2] = __ldcg(&ls->need);
-            }
+            base_gt += tot_gt;
+            base_eq += tot_eq;
+            __syncthreads();   // pref is rewritten by the next batch
         }
-        __syncthreads();
-        int s = 0;
-        TtBatch tb;
-        for (int q = g.qa + warp; q < g.qb; q += kSelWarps) {
-            if ((q - g.qa - warp) % (32 * kSelWarps) == 0) tt_fetch(p, q, g.qb, lane, tb);
-            const int slot = tile_slot(g, gs, q, s);
-            if (slot < 0) continue;
-            const uint4 t = tt_get(tb, q);
-            if (t.y == 0) continue;
-            const uint32_t T = misc[kMTabA + slot], need = misc[kMTabB + slot];
-            const int64_t lo = (gs->start[slot] / kTile + (q - gs->tf[slot])) * kTile;
-            const int64_t out_off = gs->out_off[slot];
-            uint32_t gt_before = t.z, eq_before = t.w;
-            const bool all_res = t.x + t.y <= (uint32_t)kResident;
-            for (uint32_t e0 = 0; e0 < t.y; e0 += 32) {
-                const uint32_t e = e0 + lane;
-                const bool valid = e < t.y;
-                uint2 ent = make_uint2(0u, 0u);
-                if (valid) ent = stage_get_tile(st, res_sh, all_res, t.x + e);
-                emit_batch(p, out_off, lo, valid, ent.x, (int64_t)ent.y, T, need, gt_before, eq_before, lane);
-            }
-        }
-        __syncthreads();
     }
 }
 
 // ---------------------------------------------------------------------------------
 // direct layers: one CTA loads the layer whole and finishes it from shared memory
+// (digits: bits 30..19, 18..9, 8..0)
 // ---------------------------------------------------------------------------------
 __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsigned char* smem) {
     uint32_t* skey = reinterpret_cast<uint32_t*>(smem + kSmMain);
     uint32_t* h1 = reinterpret_cast<uint32_t*>(smem + kSmAux);
-    uint32_t* h = h1 + kBins1;
+    uint32_t* h = h1 + kDBins1;
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint32_t* scratch = misc + kMScratch;
     uint32_t* out3 = misc + kMOut3;
@@ -731,8 +701,8 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
     const uint32_t k = (uint32_t)p.desc[j].k;
     const int64_t out_off = p.desc[j].out_off;
     const uint32_t* x = reinterpret_cast<const uint32_t*>(p.acc + start);
-    for (int i = tid; i < kBins1; i += kSelThreads) h1[i] = 0;
-    for (int i = tid; i < kBins2; i += kSelThreads) h[i] = 0;
+    for (int i = tid; i < kDBins1; i += kSelThreads) h1[i] = 0;
+    for (int i = tid; i < kDBins2; i += kSelThreads) h[i] = 0;
     __syncthreads();
     // level 1 over the whole layer
     for (uint32_t fb = 0; fb < n; fb += 8 * kSelThreads) {
@@ -747,35 +717,35 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
             const uint32_t f = fb + u * kSelThreads + tid;
             if (f < n) {
                 skey[f] = v[u];
-                atomicAdd(&h1[key_of(v[u]) >> kShift1], 1u);
+                atomicAdd(&h1[key_of(v[u]) >> kDShift1], 1u);
             }
         }
     }
     __syncthreads();
-    block_scan_select<false>(h1, kBins1, k, scratch, out3);
+    block_scan_select<kDBins1, false>(h1, k, scratch, out3);
     const uint32_t b1 = out3[0], above1 = out3[1];
     __syncthreads();
     // level 2 inside bucket b1
     for (uint32_t f = tid; f < n; f += kSelThreads) {
         const uint32_t key = key_of(skey[f]);
-        if ((key >> kShift1) == b1) atomicAdd(&h[(key >> kShift2) & (kBins2 - 1)], 1u);
+        if ((key >> kDShift1) == b1) atomicAdd(&h[(key >> kDShift2) & (kDBins2 - 1)], 1u);
     }
     __syncthreads();
-    block_scan_select<false>(h, kBins2, k - above1, scratch, out3);
+    block_scan_select<kDBins2, false>(h, k - above1, scratch, out3);
     const uint32_t b2 = out3[0];
     const uint32_t krem2 = k - above1 - out3[1];
     __syncthreads();
-    for (int i = tid; i < kBins3; i += kSelThreads) h[i] = 0;
+    for (int i = tid; i < kDBins3; i += kSelThreads) h[i] = 0;
     __syncthreads();
     // level 3 inside (b1, b2)
-    const uint32_t prefix = (b1 << (kShift1 - kShift2)) | b2;
+    const uint32_t prefix = (b1 << (kDShift1 - kDShift2)) | b2;
     for (uint32_t f = tid; f < n; f += kSelThreads) {
         const uint32_t key = key_of(skey[f]);
-        if ((key >> kShift2) == prefix) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+        if ((key >> kDShift2) == prefix) atomicAdd(&h[key & (kDBins3 - 1)], 1u);
     }
     __syncthreads();
-    block_scan_select<false>(h, kBins3, krem2, scratch, out3);
-    const uint32_t T = (prefix << kShift2) | out3[0];
+    block_scan_select<kDBins3, false>(h, krem2, scratch, out3);
+    const uint32_t T = (prefix << kDShift2) | out3[0];
     const uint32_t need = krem2 - out3[1];
     __syncthreads();
     // every warp counts its contiguous share, then the ordered, coalesced write
@@ -816,7 +786,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         p.timing[0] = t;
     }
+    LayerTable* lt = reinterpret_cast<LayerTable*>(smem + kSmLayer);
+    TileTable* tt = reinterpret_cast<TileTable*>(smem + kSmTile);
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const CtaRange r = cta_range(p);
+    const int nl = build_layer_table(p, r, lt, misc + kMScratch);
     Stage st;
     st.res = reinterpret_cast<uint2*>(smem + kSmMain);
     st.spill = p.staging;
@@ -826,20 +800,21 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
         st.spill = p.staging + p.desc[r.jA].elem_off + (ts.lo + ts.s - p.desc[r.jA].start);
     }
 
-    step_hist1(p, r, smem);
+    step_hist1(p, r, lt, nl, smem);
     stamp(p, 1);
     grid.sync();
-    step_filter(p, r, st, smem);
+    step_filter(p, r, lt, nl, tt, st, smem);
     stamp(p, 2);
     grid.sync();
-    step_hist3(p, r, st, smem);
+    step_hist3(p, lt, nl, st, smem);
     stamp(p, 3);
     grid.sync();
-    step_count(p, r, st, smem);
+    step_count(p, r, lt, nl, tt, st, smem);
     stamp(p, 4);
     grid.sync();
-    step_emit(p, r, st, smem);
+    step_emit(p, r, lt, nl, tt, st, smem);
     stamp(p, 5);
+    __syncthreads();
     for (int j = blockIdx.x; j < p.n_my; j += gridDim.x)
         if (is_direct(p, j)) resolve_direct(p, j, smem);   // uniform over the CTA
     stamp(p, 6);
@@ -862,15 +837,9 @@ deft_status launch_select(const SelParams& p, cudaStream_t stream) {
                                            kSmemBytes));
         attr_dev = dev;
     }
-    // one CTA per SM at most (co-resident by construction); fewer when the rank is small
-    const int sms = sm_count();
-    int want = (p.tiles + 1) / 2;
-    if (want < p.n_my) want = p.n_my;
-    if (want < 1) want = 1;
-    const int grid = want < sms ? want : sms;
     SelParams args = p;
     void* kargs[] = {&args};
-    DEFT_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_select_fused), dim3(grid),
+    DEFT_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_select_fused), dim3(p.grid),
                                               dim3(kSelThreads), kargs, kSmemBytes, stream));
     return DEFT_OK;
 }

@@ -48,12 +48,15 @@ static_assert(kBSlots * kBins2 * 4 <= kSmAuxBytes && kS2Chunk * kBins3 * 4 <= kS
 constexpr int kSmTile = kSmAux + kSmAuxBytes;    // per local tile: first entry, entries, counts
 constexpr int kSmTileBytes = kMaxLocalTiles * 10;
 constexpr int kSmLayer = kSmTile + kSmTileBytes; // per local streamed layer, see LayerTable
-constexpr int kSmLayerBytes = kMaxLocalLayers * 64;
+constexpr int kSmLayerBytes = kMaxLocalLayers * 64;   // >= sizeof(LayerTable)
 constexpr int kSmPref = kSmLayer + kSmLayerBytes;   // prefixes of one batch of tiles in S4
 constexpr int kSmPrefBytes = kSelThreads * 8;
 constexpr int kSmMisc = kSmPref + kSmPrefBytes;
 constexpr int kSmMiscBytes = 1024;
-constexpr int kSmemBytes = kSmMisc + kSmMiscBytes;
+constexpr int kSmTf = kSmMisc + kSmMiscBytes;       // tile_first of the rank's first layers (start-up search)
+constexpr int kTfCache = 1024;
+constexpr int kSmTfBytes = (kTfCache + 1) * 4 + 12;
+constexpr int kSmemBytes = kSmTf + kSmTfBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 enum MiscOff : int {   // word offsets inside the misc area
@@ -75,6 +78,7 @@ struct LayerTable {
     int64_t start[kMaxLocalLayers];  // first element
     int64_t end[kMaxLocalLayers];
     int64_t out_off[kMaxLocalLayers];
+    uint32_t k[kMaxLocalLayers];     // entries to select
     uint32_t v0[kMaxLocalLayers];    // step value: prefix (b1, b2) | T
     uint32_t v1[kMaxLocalLayers];    // step value: krem1 | krem2 | need
     uint32_t base_gt[kMaxLocalLayers];
@@ -379,14 +383,34 @@ struct CtaRange { int q0, q1, jA, jB; };
 
 __device__ __forceinline__ int cta_q0(const SelParams& p, int b) { return (int)((int64_t)p.tiles * b / gridDim.x); }
 
-__device__ __forceinline__ CtaRange cta_range(const SelParams& p) {
+// Largest j in [0, n-1] with tf[j] <= q (tf in shared memory).
+__device__ __forceinline__ int layer_of_tile_sh(const int* tf, int n, int q) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (tf[mid] <= q) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// The CTA's tiles and the layers they belong to.  The first kTfCache layers' tile_first are
+// fetched with one coalesced request so that the search does not chase cold global loads.
+__device__ __forceinline__ CtaRange cta_range(const SelParams& p, int* tf_cache) {
+    const int nc = p.n_my < kTfCache ? p.n_my : kTfCache;
+    for (int i = threadIdx.x; i <= nc; i += kSelThreads) tf_cache[i] = p.desc[i].tile_first;
+    __syncthreads();
     CtaRange r;
     r.q0 = cta_q0(p, blockIdx.x);
     r.q1 = cta_q0(p, blockIdx.x + 1);
     r.jA = 0; r.jB = -1;
     if (r.q0 < r.q1) {
-        r.jA = layer_of_tile(p.desc, p.n_my, r.q0);
-        r.jB = layer_of_tile(p.desc, p.n_my, r.q1 - 1);
+        if (p.n_my <= kTfCache || r.q1 <= tf_cache[nc]) {
+            r.jA = layer_of_tile_sh(tf_cache, nc, r.q0);
+            r.jB = layer_of_tile_sh(tf_cache, nc, r.q1 - 1);
+        } else {
+            r.jA = layer_of_tile(p.desc, p.n_my, r.q0);
+            r.jB = layer_of_tile(p.desc, p.n_my, r.q1 - 1);
+        }
     }
     return r;
 }
@@ -418,6 +442,7 @@ __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRa
             lt->start[c] = p.desc[j].start;
             lt->end[c] = p.desc[j].end;
             lt->out_off[c] = p.desc[j].out_off;
+            lt->k[c] = (uint32_t)p.desc[j].k;
         }
         nl += (int)tot;
     }
@@ -444,6 +469,7 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
         const int ns = nl - c0 < kSlots ? nl - c0 : kSlots;
         for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) hist[i] = 0;
         __syncthreads();
+        stamp(p, 8);
         const int qa = r.q0 > lt->tf[c0] ? r.q0 : lt->tf[c0];
         const int qb = r.q1 < lt->tfe[c0 + ns - 1] ? r.q1 : lt->tfe[c0 + ns - 1];
         int c = c0;
@@ -454,11 +480,13 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
             hist_tile(p.acc, ts, hist + (cl - c0) * kBins1, lane);
         }
         __syncthreads();
+        stamp(p, 9);
         for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) {
             const uint32_t cnt = hist[i];
             if (cnt) atomicAdd(p.hist1 + (size_t)lt->lid[c0 + i / kBins1] * kBins1 + (i % kBins1), cnt);
         }
         __syncthreads();
+        stamp(p, 10);
         // ticket per layer: the CTA that flushes a layer's last tiles sees the complete histogram
         if ((int)threadIdx.x < ns) {
             const int cl = c0 + threadIdx.x;
@@ -469,12 +497,13 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
             misc[kMLast + threadIdx.x] = (old + mine == (uint32_t)(lt->tfe[cl] - lt->tf[cl])) ? 1u : 0u;
         }
         __syncthreads();
+        stamp(p, 11);
         for (int s = 0; s < ns; ++s) {
             if (!misc[kMLast + s]) continue;   // uniform over the CTA
             const int cl = c0 + s;
             const int lid = lt->lid[cl];
             __threadfence();
-            block_scan_select<kBins1, true>(p.hist1 + (size_t)lid * kBins1, (uint32_t)p.desc[lt->j[cl]].k,
+            block_scan_select<kBins1, true>(p.hist1 + (size_t)lid * kBins1, lt->k[cl],
                                             misc + kMScratch, misc + kMOut3);
             if (threadIdx.x == 0) {
                 p.state[lid].b1 = misc[kMOut3];
@@ -500,7 +529,7 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
         if ((int)threadIdx.x < ns) {
             const LayerState* ls = p.state + lt->lid[c0 + threadIdx.x];
             misc[kMTab + threadIdx.x] = __ldcg(&ls->b1);
-            lt->v1[c0 + threadIdx.x] = (uint32_t)p.desc[lt->j[c0 + threadIdx.x]].k - __ldcg(&ls->above1);   // krem1
+            lt->v1[c0 + threadIdx.x] = lt->k[c0 + threadIdx.x] - __ldcg(&ls->above1);   // krem1
         }
         for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) hist2s[i] = 0;
         __syncthreads();
@@ -789,7 +818,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     LayerTable* lt = reinterpret_cast<LayerTable*>(smem + kSmLayer);
     TileTable* tt = reinterpret_cast<TileTable*>(smem + kSmTile);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
-    const CtaRange r = cta_range(p);
+    const CtaRange r = cta_range(p, reinterpret_cast<int*>(smem + kSmTf));
     const int nl = build_layer_table(p, r, lt, misc + kMScratch);
     Stage st;
     st.res = reinterpret_cast<uint2*>(smem + kSmMain);

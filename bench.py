@@ -175,6 +175,75 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------
 # the CUDA path
 # ------------------------------------------------------------------------------------------
+def run_sweep(args, dev):
+    """Selection time of the slowest simulated worker against full-vector Top-k on the same
+    GPU, over worker counts and densities (the shape of the paper's Figure 8 / Eq. 7-9 study).
+    Prints one table row per configuration to stderr and a JSON list to stdout."""
+    import torch
+    from paper_2307_03500_b200 import deft
+    from paper_2307_03500_b200.pipeline import DeftStep
+
+    stream = torch.cuda.current_stream()
+    base = W.WORKLOADS[args.workload]()
+    g = torch.from_numpy(base.gradient(0)).to(dev)
+    rows = []
+    print("%-12s %7s %4s %9s %5s | %9s %9s %9s %9s | %9s %8s %8s" % (
+        "workload", "d", "N", "k", "L", "norms_us", "host_us", "sel_max", "sel_sum", "topk_us", "speedup", "model"),
+        file=sys.stderr)
+    for d in ([args.density] if args.density else [0.1, 0.01, 0.001]):
+        for N in ([args.n_workers] if args.n_workers else [1, 2, 4, 8, 16, 32, 64]):
+            ds = DeftStep(base.sizes, N, d, device=dev)
+            e = torch.zeros_like(g)
+            reps, warm = 5, 3
+            sel, acc, host = [], [], []
+            for it in range(warm + reps):
+                tri = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(N)]
+                for t3 in tri:
+                    for x in t3:
+                        x.record(stream)
+                a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
+                a0.record(stream)
+                deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)
+                a1.record(stream)
+                ds.norms_h.copy_(ds.norms_d, non_blocking=True)
+                stream.synchronize()
+                t0 = time.perf_counter()
+                plan = ds.plan(ds.norms_h.numpy(), it)
+                t1 = time.perf_counter()
+                ds.select_and_update_all(e, plan, tri)
+                stream.synchronize()
+                if it >= warm:
+                    sel.append([a.elapsed_time(b) for (a, b, c) in tri])
+                    acc.append(a0.elapsed_time(a1))
+                    host.append((t1 - t0) * 1e3)
+            sel_med = np.median(np.array(sel), axis=0)
+            tk_val = torch.empty(ds.k, dtype=torch.float32, device=dev)
+            tk_idx = torch.empty(ds.k, dtype=torch.int64, device=dev)
+            tk = []
+            for i in range(3 + 5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                deft.deft_topk_baseline(e, ds.k, tk_val, tk_idx, ds.ws)
+                b.record(stream)
+                stream.synchronize()
+                if i >= 3:
+                    tk.append(a.elapsed_time(b))
+            t_topk = float(np.median(tk))
+            cost_max = float(plan.bin_load.max())
+            row = {"workload": base.name, "density": d, "n_workers": N, "k": ds.k, "layers": ds.L,
+                   "norms_us": float(np.median(acc)) * 1e3, "host_us": float(np.median(host)) * 1e3,
+                   "select_us_max": float(sel_med.max()) * 1e3, "select_us_sum": float(sel_med.sum()) * 1e3,
+                   "topk_us": t_topk * 1e3, "speedup_vs_topk": t_topk / float(sel_med.max()),
+                   "model_f_n": ds.n_g * math.log(ds.k) / cost_max if cost_max > 0 else None}
+            rows.append(row)
+            print("%-12s %7g %4d %9d %5d | %9.1f %9.1f %9.1f %9.1f | %9.1f %8.2f %8.2f" % (
+                base.name, d, N, ds.k, ds.L, row["norms_us"], row["host_us"], row["select_us_max"],
+                row["select_us_sum"], row["topk_us"], row["speedup_vs_topk"], row["model_f_n"] or 0.0), file=sys.stderr)
+            del ds, e, tk_val, tk_idx
+            torch.cuda.empty_cache()
+    print(json.dumps(rows))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -235,10 +304,14 @@ def run_ours(args):
         launches["n"] += 2
         marks = mark_pool.pop() if (rec is not None and mark_pool) else None
         ds.select_and_update_all(e, plan, marks)
-        launches["n"] += 2 * int((plan.rank_k > 0).sum())
+        launches["n"] += int((plan.rank_k > 0).sum())   # one fused kernel per rank (the zeroing is inside it)
         if rec is not None:
             rec.append({"acc": (e0, e1), "host_s": th1 - th0, "ranks": marks, "plan": plan})
         return plan
+
+    if args.mode == "sweep":
+        run_sweep(args, dev)
+        return
 
     if args.mode != "step":
         # profiling helper: repeat one call only (no JSON line; use it under ncu on a small workload)
@@ -407,8 +480,9 @@ def main():
     ap.add_argument("--density", type=float, default=0.0)
     ap.add_argument("--cpu-ranks", type=int, default=4, help="ranks the oracle runs for the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select"],
-                    help="step = the benchmark; the others repeat one call only, for profiler captures")
+    ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select", "sweep"],
+                    help="step = the benchmark; sweep = selection vs Top-k over N and d for --workload; "
+                         "the others repeat one call only, for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

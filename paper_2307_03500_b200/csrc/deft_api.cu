@@ -142,6 +142,12 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.grid = want < sms ? want : sms;
     // limits of one CTA's share: tiles, and streamed (non-direct) layers
     const LayerDesc* hd = plan_descs(plan_h, hdr->N) + R.desc_first;
+    p.interleave = (R.n_my == 1 && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) ? 1 : 0;
+    if (p.interleave) {
+        const int nsuper = (R.tiles + kSuper - 1) / kSuper;
+        if ((int64_t)((nsuper + p.grid - 1) / p.grid) * kSuper > kMaxLocalTiles) return DEFT_ERR_INVALID_ARG;
+        return launch_select(p, stream);
+    }
     int j = 0;
     for (int b = 0; b < p.grid; ++b) {
         const int q0 = (int)((int64_t)R.tiles * b / p.grid), q1 = (int)((int64_t)R.tiles * (b + 1) / p.grid);

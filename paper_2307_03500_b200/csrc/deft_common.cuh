@@ -37,6 +37,10 @@ constexpr int kResident = 16384;
 // Limits of one CTA's share of a rank (checked on the host before launch).
 constexpr int kMaxLocalTiles = 4096;    // tiles per CTA
 constexpr int kMaxLocalLayers = 256;    // streamed layers per CTA
+// A rank that is one layer of at least kInterleaveTiles tiles per CTA is split over the CTAs in
+// super-tiles of kSuper tiles dealt out round-robin instead of one contiguous run per CTA.
+constexpr int kSuper = 16;
+constexpr int kInterleaveTiles = 64;
 
 constexpr int kMaxRanks = 4096;      // workers per plan
 
@@ -130,7 +134,8 @@ inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
     w.zero_end = off;
     const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
     w.runge = off;    off += align_up(sizeof(uint2) * slots, 256);
-    w.staging = off;  off += align_up(sizeof(uint2) * (size_t)elems, 256);
+    // + slack: the interleaved split rounds a rank up to whole super-tiles
+    w.staging = off;  off += align_up(sizeof(uint2) * ((size_t)elems + 4 * (size_t)kSuper * kTile), 256);
     w.total = off;
     return w;
 }
@@ -149,6 +154,7 @@ struct SelParams {
     const LayerDesc* desc;           // the rank's layers + sentinel (device)
     int32_t n_my, tiles;
     int32_t grid;                    // CTAs of the launch (one per SM at most)
+    int32_t interleave;              // 1: super-tiles dealt out round-robin (one large layer); 0: contiguous runs
     LayerState* state;               // [L]
     uint32_t* hist1;                 // [L][kBins1]
     uint32_t* hist2;                 // [L][kBins2]

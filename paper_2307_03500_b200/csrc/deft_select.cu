@@ -56,7 +56,9 @@ constexpr int kSmMiscBytes = 1024;
 constexpr int kSmTf = kSmMisc + kSmMiscBytes;       // tile_first of the rank's first layers (start-up search)
 constexpr int kTfCache = 1024;
 constexpr int kSmTfBytes = (kTfCache + 1) * 4 + 12;
-constexpr int kSmemBytes = kSmTf + kSmTfBytes;
+constexpr int kSmSuper = (kSmTf + kSmTfBytes + 15) / 16 * 16;   // interleaved split: prefix at each own super-tile
+constexpr int kSmSuperBytes = (kMaxLocalTiles / kSuper) * 8;
+constexpr int kSmemBytes = kSmSuper + kSmSuperBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 enum MiscOff : int {   // word offsets inside the misc area
@@ -301,6 +303,30 @@ __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
     return pos < (uint32_t)kResident ? st.res[pos] : __ldcg(st.spill + (pos - kResident));
 }
 
+// CTA-wide pass over the CTA's staged entries, in no particular order.  The spilled part is
+// read in batches of kSpillBatch loads per thread so that the pass is not bound by one
+// HBM round trip per entry.
+constexpr int kSpillBatch = 8;
+constexpr int kEmitBatch = 4;
+template <typename F>
+__device__ __forceinline__ void for_each_staged(const Stage& st, uint32_t total, F f) {
+    const uint32_t nres = total < (uint32_t)kResident ? total : (uint32_t)kResident;
+    for (uint32_t pos = threadIdx.x; pos < nres; pos += kSelThreads) f(st.res[pos]);
+    if (total <= (uint32_t)kResident) return;
+    const uint32_t nsp = total - kResident;
+    for (uint32_t base = 0; base < nsp; base += kSpillBatch * kSelThreads) {
+        uint2 ent[kSpillBatch];
+#pragma unroll
+        for (int u = 0; u < kSpillBatch; ++u) {
+            const uint32_t i = base + u * kSelThreads + threadIdx.x;
+            ent[u] = i < nsp ? __ldcg(st.spill + i) : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < kSpillBatch; ++u)
+            if (base + u * kSelThreads + threadIdx.x < nsp) f(ent[u]);
+    }
+}
+
 // Bit c of the result: component c of v has key >= thr.
 __device__ __forceinline__ uint32_t keep4(const uint4& v, uint32_t thr) {
     return (key_of(v.x) >= thr ? 1u : 0u) | (key_of(v.y) >= thr ? 2u : 0u) |
@@ -379,9 +405,28 @@ __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, cons
 // ---------------------------------------------------------------------------------
 // work split
 // ---------------------------------------------------------------------------------
-struct CtaRange { int q0, q1, jA, jB; };
+// Two ways to split a rank's tiles over the CTAs.
+//   contiguous:  CTA b owns tiles [q0, q1); local tile lq is tile q0 + lq.
+//   interleaved: (one large layer only) the tiles are cut into super-tiles of kSuper tiles and
+//                CTA b owns super-tiles b, b + G, b + 2G, ...; local tile lq is tile kSuper *
+//                (b + (lq / kSuper) * G) + lq % kSuper.  Entries above the threshold cluster
+//                wherever the vector is large; this split gives every CTA a sample of the whole
+//                vector and hence an equal share of them.
+struct CtaRange {
+    int q0, q1, jA, jB;
+    int nloc;      // local tiles (interleaved: the last super-tile may run past p.tiles)
+    int il;        // interleaved
+    int nsuper;    // interleaved: super-tiles of the rank
+};
 
 __device__ __forceinline__ int cta_q0(const SelParams& p, int b) { return (int)((int64_t)p.tiles * b / gridDim.x); }
+
+// Tile id of local tile lq, or -1 where an interleaved CTA's last super-tile runs past the end.
+__device__ __forceinline__ int local_tile(const SelParams& p, const CtaRange& r, int lq) {
+    if (!r.il) return r.q0 + lq;
+    const int q = kSuper * ((int)blockIdx.x + (lq / kSuper) * (int)gridDim.x) + lq % kSuper;
+    return q < p.tiles ? q : -1;
+}
 
 // Largest j in [0, n-1] with tf[j] <= q (tf in shared memory).
 __device__ __forceinline__ int layer_of_tile_sh(const int* tf, int n, int q) {
@@ -396,12 +441,23 @@ __device__ __forceinline__ int layer_of_tile_sh(const int* tf, int n, int q) {
 // The CTA's tiles and the layers they belong to.  The first kTfCache layers' tile_first are
 // fetched with one coalesced request so that the search does not chase cold global loads.
 __device__ __forceinline__ CtaRange cta_range(const SelParams& p, int* tf_cache) {
+    CtaRange r;
+    r.il = p.interleave;
+    r.nsuper = (p.tiles + kSuper - 1) / kSuper;
+    if (r.il) {   // one streamed layer
+        const int b = blockIdx.x, G = gridDim.x;
+        const int nm = b < r.nsuper ? (r.nsuper - b + G - 1) / G : 0;
+        r.nloc = nm * kSuper;
+        r.q0 = 0; r.q1 = nm ? p.tiles : 0;
+        r.jA = 0; r.jB = nm ? 0 : -1;
+        return r;
+    }
     const int nc = p.n_my < kTfCache ? p.n_my : kTfCache;
     for (int i = threadIdx.x; i <= nc; i += kSelThreads) tf_cache[i] = p.desc[i].tile_first;
     __syncthreads();
-    CtaRange r;
     r.q0 = cta_q0(p, blockIdx.x);
     r.q1 = cta_q0(p, blockIdx.x + 1);
+    r.nloc = r.q1 - r.q0;
     r.jA = 0; r.jB = -1;
     if (r.q0 < r.q1) {
         if (p.n_my <= kTfCache || r.q1 <= tf_cache[nc]) {
@@ -413,6 +469,23 @@ __device__ __forceinline__ CtaRange cta_range(const SelParams& p, int* tf_cache)
         }
     }
     return r;
+}
+
+// Local tiles [a, b) of the CTA that can belong to local layers c0 .. c1 (inclusive).
+__device__ __forceinline__ void local_span(const CtaRange& r, const LayerTable* lt, int c0, int c1, int& a, int& b) {
+    if (r.il) { a = 0; b = r.nloc; return; }
+    a = (r.q0 > lt->tf[c0] ? r.q0 : lt->tf[c0]) - r.q0;
+    b = (r.q1 < lt->tfe[c1] ? r.q1 : lt->tfe[c1]) - r.q0;
+}
+
+// Tiles of local layer c that this CTA owns.
+__device__ __forceinline__ uint32_t own_tiles(const SelParams& p, const CtaRange& r, const LayerTable* lt, int c) {
+    if (r.il) {
+        const int owns_last = (r.nsuper - 1) % (int)gridDim.x == (int)blockIdx.x;
+        return (uint32_t)(r.nloc - (owns_last ? r.nsuper * kSuper - p.tiles : 0));
+    }
+    const int a = r.q0 > lt->tf[c] ? r.q0 : lt->tf[c], b = r.q1 < lt->tfe[c] ? r.q1 : lt->tfe[c];
+    return b > a ? (uint32_t)(b - a) : 0u;
 }
 
 // The CTA whose run of tiles contains tile q.
@@ -470,10 +543,12 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
         for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) hist[i] = 0;
         __syncthreads();
         stamp(p, 8);
-        const int qa = r.q0 > lt->tf[c0] ? r.q0 : lt->tf[c0];
-        const int qb = r.q1 < lt->tfe[c0 + ns - 1] ? r.q1 : lt->tfe[c0 + ns - 1];
+        int la, lb;
+        local_span(r, lt, c0, c0 + ns - 1, la, lb);
         int c = c0;
-        for (int q = qa + warp; q < qb; q += kSelWarps) {
+        for (int lq = la + warp; lq < lb; lq += kSelWarps) {
+            const int q = local_tile(p, r, lq);
+            if (q < 0) continue;
             const int cl = tile_layer(lt, c0 + ns, q, c);
             if (cl < 0) continue;
             const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
@@ -490,8 +565,7 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
         // ticket per layer: the CTA that flushes a layer's last tiles sees the complete histogram
         if ((int)threadIdx.x < ns) {
             const int cl = c0 + threadIdx.x;
-            const int a = r.q0 > lt->tf[cl] ? r.q0 : lt->tf[cl], b = r.q1 < lt->tfe[cl] ? r.q1 : lt->tfe[cl];
-            const uint32_t mine = b > a ? (uint32_t)(b - a) : 0u;
+            const uint32_t mine = own_tiles(p, r, lt, cl);
             __threadfence();
             const uint32_t old = atomicAdd(&p.state[lt->lid[cl]].ticket1, mine);
             misc[kMLast + threadIdx.x] = (old + mine == (uint32_t)(lt->tfe[cl] - lt->tf[cl])) ? 1u : 0u;
@@ -533,16 +607,17 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
         }
         for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) hist2s[i] = 0;
         __syncthreads();
-        const int qa = r.q0 > lt->tf[c0] ? r.q0 : lt->tf[c0];
-        const int qb = r.q1 < lt->tfe[c0 + ns - 1] ? r.q1 : lt->tfe[c0 + ns - 1];
+        int la, lb;
+        local_span(r, lt, c0, c0 + ns - 1, la, lb);
         int c = c0;
-        for (int q = qa + warp; q < qb; q += kSelWarps) {
+        for (int lq = la + warp; lq < lb; lq += kSelWarps) {
+            const int q = local_tile(p, r, lq);
+            if (q < 0) continue;
             const int cl = tile_layer(lt, c0 + ns, q, c);
             if (cl < 0) continue;
             const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-            const uint32_t lq = (uint32_t)(q - r.q0);
             const uint2 fn = filter_tile(p.acc, ts, misc[kMTab + cl - c0], hist2s + (cl - c0) * kBins2, st,
-                                         pack_y(0u, (uint32_t)cl, lq), misc + kMCursor, lane);
+                                         pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor, lane);
             if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
         }
         __syncthreads();
@@ -579,13 +654,12 @@ __device__ __forceinline__ void step_hist3(const SelParams& p, LayerTable* lt, i
         const int ns = nl - c0 < kS2Chunk ? nl - c0 : kS2Chunk;
         for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) h3[i] = 0;
         __syncthreads();
-        for (uint32_t pos = threadIdx.x; pos < total; pos += kSelThreads) {
-            const uint2 ent = stage_get(st, pos);
+        for_each_staged(st, total, [&](const uint2 ent) {
             const int c = (int)y_layer(ent.y);
             const uint32_t key = key_of(ent.x);
             if (c >= c0 && c < c0 + ns && (key >> kShift2) == lt->v0[c])
                 atomicAdd(&h3[(c - c0) * kBins3 + (key & (kBins3 - 1))], 1u);
-        }
+        });
         __syncthreads();
         for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) {
             const uint32_t cnt = h3[i];
@@ -612,17 +686,26 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
             lt->v1[c] = lt->v1[c] - above3;            // need
         }
     }
-    for (int i = threadIdx.x; i < r.q1 - r.q0; i += kSelThreads) tt->ge[i] = 0;
+    for (int i = threadIdx.x; i < r.nloc; i += kSelThreads) tt->ge[i] = 0;
     __syncthreads();
-    for (uint32_t pos = threadIdx.x; pos < total; pos += kSelThreads) {
-        const uint2 ent = stage_get(st, pos);
+    for_each_staged(st, total, [&](const uint2 ent) {
         const uint32_t key = key_of(ent.x), T = lt->v0[y_layer(ent.y)];
         if (key > T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u);
         else if (key == T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u << 16);
-    }
+    });
     __syncthreads();
+    if (r.il) {   // totals per own super-tile, published under the super-tile's id
+        for (int m = threadIdx.x; m < r.nloc / kSuper; m += kSelThreads) {
+            uint32_t gt = 0, eq = 0;
+#pragma unroll
+            for (int i = 0; i < kSuper; ++i) { const uint32_t v = tt->ge[m * kSuper + i]; gt += v & 0xffffu; eq += v >> 16; }
+            p.runge[blockIdx.x + m * gridDim.x] = make_uint2(gt, eq);
+        }
+        return;
+    }
     for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of its tiles here
-        const int a = (r.q0 > lt->tf[c] ? r.q0 : lt->tf[c]) - r.q0, b = (r.q1 < lt->tfe[c] ? r.q1 : lt->tfe[c]) - r.q0;
+        int a, b;
+        local_span(r, lt, c, c, a, b);
         uint32_t gt = 0, eq = 0;
         for (int i = a + lane; i < b; i += 32) { const uint32_t v = tt->ge[i]; gt += v & 0xffffu; eq += v >> 16; }
         gt = __reduce_add_sync(0xffffffffu, gt);
@@ -653,14 +736,88 @@ __device__ __forceinline__ void emit_batch(const SelParams& p, int64_t out_off, 
 }
 
 // ---------------------------------------------------------------------------------
-// step S4: totals of the CTAs before this one, scan of the own tiles, ordered write
+// step S4: totals of the tiles before this CTA's, scan of the own tiles, ordered write
 // ---------------------------------------------------------------------------------
+// One batch of local tiles [t0, tend): pref[lq - t0] = entries above / equal to T that precede
+// tile lq in its layer.  One warp per tile writes the tile's selected entries.
+__device__ __forceinline__ void emit_tiles(const SelParams& p, const CtaRange& r, const TileTable* tt,
+                                           const Stage& st, const uint2* pref, int t0, int tend, int64_t start,
+                                           int tf, int64_t out_off, uint32_t T, uint32_t need) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int lq = t0 + warp; lq < tend; lq += kSelWarps) {
+        const int q = local_tile(p, r, lq);
+        if (q < 0) continue;
+        const uint32_t n = tt->n[lq];
+        if (n == 0) continue;
+        const uint32_t first = tt->first[lq];
+        const int64_t lo = (start / kTile + (q - tf)) * kTile;
+        uint32_t gt_before = pref[lq - t0].x, eq_before = pref[lq - t0].y;
+        for (uint32_t e0 = 0; e0 < n; e0 += 32 * kEmitBatch) {   // loads of a round are in flight together
+            uint2 ent[kEmitBatch];
+#pragma unroll
+            for (int u = 0; u < kEmitBatch; ++u) {
+                const uint32_t e = e0 + u * 32 + lane;
+                ent[u] = e < n ? stage_get(st, first + e) : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < kEmitBatch; ++u) {
+                if (e0 + u * 32 < n)   // uniform over the warp
+                    emit_batch(p, out_off, lo, e0 + u * 32 + lane < n, ent[u].x, (int64_t)y_off(ent[u].y), T, need,
+                               gt_before, eq_before, lane);
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
                                           const TileTable* tt, const Stage& st, unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint2* pref = reinterpret_cast<uint2*>(smem + kSmPref);
     uint32_t* scratch = misc + kMScratch;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (r.il) {
+        if (nl == 0) return;
+        // Prefix at each own super-tile b + mG: the totals of all super-tiles are summed in
+        // windows [b + (m-1)G, b + mG) (window 0 = [0, b)), one warp per window, then scanned.
+        uint2* sbase = reinterpret_cast<uint2*>(smem + kSmSuper);
+        const int nm = r.nloc / kSuper, G = gridDim.x, b = blockIdx.x;
+        for (int m = warp; m < nm; m += kSelWarps) {
+            const int hi = b + m * G, lo = m ? hi - G : 0;
+            uint32_t gt = 0, eq = 0;
+            for (int s = lo + lane; s < hi; s += 32) { const uint2 v = __ldcg(p.runge + s); gt += v.x; eq += v.y; }
+            gt = __reduce_add_sync(0xffffffffu, gt);
+            eq = __reduce_add_sync(0xffffffffu, eq);
+            if (lane == 0) sbase[m] = make_uint2(gt, eq);
+        }
+        __syncthreads();
+        {
+            const uint2 w = (int)threadIdx.x < nm ? sbase[threadIdx.x] : make_uint2(0u, 0u);
+            uint32_t tg, te;
+            const uint32_t e_gt = block_excl_scan(w.x, scratch, tg);
+            const uint32_t e_eq = block_excl_scan(w.y, scratch, te);
+            if ((int)threadIdx.x < nm) sbase[threadIdx.x] = make_uint2(e_gt + w.x, e_eq + w.y);
+        }
+        __syncthreads();
+        const uint32_t T = lt->v0[0], need = lt->v1[0];
+        for (int t0 = 0; t0 < r.nloc; t0 += kSelThreads) {
+            const int i = t0 + (int)threadIdx.x;
+            const uint32_t v = i < r.nloc ? tt->ge[i] : 0u;   // counts <= kTile each: 16 of them fit 16 bits
+            uint32_t incl = v;
+#pragma unroll
+            for (int o = 1; o < kSuper; o <<= 1) {
+                const uint32_t x = __shfl_up_sync(0xffffffffu, incl, o, kSuper);
+                if ((lane & (kSuper - 1)) >= o) incl += x;
+            }
+            const uint32_t ex = incl - v;
+            const uint2 sb = i < r.nloc ? sbase[i / kSuper] : make_uint2(0u, 0u);
+            pref[threadIdx.x] = make_uint2(sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
+            __syncthreads();
+            const int tend = t0 + kSelThreads < r.nloc ? t0 + kSelThreads : r.nloc;
+            emit_tiles(p, r, tt, st, pref, t0, tend, lt->start[0], lt->tf[0], lt->out_off[0], T, need);
+            __syncthreads();   // pref is rewritten by the next batch
+        }
+        return;
+    }
     for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of earlier CTAs
         const int j = lt->j[c];
         uint32_t gt = 0, eq = 0;
@@ -677,10 +834,9 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
     }
     __syncthreads();
     for (int c = 0; c < nl; ++c) {
-        const int ta = (r.q0 > lt->tf[c] ? r.q0 : lt->tf[c]) - r.q0, tb = (r.q1 < lt->tfe[c] ? r.q1 : lt->tfe[c]) - r.q0;
+        int ta, tb;
+        local_span(r, lt, c, c, ta, tb);
         const uint32_t T = lt->v0[c], need = lt->v1[c];
-        const int64_t start = lt->start[c], out_off = lt->out_off[c];
-        const int tf = lt->tf[c];
         uint32_t base_gt = lt->base_gt[c], base_eq = lt->base_eq[c];
         for (int t0 = ta; t0 < tb; t0 += kSelThreads) {   // batches of kSelThreads tiles
             const int i = t0 + (int)threadIdx.x;
@@ -691,20 +847,7 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             pref[threadIdx.x] = make_uint2(base_gt + e_gt, base_eq + e_eq);
             __syncthreads();
             const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
-            for (int lq = t0 + warp; lq < tend; lq += kSelWarps) {
-                const uint32_t n = tt->n[lq];
-                if (n == 0) continue;
-                const uint32_t first = tt->first[lq];
-                const int64_t lo = (start / kTile + (r.q0 + lq - tf)) * kTile;
-                uint32_t gt_before = pref[lq - t0].x, eq_before = pref[lq - t0].y;
-                for (uint32_t e0 = 0; e0 < n; e0 += 32) {
-                    const uint32_t e = e0 + lane;
-                    const bool valid = e < n;
-                    uint2 ent = make_uint2(0u, 0u);
-                    if (valid) ent = stage_get(st, first + e);
-                    emit_batch(p, out_off, lo, valid, ent.x, (int64_t)y_off(ent.y), T, need, gt_before, eq_before, lane);
-                }
-            }
+            emit_tiles(p, r, tt, st, pref, t0, tend, lt->start[c], lt->tf[c], lt->out_off[c], T, need);
             base_gt += tot_gt;
             base_eq += tot_eq;
             __syncthreads();   // pref is rewritten by the next batch
@@ -823,7 +966,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     Stage st;
     st.res = reinterpret_cast<uint2*>(smem + kSmMain);
     st.spill = p.staging;
-    if (r.q0 < r.q1) {
+    if (r.il) {
+        // the CTA's part of the staging area: one slot per element of the super-tiles of the CTAs before it
+        const int64_t before = (int64_t)blockIdx.x * (r.nsuper / (int)gridDim.x) +
+                               min((int)blockIdx.x, r.nsuper % (int)gridDim.x);
+        st.spill = p.staging + p.desc[0].elem_off + before * (kSuper * kTile);
+    } else if (r.q0 < r.q1) {
         // the CTA's part of the staging area starts where its first tile's elements would go
         const TileSpan ts = tile_span(p.desc[r.jA].start, p.desc[r.jA].end, p.desc[r.jA].tile_first, r.q0);
         st.spill = p.staging + p.desc[r.jA].elem_off + (ts.lo + ts.s - p.desc[r.jA].start);
@@ -832,7 +980,16 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     step_hist1(p, r, lt, nl, smem);
     stamp(p, 1);
     grid.sync();
+    unsigned long long tb0 = 0;
+    if (p.timing && threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tb0));
     step_filter(p, r, lt, nl, tt, st, smem);
+    if (p.timing && threadIdx.x == 0) {
+        unsigned long long tb1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tb1));
+        p.timing[16 + blockIdx.x] = tb1 - tb0;
+        p.timing[16 + 160 + blockIdx.x] = misc[kMCursor];
+        p.timing[16 + 320 + blockIdx.x] = (unsigned long long)nl;
+    }
     stamp(p, 2);
     grid.sync();
     step_hist3(p, lt, nl, st, smem);

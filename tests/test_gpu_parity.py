@@ -245,6 +245,29 @@ def test_topk_baseline(deft, n, k):
     assert val_d.cpu().numpy().tobytes() == want_val.tobytes()
 
 
+@pytest.mark.parametrize("kind,k", [("clustered", 21_000), ("clustered", 2_100_000), ("few_values", 300_001)])
+def test_topk_single_large_layer_round_robin_split(deft, kind, k):
+    """One layer large enough that the kernel deals its tiles out to the CTAs round-robin
+    (several thousand tiles per CTA-round, a ragged last super-tile, an unaligned start)."""
+    n = 21_000_003
+    if kind == "clustered":     # the large entries sit in a few narrow regions
+        x = W.adversarial_vector("gauss", n + 3, seed=5)
+        x[1_000_000:1_300_000] *= np.float32(50.0)
+        x[-70_000:] *= np.float32(80.0)
+    else:                       # eight distinct magnitudes: the threshold value repeats millions of times
+        x = W.adversarial_vector("few_values", n + 3, seed=6)
+    acc_d = _dev(x)
+    start = np.array([3, n + 3], dtype=np.int64)      # layer starts 12 bytes into the buffer
+    ws = deft.alloc_workspace(n, 1)
+    val_d = torch.empty(k, dtype=torch.float32, device="cuda")
+    idx_d = torch.empty(k, dtype=torch.int64, device="cuda")
+    deft.deft_select(acc_d, start, np.array([k], dtype=np.int64), np.array([0], dtype=np.int32), val_d, idx_d, ws)
+    torch.cuda.synchronize()
+    want_val, want_idx = oracle.select_layer(x, 3, n + 3, k)
+    assert np.array_equal(idx_d.cpu().numpy(), want_idx)
+    assert val_d.cpu().numpy().tobytes() == want_val.tobytes()
+
+
 def test_select_is_bit_deterministic_run_to_run(deft):
     w = W.scaled_down(W.gpt2_medium(4, 0.01), 16)
     x = w.gradient(0)

@@ -142,21 +142,47 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.grid = want < sms ? want : sms;
     // limits of one CTA's share: tiles, and streamed (non-direct) layers
     const LayerDesc* hd = plan_descs(plan_h, hdr->N) + R.desc_first;
+    p.weighted = 0;
     p.interleave = (R.n_my == 1 && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) ? 1 : 0;
     if (p.interleave) {
         const int nsuper = (R.tiles + kSuper - 1) / kSuper;
         if ((int64_t)((nsuper + p.grid - 1) / p.grid) * kSuper > kMaxLocalTiles) return DEFT_ERR_INVALID_ARG;
         return launch_select(p, stream);
     }
-    int j = 0;
-    for (int b = 0; b < p.grid; ++b) {
-        const int q0 = (int)((int64_t)R.tiles * b / p.grid), q1 = (int)((int64_t)R.tiles * (b + 1) / p.grid);
-        if (q1 - q0 > kMaxLocalTiles) return DEFT_ERR_INVALID_ARG;
-        while (j + 1 < R.n_my && hd[j + 1].tile_first <= q0) ++j;
-        int streamed = 0;
-        for (int jj = j; jj < R.n_my && hd[jj].tile_first < q1; ++jj)
-            streamed += (hd[jj].end - hd[jj].start > kDirectElems);
-        if (streamed > kMaxLocalLayers) return DEFT_ERR_INVALID_ARG;
+    // q0[b] = first tile of CTA b, b = 0..grid
+    auto within_limits = [&](const std::vector<int>& q0) {
+        int j = 0;
+        for (int b = 0; b < p.grid; ++b) {
+            if (q0[b + 1] - q0[b] > kMaxLocalTiles) return false;
+            while (j + 1 < R.n_my && hd[j + 1].tile_first <= q0[b]) ++j;
+            int streamed = 0;
+            for (int jj = j; jj < R.n_my && hd[jj].tile_first < q0[b + 1]; ++jj)
+                streamed += (hd[jj].end - hd[jj].start > kDirectElems);
+            if (streamed > kMaxLocalLayers) return false;
+        }
+        return true;
+    };
+    std::vector<int> q0((size_t)p.grid + 1);
+    for (int b = 0; b <= p.grid; ++b) q0[b] = (int)((int64_t)R.tiles * b / p.grid);
+    if (!within_limits(q0)) return DEFT_ERR_INVALID_ARG;
+    if (R.n_my > 1 && R.n_my <= kMaxWeightedLayers && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) {
+        const int n = R.n_my;
+        std::vector<uint32_t> Wp((size_t)n + 1), wt((size_t)n);
+        std::vector<int> tf((size_t)n + 1);
+        uint64_t acc = 0;
+        for (int j = 0; j < n; ++j) {
+            wt[j] = tile_weight(hd[j].k, hd[j].end - hd[j].start);
+            tf[j] = hd[j].tile_first;
+            Wp[j] = (uint32_t)acc;
+            acc += (uint64_t)wt[j] * (uint64_t)(hd[j + 1].tile_first - hd[j].tile_first);
+            if (acc > 0xffffffffull) break;
+        }
+        if (acc > 0 && acc <= 0xffffffffull) {
+            Wp[n] = (uint32_t)acc;
+            tf[n] = R.tiles;
+            for (int b = 0; b <= p.grid; ++b) q0[b] = weighted_boundary(Wp.data(), wt.data(), tf.data(), n, R.tiles, b, p.grid);
+            if (within_limits(q0)) p.weighted = 1;
+        }
     }
     return launch_select(p, stream);
 }

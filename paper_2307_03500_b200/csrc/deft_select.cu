@@ -58,7 +58,9 @@ constexpr int kTfCache = 1024;
 constexpr int kSmTfBytes = (kTfCache + 1) * 4 + 12;
 constexpr int kSmSuper = (kSmTf + kSmTfBytes + 15) / 16 * 16;   // interleaved split: prefix at each own super-tile
 constexpr int kSmSuperBytes = (kMaxLocalTiles / kSuper) * 8;
-constexpr int kSmemBytes = kSmSuper + kSmSuperBytes;
+constexpr int kSmWBase = kSmSuper + kSmSuperBytes;   // staging pass: 16 words per warp
+constexpr int kSmWBaseBytes = kSelWarps * 16 * 4;
+constexpr int kSmemBytes = kSmWBase + kSmWBaseBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 enum MiscOff : int {   // word offsets inside the misc area
@@ -252,17 +254,30 @@ struct TileRegs {
 };
 static_assert(kTile == 16 * 32 * 4, "16 vector loads per lane");
 
+// Bit c of the result: offset o + c lies in [s, e).
+__device__ __forceinline__ uint32_t valid4(int o, int s, int e) {
+    const int lo = s - o > 0 ? s - o : 0, hi = e - o < 4 ? e - o : 4;
+    return hi > lo ? ((1u << hi) - 1u) & ~((1u << lo) - 1u) : 0u;
+}
+
+// vm: bit (4 * (i % 8) + c) of vm[i / 8] = component c of load i belongs to the layer.
+// Components outside the layer come back as +0.
 __device__ __forceinline__ void load_tile(const float* __restrict__ acc, const TileSpan& ts, int lane,
-                                          TileRegs& t) {
+                                          TileRegs& t, uint32_t (&vm)[2]) {
     const uint4* p4 = reinterpret_cast<const uint4*>(acc + ts.lo) + lane;
     if (ts.s == 0 && ts.e == kTile) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) t.v[i] = __ldg(p4 + i * 32);
+        vm[0] = vm[1] = 0xffffffffu;
     } else {
+        vm[0] = vm[1] = 0u;
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const int o = (i * 32 + lane) * 4;
-            t.v[i] = (o + 4 > ts.s && o < ts.e) ? __ldg(p4 + i * 32) : make_uint4(0u, 0u, 0u, 0u);
+            const uint32_t m = valid4((i * 32 + lane) * 4, ts.s, ts.e);
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (m) v = __ldg(p4 + i * 32);
+            t.v[i] = make_uint4(m & 1u ? v.x : 0u, m & 2u ? v.y : 0u, m & 4u ? v.z : 0u, m & 8u ? v.w : 0u);
+            vm[i >> 3] |= m << (4 * (i & 7));
         }
     }
 }
@@ -270,25 +285,17 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ acc, const T
 __device__ __forceinline__ void hist_tile(const float* __restrict__ acc, const TileSpan& ts,
                                           uint32_t* h, int lane) {
     TileRegs t;
-    load_tile(acc, ts, lane, t);
-    if (ts.s == 0 && ts.e == kTile) {
+    uint32_t vm[2];
+    load_tile(acc, ts, lane, t, vm);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            atomicAdd(&h[key_of(t.v[i].x) >> kShift1], 1u);
-            atomicAdd(&h[key_of(t.v[i].y) >> kShift1], 1u);
-            atomicAdd(&h[key_of(t.v[i].z) >> kShift1], 1u);
-            atomicAdd(&h[key_of(t.v[i].w) >> kShift1], 1u);
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int o = (i * 32 + lane) * 4;
-            const uint32_t w[4] = {t.v[i].x, t.v[i].y, t.v[i].z, t.v[i].w};
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (o + c >= ts.s && o + c < ts.e) atomicAdd(&h[key_of(w[c]) >> kShift1], 1u);
-        }
+    for (int i = 0; i < 16; ++i) {
+        atomicAdd(&h[key_of(t.v[i].x) >> kShift1], 1u);
+        atomicAdd(&h[key_of(t.v[i].y) >> kShift1], 1u);
+        atomicAdd(&h[key_of(t.v[i].z) >> kShift1], 1u);
+        atomicAdd(&h[key_of(t.v[i].w) >> kShift1], 1u);
     }
+    // the components outside the layer were counted as zeros
+    if (lane == 0 && ts.e - ts.s != kTile) atomicSub(&h[0], (uint32_t)(kTile - (ts.e - ts.s)));
 }
 
 // Where a CTA's staged entry number `pos` lives.
@@ -333,73 +340,83 @@ __device__ __forceinline__ uint32_t keep4(const uint4& v, uint32_t thr) {
            (key_of(v.z) >= thr ? 4u : 0u) | (key_of(v.w) >= thr ? 8u : 0u);
 }
 
-// Bit c of the result: offset o + c lies in [s, e).
-__device__ __forceinline__ uint32_t valid4(int o, int s, int e) {
-    const int lo = s - o > 0 ? s - o : 0, hi = e - o < 4 ? e - o : 4;
-    return hi > lo ? ((1u << hi) - 1u) & ~((1u << lo) - 1u) : 0u;
+__device__ __forceinline__ uint32_t pick4(uint32_t a, uint32_t b, uint32_t c, uint32_t d, int sel) {
+    const uint32_t ab = (sel & 1) ? b : a, cd = (sel & 1) ? d : c;
+    return (sel & 2) ? cd : ab;
 }
 
-// Moves the tile's entries with bucket >= b1 behind the CTA's cursor, in index order
-// (load, lane, component = ascending offset).  Returns (first entry, entries).
-// The common case (a handful of entries per tile) costs about 3 instructions per element.
+// The rare part of the staging pass, kept out of line and small (the hot loop around it must
+// stay resident in the instruction cache): moves the tile's marked entries behind the CTA's
+// cursor in index order (load, lane, component = ascending offset).  k0 / k1: bit (4 * (i % 8)
+// + c) of word i / 8 marks component c of this lane's load i.  The values are read again from
+// the vector (the tile has just been loaded: they come from L1 / L2).  wbase: 16 words of
+// shared memory private to the warp.  Returns (first entry, entries).
+__device__ __noinline__ uint2 filter_marked(const uint32_t* __restrict__ tile, uint32_t k0, uint32_t k1, uint32_t b1,
+                                            uint32_t* h2, uint2* res, uint2* spill, uint32_t ytag,
+                                            uint32_t* cursor, uint32_t* wbase) {
+    const int lane = threadIdx.x & 31;
+#ifdef DEFT_PROFILE_FILTER
+    const long long pf0 = clock64();
+#endif
+    // per-load counts of this lane, 8 bits each, four loads per word; scanned over the lanes
+    uint32_t excl[4], tot[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t kw = (g < 2 ? k0 : k1) >> (16 * (g & 1));
+        const uint32_t packed = __popc(kw & 0xfu) | (__popc(kw & 0xf0u) << 8) | (__popc(kw & 0xf00u) << 16) |
+                                (__popc(kw & 0xf000u) << 24);
+        const uint32_t incl = warp_incl_scan(packed, lane);
+        tot[g] = __shfl_sync(0xffffffffu, incl, 31);
+        excl[g] = incl - packed;
+    }
+    // lane i < 16 owns load i: where the load's entries start
+    const uint32_t mytot = lane < 16 ? (pick4(tot[0], tot[1], tot[2], tot[3], lane >> 2) >> (8 * (lane & 3))) & 0xffu : 0u;
+    const uint32_t incl = warp_incl_scan(mytot, lane);
+    const uint32_t n = __shfl_sync(0xffffffffu, incl, 31);
+    uint32_t first = 0;
+    if (lane == 0) first = atomicAdd(cursor, n);
+    first = __shfl_sync(0xffffffffu, first, 0);
+    if (lane < 16) wbase[lane] = first + incl - mytot;
+    __syncwarp();
+    const Stage st{res, spill};
+    unsigned long long m = (unsigned long long)k0 | ((unsigned long long)k1 << 32);
+    const unsigned long long all = m;
+    while (m) {
+        const int bit = __ffsll((long long)m) - 1;
+        m &= m - 1;
+        const int i = bit >> 2, c = bit & 3;
+        const uint32_t before_lanes = (pick4(excl[0], excl[1], excl[2], excl[3], i >> 2) >> (8 * (i & 3))) & 0xffu;
+        const uint32_t before_mine = __popc((uint32_t)(all >> (4 * i)) & ((1u << c) - 1u));
+        const uint32_t off = (uint32_t)((i * 32 + lane) * 4 + c);
+        const uint32_t bits = __ldg(tile + off);
+        const uint32_t key = key_of(bits);
+        if ((key >> kShift1) == b1) atomicAdd(&h2[(key >> kShift2) & (kBins2 - 1)], 1u);
+        stage_put(st, wbase[i] + before_lanes + before_mine, make_uint2(bits, ytag | off));
+    }
+    __syncwarp();   // wbase is rewritten by the warp's next tile
+#ifdef DEFT_PROFILE_FILTER
+    if (lane == 0) { atomicAdd(cursor + 1, 1u); atomicAdd(cursor + 2, (uint32_t)(clock64() - pf0)); }
+#endif
+    return make_uint2(first, n);
+}
+
+// Staging pass over one tile: marks the entries with bucket >= b1; tiles without any cost a
+// compare per element.
 __device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t b1,
                                              uint32_t* h2, const Stage& st, uint32_t ytag, uint32_t* cursor,
-                                             int lane) {
+                                             uint32_t* wbase, int lane) {
     TileRegs t;
-    load_tile(acc, ts, lane, t);
+    uint32_t vm[2];
+    load_tile(acc, ts, lane, t, vm);
     const uint32_t thr = b1 << kShift1;          // key >= thr  <=>  bucket >= b1
     uint32_t keep[2] = {0u, 0u};                 // bit (4*(i%8) + c) of keep[i/8]
 #pragma unroll
     for (int i = 0; i < 16; ++i) keep[i >> 3] |= keep4(t.v[i], thr) << (4 * (i & 7));
-    if (!(ts.s == 0 && ts.e == kTile)) {
-        uint32_t vm[2] = {0u, 0u};
-#pragma unroll
-        for (int i = 0; i < 16; ++i) vm[i >> 3] |= valid4((i * 32 + lane) * 4, ts.s, ts.e) << (4 * (i & 7));
-        keep[0] &= vm[0];
-        keep[1] &= vm[1];
-    }
+    keep[0] &= vm[0];
+    keep[1] &= vm[1];
     if (!__any_sync(0xffffffffu, (keep[0] | keep[1]) != 0)) return make_uint2(0u, 0u);
-    // per-load counts, 8 bits each (a warp holds <= 128 per load), four loads per word
-    uint32_t packed[4];
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        const uint32_t kw = keep[g >> 1] >> (16 * (g & 1));
-        packed[g] = __popc(kw & 0xfu) | (__popc(kw & 0xf0u) << 8) | (__popc(kw & 0xf00u) << 16) |
-                    (__popc(kw & 0xf000u) << 24);
-    }
-    uint32_t excl[4], tot[4];
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        const uint32_t incl = warp_incl_scan(packed[g], lane);
-        tot[g] = __shfl_sync(0xffffffffu, incl, 31);
-        excl[g] = incl - packed[g];
-    }
-    uint32_t n = 0;
-#pragma unroll
-    for (int g = 0; g < 4; ++g) n += (tot[g] & 0xff) + ((tot[g] >> 8) & 0xff) + ((tot[g] >> 16) & 0xff) + (tot[g] >> 24);
-    uint32_t first = 0;
-    if (lane == 0) first = atomicAdd(cursor, n);
-    first = __shfl_sync(0xffffffffu, first, 0);
-    uint32_t load_base = first;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const uint32_t tot_i = (tot[i >> 2] >> (8 * (i & 3))) & 0xff;
-        const uint32_t k4 = (keep[i >> 3] >> (4 * (i & 7))) & 0xfu;
-        if (k4) {
-            const uint32_t w[4] = {t.v[i].x, t.v[i].y, t.v[i].z, t.v[i].w};
-            uint32_t pos = load_base + ((excl[i >> 2] >> (8 * (i & 3))) & 0xff);
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (k4 & (1u << c)) {
-                    const uint32_t key = key_of(w[c]);
-                    if ((key >> kShift1) == b1) atomicAdd(&h2[(key >> kShift2) & (kBins2 - 1)], 1u);
-                    stage_put(st, pos, make_uint2(w[c], ytag | (uint32_t)((i * 32 + lane) * 4 + c)));
-                    ++pos;
-                }
-        }
-        load_base += tot_i;
-    }
-    return make_uint2(first, n);
+    return filter_marked(reinterpret_cast<const uint32_t*>(acc + ts.lo), keep[0], keep[1], b1, h2, st.res, st.spill,
+                         ytag, cursor, wbase);
 }
 
 // ---------------------------------------------------------------------------------
@@ -417,6 +434,7 @@ struct CtaRange {
     int nloc;      // local tiles (interleaved: the last super-tile may run past p.tiles)
     int il;        // interleaved
     int nsuper;    // interleaved: super-tiles of the rank
+    const int* q0tab;   // cost-weighted split: first tile of every CTA (gridDim.x + 1 entries); else NULL
 };
 
 __device__ __forceinline__ int cta_q0(const SelParams& p, int b) { return (int)((int64_t)p.tiles * b / gridDim.x); }
@@ -443,6 +461,7 @@ __device__ __forceinline__ int layer_of_tile_sh(const int* tf, int n, int q) {
 __device__ __forceinline__ CtaRange cta_range(const SelParams& p, int* tf_cache) {
     CtaRange r;
     r.il = p.interleave;
+    r.q0tab = nullptr;
     r.nsuper = (p.tiles + kSuper - 1) / kSuper;
     if (r.il) {   // one streamed layer
         const int b = blockIdx.x, G = gridDim.x;
@@ -471,6 +490,67 @@ __device__ __forceinline__ CtaRange cta_range(const SelParams& p, int* tf_cache)
     return r;
 }
 
+// First tile of CTA b under the split in force.
+__device__ __forceinline__ int split_q0(const SelParams& p, const CtaRange& r, int b) {
+    return r.q0tab ? r.q0tab[b] : cta_q0(p, b);
+}
+
+// The CTA whose run of tiles contains tile q.
+__device__ __forceinline__ int split_cta_of_tile(const SelParams& p, const CtaRange& r, int q) {
+    if (!r.q0tab) return (int)((((int64_t)q + 1) * gridDim.x + p.tiles - 1) / p.tiles) - 1;
+    int lo = 0, hi = (int)gridDim.x - 1;          // largest b with q0tab[b] <= q
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (r.q0tab[mid] <= q) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// The cost-weighted split (see tile_weight): every CTA computes the same table of boundaries
+// with integer arithmetic.  `work` = at least 3 * (n_my + 1) words of shared memory, free at
+// the time of the call; q0tab = gridDim.x + 1 words that stay.
+__device__ __forceinline__ CtaRange weighted_range(const SelParams& p, uint32_t* work, int* q0tab, uint32_t* scratch) {
+    const int n = p.n_my;
+    uint32_t* Wp = work;                 // n + 1
+    uint32_t* w = work + (n + 1);        // n
+    int* tf = reinterpret_cast<int*>(work + 2 * (n + 1));   // n + 1
+    uint32_t carry = 0;
+    for (int j0 = 0; j0 < n; j0 += kSelThreads) {
+        const int j = j0 + (int)threadIdx.x;
+        uint32_t cost = 0;
+        if (j < n) {
+            const uint32_t wj = tile_weight(p.desc[j].k, p.desc[j].end - p.desc[j].start);
+            const int t0 = p.desc[j].tile_first;
+            w[j] = wj;
+            tf[j] = t0;
+            cost = wj * (uint32_t)(p.desc[j + 1].tile_first - t0);
+        }
+        uint32_t tot;
+        const uint32_t ex = block_excl_scan(cost, scratch, tot);
+        if (j < n) Wp[j] = carry + ex;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) { Wp[n] = carry; tf[n] = p.tiles; }
+    __syncthreads();
+    for (int b = threadIdx.x; b <= (int)gridDim.x; b += kSelThreads)
+        q0tab[b] = weighted_boundary(Wp, w, tf, n, p.tiles, b, (int)gridDim.x);
+    __syncthreads();
+    CtaRange r;
+    r.il = 0;
+    r.nsuper = 0;
+    r.q0tab = q0tab;
+    r.q0 = q0tab[blockIdx.x];
+    r.q1 = q0tab[blockIdx.x + 1];
+    r.nloc = r.q1 - r.q0;
+    r.jA = 0; r.jB = -1;
+    if (r.q0 < r.q1) {
+        r.jA = layer_of_tile_sh(tf, n, r.q0);
+        r.jB = layer_of_tile_sh(tf, n, r.q1 - 1);
+    }
+    __syncthreads();   // `work` is free again
+    return r;
+}
+
 // Local tiles [a, b) of the CTA that can belong to local layers c0 .. c1 (inclusive).
 __device__ __forceinline__ void local_span(const CtaRange& r, const LayerTable* lt, int c0, int c1, int& a, int& b) {
     if (r.il) { a = 0; b = r.nloc; return; }
@@ -486,11 +566,6 @@ __device__ __forceinline__ uint32_t own_tiles(const SelParams& p, const CtaRange
     }
     const int a = r.q0 > lt->tf[c] ? r.q0 : lt->tf[c], b = r.q1 < lt->tfe[c] ? r.q1 : lt->tfe[c];
     return b > a ? (uint32_t)(b - a) : 0u;
-}
-
-// The CTA whose run of tiles contains tile q.
-__device__ __forceinline__ int cta_of_tile(const SelParams& p, int q) {
-    return (int)((((int64_t)q + 1) * gridDim.x + p.tiles - 1) / p.tiles) - 1;
 }
 
 __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
@@ -597,7 +672,7 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
     uint32_t* hist2s = reinterpret_cast<uint32_t*>(smem + kSmAux);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) misc[kMCursor] = 0;
+    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMCursor + 1] = 0; misc[kMCursor + 2] = 0; }   // +1, +2: profiling build
     for (int c0 = 0; c0 < nl; c0 += kBSlots) {
         const int ns = nl - c0 < kBSlots ? nl - c0 : kBSlots;
         if ((int)threadIdx.x < ns) {
@@ -617,7 +692,8 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
             if (cl < 0) continue;
             const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
             const uint2 fn = filter_tile(p.acc, ts, misc[kMTab + cl - c0], hist2s + (cl - c0) * kBins2, st,
-                                         pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor, lane);
+                                         pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
+                                         reinterpret_cast<uint32_t*>(smem + kSmWBase) + 16 * warp, lane);
             if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
         }
         __syncthreads();
@@ -821,8 +897,8 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
     for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of earlier CTAs
         const int j = lt->j[c];
         uint32_t gt = 0, eq = 0;
-        for (int b = cta_of_tile(p, lt->tf[c]) + lane; b < (int)blockIdx.x; b += 32) {
-            if (cta_q0(p, b) < cta_q0(p, b + 1)) {
+        for (int b = split_cta_of_tile(p, r, lt->tf[c]) + lane; b < (int)blockIdx.x; b += 32) {
+            if (split_q0(p, r, b) < split_q0(p, r, b + 1)) {
                 const uint2 v = __ldcg(p.runge + b + j);
                 gt += v.x;
                 eq += v.y;
@@ -946,6 +1022,22 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
 }
 static_assert(kDirectElems < 65536, "packed per-warp counts");
 
+// The CTA's part of the staging area in HBM.
+__device__ __forceinline__ uint2* spill_base(const SelParams& p, const CtaRange& r) {
+    if (r.il) {
+        // one slot per element of the super-tiles of the CTAs before it
+        const int64_t before = (int64_t)blockIdx.x * (r.nsuper / (int)gridDim.x) +
+                               min((int)blockIdx.x, r.nsuper % (int)gridDim.x);
+        return p.staging + p.desc[0].elem_off + before * (kSuper * kTile);
+    }
+    if (r.q0 < r.q1) {
+        // it starts where the CTA's first tile's elements would go
+        const TileSpan ts = tile_span(p.desc[r.jA].start, p.desc[r.jA].end, p.desc[r.jA].tile_first, r.q0);
+        return p.staging + p.desc[r.jA].elem_off + (ts.lo + ts.s - p.desc[r.jA].start);
+    }
+    return p.staging;
+}
+
 // ---------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------
@@ -961,25 +1053,21 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     LayerTable* lt = reinterpret_cast<LayerTable*>(smem + kSmLayer);
     TileTable* tt = reinterpret_cast<TileTable*>(smem + kSmTile);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
-    const CtaRange r = cta_range(p, reinterpret_cast<int*>(smem + kSmTf));
-    const int nl = build_layer_table(p, r, lt, misc + kMScratch);
+    CtaRange r = cta_range(p, reinterpret_cast<int*>(smem + kSmTf));
+    int nl = build_layer_table(p, r, lt, misc + kMScratch);
     Stage st;
     st.res = reinterpret_cast<uint2*>(smem + kSmMain);
-    st.spill = p.staging;
-    if (r.il) {
-        // the CTA's part of the staging area: one slot per element of the super-tiles of the CTAs before it
-        const int64_t before = (int64_t)blockIdx.x * (r.nsuper / (int)gridDim.x) +
-                               min((int)blockIdx.x, r.nsuper % (int)gridDim.x);
-        st.spill = p.staging + p.desc[0].elem_off + before * (kSuper * kTile);
-    } else if (r.q0 < r.q1) {
-        // the CTA's part of the staging area starts where its first tile's elements would go
-        const TileSpan ts = tile_span(p.desc[r.jA].start, p.desc[r.jA].end, p.desc[r.jA].tile_first, r.q0);
-        st.spill = p.staging + p.desc[r.jA].elem_off + (ts.lo + ts.s - p.desc[r.jA].start);
-    }
+    st.spill = spill_base(p, r);
 
     step_hist1(p, r, lt, nl, smem);
     stamp(p, 1);
     grid.sync();
+    if (p.weighted) {   // from here on: contiguous runs of equal estimated cost
+        r = weighted_range(p, reinterpret_cast<uint32_t*>(smem + kSmMain), reinterpret_cast<int*>(smem + kSmTf),
+                           misc + kMScratch);
+        nl = build_layer_table(p, r, lt, misc + kMScratch);
+        st.spill = spill_base(p, r);
+    }
     unsigned long long tb0 = 0;
     if (p.timing && threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tb0));
     step_filter(p, r, lt, nl, tt, st, smem);
@@ -988,7 +1076,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tb1));
         p.timing[16 + blockIdx.x] = tb1 - tb0;
         p.timing[16 + 160 + blockIdx.x] = misc[kMCursor];
-        p.timing[16 + 320 + blockIdx.x] = (unsigned long long)nl;
+        p.timing[16 + 320 + blockIdx.x] = (unsigned long long)nl | ((unsigned long long)r.nloc << 16) |
+                                          ((unsigned long long)misc[kMCursor + 1] << 32);
+        p.timing[16 + 480 + blockIdx.x] = misc[kMCursor + 2];
     }
     stamp(p, 2);
     grid.sync();

@@ -268,6 +268,24 @@ def test_topk_single_large_layer_round_robin_split(deft, kind, k):
     assert val_d.cpu().numpy().tobytes() == want_val.tobytes()
 
 
+def test_large_multi_layer_rank_cost_weighted_split(deft):
+    """A rank large enough (> 64 tiles per CTA) that the kernel re-deals its tiles by estimated
+    cost after the first read: layers whose density of selected entries differs by five orders
+    of magnitude, small and tiny layers between large ones, layers skipped by the rank."""
+    sizes = [5_000_000, 3_000_001, 20_000, 1_000, 8_000_005, 1_500_000, 6_000_000, 17, 2_500_000]
+    start = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    x = W.adversarial_vector("gauss", int(start[-1]), seed=12)
+    x[start[4]:start[4] + 2_000_000] *= np.float32(30.0)          # the large entries of layer 4 sit at its head
+    x[start[6]:start[7]] = W.adversarial_vector("few_values", sizes[6], seed=13)
+    k_l = np.array([5, 900_000, 100, 10, 8_000, 1, 600_000, 17, 2_499_999], dtype=np.int64)
+    my = np.array([0, 1, 2, 3, 4, 6, 7, 8], dtype=np.int32)       # layer 5 belongs to another rank
+    acc_d = _dev(x)
+    val, idx = _gpu_select(deft, acc_d, start, k_l, my)
+    want_val, want_idx = oracle.select_rank(x, start, k_l, my)
+    assert np.array_equal(idx, want_idx)
+    assert val.tobytes() == want_val.tobytes()
+
+
 def test_select_is_bit_deterministic_run_to_run(deft):
     w = W.scaled_down(W.gpt2_medium(4, 0.01), 16)
     x = w.gradient(0)

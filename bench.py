@@ -281,18 +281,11 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     launches = {"n": 0}
-    # per-rank event triples for every timed step, created (and their handles forced) before timing
-    mark_pool = []
-    if args.mode == "step":
-        for _ in range(args.steps):
-            tri = [(ev(), ev(), ev()) for _ in range(N)]
-            for t3 in tri:
-                for x in t3:
-                    x.record(stream)
-            mark_pool.append(tri)
 
-    def one_step(it, rec=None, grad=g):
-        """The whole path for all N simulated ranks.  rec: optional dict collecting events."""
+    def one_step(it, rec=None, grad=g, marks=None):
+        """The whole path for all N simulated ranks: accumulate + norms, D2H norms, host planner, plan
+        upload, then every rank's selection + residual update — in ONE launch, or, with `marks`
+        (per-rank event triples), one launch per rank for per-worker timings."""
         e0 = ev(); e0.record(stream)
         deft.deft_layer_norms(e, grad, ds.layer_start_d, ds.norms_d, ds.ws)
         e1 = ev(); e1.record(stream)
@@ -301,12 +294,13 @@ def run_ours(args):
         th0 = time.perf_counter()
         plan = ds.plan(ds.norms_h.numpy(), it)
         th1 = time.perf_counter()
-        launches["n"] += 2
-        marks = mark_pool.pop() if (rec is not None and mark_pool) else None
+        launches["n"] += 2                       # k_accum_norms, k_norm_finalize
+        e2 = ev(); e2.record(stream)
         ds.select_and_update_all(e, plan, marks)
-        launches["n"] += int((plan.rank_k > 0).sum())   # one fused kernel per rank (the zeroing is inside it)
+        e3 = ev(); e3.record(stream)
+        launches["n"] += 1 if marks is None else int((plan.rank_k > 0).sum())   # k_select_fused
         if rec is not None:
-            rec.append({"acc": (e0, e1), "host_s": th1 - th0, "ranks": marks, "plan": plan})
+            rec.append({"acc": (e0, e1), "sel": (e2, e3), "host_s": th1 - th0, "ranks": marks, "plan": plan})
         return plan
 
     if args.mode == "sweep":
@@ -362,12 +356,23 @@ def run_ours(args):
     # per-call statistics from the events recorded inside the timed region
     t_acc = np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in recs])
     t_host = np.array([r["host_s"] * 1e3 for r in recs])
-    t_sel = np.array([[a.elapsed_time(b) for (a, b, c) in r["ranks"]] for r in recs])      # [steps, N]
-    t_upd = np.array([[b.elapsed_time(c) for (a, b, c) in r["ranks"]] for r in recs])
+    t_all = np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in recs])
     plan = recs[-1]["plan"]
+
+    # the per-worker view: the same steps with one launch per rank and events around every launch
+    # (outside the timed region; the vector keeps evolving as in training)
+    rank_recs = []
+    for it in range(max(3, min(args.steps, 20))):
+        tri = [(ev(), ev(), ev()) for _ in range(N)]
+        for t3 in tri:
+            for x in t3:
+                x.record(stream)
+        one_step(args.warmup + args.steps + it, rank_recs, g, tri)
+    stream.synchronize()
+    t_sel = np.array([[a.elapsed_time(b) for (a, b, c) in r["ranks"]] for r in rank_recs])      # [steps, N]
+    plan_w = rank_recs[-1]["plan"]
     sel_med = np.median(t_sel, axis=0)
-    upd_med = np.median(t_upd, axis=0)
-    worker_ms = float(np.median(t_acc) + np.median(t_host) + np.max(sel_med + upd_med))
+    worker_ms = float(np.median(t_acc) + np.median(t_host) + np.max(sel_med))
 
     # full-vector Top-k on the same GPU (comparison sparsifier), timed alone
     tk_val = torch.empty(k, dtype=torch.float32, device=dev)
@@ -415,14 +420,33 @@ def run_ours(args):
         acc_bytes = 12.0 * n_g
         acc_ms = float(np.median(t_acc))
         acc_gbs = acc_bytes / (acc_ms * 1e-3) / 1e9
-        sel_bytes = 8.0 * plan.rank_elems + 12.0 * plan.rank_k
+        # per-worker launches (worker view)
+        sel_bytes = 8.0 * plan_w.rank_elems + 12.0 * plan_w.rank_k
         with np.errstate(divide="ignore", invalid="ignore"):
             sel_gbs = np.where(sel_med > 0, sel_bytes / (sel_med * 1e-3) / 1e9, 0.0)
-        busy = plan.rank_elems > 0
-        sel_total_gbs = float(sel_bytes[busy].sum() / (sel_med[busy].sum() * 1e-3) / 1e9)
+        busy = plan_w.rank_elems > 0
         r_max = int(np.argmax(sel_med))
-        cost_max = float(plan.bin_load.max())
+        cost_max = float(plan_w.bin_load.max())
         lnk = math.log(k)
+        # the all-ranks launch of the timed step
+        all_ms = float(np.median(t_all))
+        all_bytes = 8.0 * n_g + 12.0 * float(plan.sum_k)
+        all_gbs = all_bytes / (all_ms * 1e-3) / 1e9
+        roof_sel = {"bound": "hbm", "kernel": "k_select_fused (all %d workers' partitions in one launch)" % N,
+                    "achieved": all_gbs, "peak": peak, "unit": "GB/s", "frac": all_gbs / peak, "peak_kind": peak_kind,
+                    "traffic": 8.0 * n_g + 4.0e6 * n_g / 135891278.0,
+                    "traffic_note": "per launch, scaled by elements from an ncu capture on 135.9 M elements "
+                                    "(8.00 B/element read, two reads of the vector; 4 MB written)",
+                    "bytes_per_launch": all_bytes, "ms_per_launch": all_ms, "bytes_per_elem": 8,
+                    "bytes_per_selected": 12, "share_of_step": all_ms / ms_per_step}
+        roof_acc = {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,
+                    "peak": peak, "unit": "GB/s", "frac": acc_gbs / peak, "peak_kind": peak_kind,
+                    "traffic": 11.69 * n_g,
+                    "traffic_note": "per launch, scaled by elements from an ncu capture on 135.9 M elements "
+                                    "(8.00 B/element read + 3.69 written before the kernel ends)",
+                    "bytes_per_launch": acc_bytes, "ms_per_launch": acc_ms, "share_of_step": acc_ms / ms_per_step,
+                    "frac_of_nominal_8TBs": acc_gbs / 8000.0}
+        sel_dominant = all_ms >= acc_ms
         cpu = None
         if not args.no_cpu_baseline:
             c = oracle_step_sample(w, g_host.numpy(), args.cpu_ranks)
@@ -440,36 +464,29 @@ def run_ours(args):
             "e2e": {"value": world * n_g / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 4 * n_g, "d2h_bytes_per_step": 12 * int(plan.sum_k) + 8 * L},
             "gpu_launches": gpu_launches,
-            # dominant kernel of the step by time (32 launches, ~65-80 % of the step): the fused selection
-            "roofline": {"bound": "hbm", "kernel": "k_select_fused (one launch per simulated worker)",
-                         "achieved": sel_total_gbs, "peak": peak, "unit": "GB/s", "frac": sel_total_gbs / peak,
-                         "peak_kind": peak_kind,
-                         "traffic": 4.02 * float(plan.rank_elems[busy].mean()) + 12.0 * float(plan.rank_k[busy].mean()),
-                         "traffic_note": "per launch, scaled by elements from an ncu capture of an 8.5 M-element "
-                                         "rank (4.02 B/element read: the second read of a rank hits L2)",
-                         "bytes_per_launch": float(sel_bytes[busy].mean()),
-                         "ms_per_launch": float(sel_med[busy].mean()),
-                         "bytes_per_elem": 8, "bytes_per_selected": 12,
-                         "frac_mean_over_ranks": float(sel_gbs[busy].mean() / peak),
-                         "frac_slowest_rank": float(sel_gbs[r_max] / peak),
-                         "floor_us_mean": float(sel_bytes[busy].mean() / peak / 1e3),
-                         "note": "ranks of 8-16 M elements: latency-bound (floor ~10 us per launch, four grid barriers)"},
-            "roofline_accum": {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,
-                               "peak": peak, "unit": "GB/s", "frac": acc_gbs / peak, "peak_kind": peak_kind,
-                               "traffic": 11.69 * n_g,
-                               "traffic_note": "scaled by elements from an ncu capture on 135.9 M elements "
-                                               "(8.00 B/element read + 3.69 written before the kernel ends)",
-                               "bytes_per_launch": acc_bytes, "ms_per_launch": acc_ms,
-                               "frac_of_nominal_8TBs": acc_gbs / 8000.0},
+            # the dominant kernel of the timed step by time, then the other one
+            "roofline": roof_sel if sel_dominant else roof_acc,
+            "roofline_other": roof_acc if sel_dominant else roof_sel,
+            "roofline_select_per_worker": {
+                "bound": "hbm", "call": "k_select_fused, one launch per worker (timed outside the step)",
+                "bytes_per_elem": 8, "bytes_per_selected": 12, "unit": "GB/s", "peak": peak,
+                "achieved_mean": float(sel_gbs[busy].mean()), "achieved_min": float(sel_gbs[busy].min()),
+                "achieved_max": float(sel_gbs[busy].max()), "frac_mean": float(sel_gbs[busy].mean() / peak),
+                "frac_slowest_rank": float(sel_gbs[r_max] / peak),
+                "floor_us_mean": float(sel_bytes[busy].mean() / peak / 1e3),
+                "traffic_per_elem_ncu": 4.02,
+                "note": "ranks of 8-16 M elements are latency-bound (floor ~10 us, four grid barriers); "
+                        "the second read of a rank hits L2"},
             "worker_view": {"ms_per_step_slowest_worker": worker_ms, "gelems": n_g / (worker_ms * 1e-3) / 1e9,
                             "t_acc_norms_ms": acc_ms, "t_host_ms": float(np.median(t_host)),
                             "select_ms_max": float(sel_med.max()), "select_ms_mean": float(sel_med[busy].mean()),
-                            "select_ms_min": float(sel_med[busy].min()), "update_ms_max": float(upd_med.max()),
+                            "select_ms_min": float(sel_med[busy].min()),
+                            "select_all_workers_one_launch_ms": all_ms,
                             "select_gelems_system": n_g / (float(sel_med.max()) * 1e-3) / 1e9,
-                            "slowest_rank": r_max, "slowest_rank_elems": int(plan.rank_elems[r_max]),
-                            "slowest_rank_k": int(plan.rank_k[r_max]),
-                            "rank_elems_max_over_mean": float(plan.rank_elems.max() / plan.rank_elems.mean()),
-                            "rank_k_min": int(plan.rank_k.min()), "rank_k_max": int(plan.rank_k.max())},
+                            "slowest_rank": r_max, "slowest_rank_elems": int(plan_w.rank_elems[r_max]),
+                            "slowest_rank_k": int(plan_w.rank_k[r_max]),
+                            "rank_elems_max_over_mean": float(plan_w.rank_elems.max() / plan_w.rank_elems.mean()),
+                            "rank_k_min": int(plan_w.rank_k.min()), "rank_k_max": int(plan_w.rank_k.max())},
             "topk_baseline": {"ms": t_topk, "gbs": 8.0 * n_g / (t_topk * 1e-3) / 1e9,
                               "speedup_vs_slowest_rank": t_topk / float(sel_med.max()),
                               "model_f_n": n_g * lnk / cost_max if cost_max > 0 else None,

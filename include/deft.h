@@ -273,6 +273,21 @@ DEFT_API deft_status deft_select_update_ranks(float* acc_d, int64_t n_g, const v
                                               size_t ws_bytes, void* const* events, void* stream);
 
 /*
+ * All N workers' selections and residual updates of an uploaded plan in ONE launch: the same
+ * bytes in val_d / idx_d / acc_d as deft_select_update_ranks(…, 0, N, …), for evaluating the
+ * method (or simulating N workers) on a single device.  The paper has each worker run only its
+ * own partition (Section 4.3); here the union of the partitions — every layer with its own
+ * k_l, Algorithm 5 — is processed as one list in address order and every layer's entries land
+ * where its worker's call would have put them.  Falls back to one launch per rank when the
+ * plan exceeds what one launch can hold (more than 256 streamed layers or 4096 tiles per CTA)
+ * or when the ranks' layers overlap.
+ * Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+DEFT_API deft_status deft_select_update_all(float* acc_d, int64_t n_g, const void* plan_h, const void* plan_d,
+                                            float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d,
+                                            size_t ws_bytes, void* stream);
+
+/*
  * Residual update — Algorithm 1 lines 11-12: acc[idx[j]] = +0.0f for j < count; the
  * buffer is then the next step's local error.  Indices must be distinct and < n_g.
  *   idx_d[count] DEVICE.  count may be 0.  Errors: INVALID_ARG, CUDA.

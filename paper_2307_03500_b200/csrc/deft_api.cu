@@ -1,5 +1,6 @@
 // C-ABI entry points of libdeft that touch the GPU: argument checks, the per-step plan
 // (host-built tables of every rank's layers), workspace carve-up and kernel launches.
+#include <algorithm>
 #include <cstring>
 #include <vector>
 
@@ -42,7 +43,7 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
     char* base = static_cast<char*>(blob);
     PlanHeader* hdr = reinterpret_cast<PlanHeader*>(base);
     RankInfo* ri = reinterpret_cast<RankInfo*>(base + sizeof(PlanHeader));
-    LayerDesc* desc = reinterpret_cast<LayerDesc*>(base + sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)N);
+    LayerDesc* desc = reinterpret_cast<LayerDesc*>(base + sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)(N + 1));
     std::memset(blob, 0, plan_bytes(L, N));
     int64_t tiles_all = 0, elems_all = 0, k_all = 0;
     int64_t d = 0;
@@ -85,6 +86,42 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
         elems_all += elems;
         k_all += k;
     }
+    // all ranks' layers as one list in address order
+    {
+        RankInfo& M = ri[N];
+        std::vector<LayerDesc> all;
+        all.reserve((size_t)L);
+        for (int64_t r = 0; r < N; ++r)
+            for (int32_t j = 0; j < ri[r].n_my; ++j) {
+                LayerDesc D = desc[ri[r].desc_first + j];
+                D.out_off += ri[r].out_off;
+                all.push_back(D);
+            }
+        std::sort(all.begin(), all.end(), [](const LayerDesc& a, const LayerDesc& b) { return a.start < b.start; });
+        bool disjoint = (int64_t)all.size() <= (int64_t)L;
+        for (size_t i = 1; i < all.size() && disjoint; ++i) disjoint = all[i].start >= all[i - 1].end;
+        M.desc_first = (int32_t)d;
+        M.n_my = 0;
+        if (disjoint && !all.empty()) {
+            int64_t tiles = 0, elems = 0;
+            for (LayerDesc& D : all) {
+                D.tile_first = (int32_t)tiles;
+                D.elem_off = elems;
+                tiles += (D.end - 1) / kTile - D.start / kTile + 1;
+                elems += D.end - D.start;
+                desc[d++] = D;
+            }
+            LayerDesc& Z = desc[d++];   // sentinel
+            Z.out_off = k_all;
+            Z.elem_off = elems;
+            Z.tile_first = (int32_t)tiles;
+            Z.layer_id = -1;
+            M.n_my = (int32_t)all.size();
+            M.tiles = (int32_t)tiles;
+            M.elems = elems;
+            M.k = k_all;
+        }
+    }
     hdr->magic = kPlanMagic;
     hdr->L = L;
     hdr->N = (int32_t)N;
@@ -112,7 +149,7 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
                         float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
                         cudaStream_t stream, bool zero_selected = false) {
     const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
-    if (rank < 0 || rank >= hdr->N) return DEFT_ERR_INVALID_ARG;
+    if (rank < 0 || rank > hdr->N) return DEFT_ERR_INVALID_ARG;   // rank N = all ranks' layers as one list
     const RankInfo& R = plan_ranks(plan_h)[rank];
     if (R.n_my == 0) return DEFT_OK;
     if (out_cap < R.k) return DEFT_ERR_CAPACITY;
@@ -264,7 +301,7 @@ deft_status deft_plan_rank_info(const void* plan_h, int32_t rank, int32_t* n_lay
                                 int64_t* elems_out, int64_t* k_out, int64_t* out_off_out) {
     if (!plan_ok(plan_h)) return DEFT_ERR_INVALID_ARG;
     const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
-    if (rank < 0 || rank >= hdr->N) return DEFT_ERR_INVALID_ARG;
+    if (rank < 0 || rank > hdr->N) return DEFT_ERR_INVALID_ARG;   // rank N = all ranks' layers as one list
     const RankInfo& R = plan_ranks(plan_h)[rank];
     if (n_layers_out) *n_layers_out = R.n_my;
     if (elems_out) *elems_out = R.elems;
@@ -330,6 +367,24 @@ deft_status deft_select_update_ranks(float* acc_d, int64_t n_g, const void* plan
         if (ev) DEFT_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(ev[2]), st));
     }
     return DEFT_OK;
+}
+
+deft_status deft_select_update_all(float* acc_d, int64_t n_g, const void* plan_h, const void* plan_d,
+                                   float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
+                                   void* stream) {
+    if (!plan_ok(plan_h) || !plan_d || !acc_d || !ws_d || !val_d || !idx_d || n_g < 1)
+        return DEFT_ERR_INVALID_ARG;
+    if (!aligned16(acc_d) || !aligned16(plan_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+    if (out_cap < hdr->total_k) return DEFT_ERR_CAPACITY;
+    const RankInfo& M = plan_ranks(plan_h)[hdr->N];
+    if (M.n_my > 0) {
+        const deft_status s = select_rank(acc_d, plan_h, plan_d, hdr->N, val_d, idx_d, M.k, ws_d, ws_bytes,
+                                          static_cast<cudaStream_t>(stream), true);
+        if (s != DEFT_ERR_INVALID_ARG) return s;   // beyond one launch's limits: one launch per rank instead
+    }
+    return deft_select_update_ranks(acc_d, n_g, plan_h, plan_d, 0, hdr->N, val_d, idx_d, out_cap, ws_d, ws_bytes,
+                                    nullptr, stream);
 }
 
 deft_status deft_select(const float* acc_d, const int64_t* layer_start_h, const int64_t* k_l_h,

@@ -90,8 +90,11 @@ constexpr int kTileA = 8192;         // elements per CTA iteration
 
 // ---------------------------------------------------------------------------------
 // The plan: a position-independent blob built on the host once per step, copied to the
-// device as it is.  [PlanHeader][RankInfo x N][LayerDesc x (L + N)] — each rank's layer
-// list is followed by one sentinel entry.
+// device as it is.  [PlanHeader][RankInfo x (N + 1)][LayerDesc x (L + N)][LayerDesc x (L + 1)]
+// — each rank's layer list is followed by one sentinel entry.  RankInfo[N] and the last list
+// describe all N ranks' layers as ONE list in address order, with output offsets that place
+// every layer where its own rank's call would put it (for running all workers' selections on
+// one device in a single launch); n_my = 0 there if the ranks' layers overlap.
 // ---------------------------------------------------------------------------------
 constexpr uint32_t kPlanMagic = 0x44454654u;  // "DEFT"
 
@@ -131,14 +134,15 @@ struct LayerDesc {                   // 64 bytes
 static_assert(sizeof(LayerDesc) == 64, "LayerDesc layout");
 
 inline size_t plan_bytes(int64_t L, int64_t N) {
-    return sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)N + sizeof(LayerDesc) * (size_t)(L + N);
+    return sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)(N + 1) + sizeof(LayerDesc) * (size_t)(L + N) +
+           sizeof(LayerDesc) * (size_t)(L + 1);
 }
 inline const RankInfo* plan_ranks(const void* plan) {
     return reinterpret_cast<const RankInfo*>(static_cast<const char*>(plan) + sizeof(PlanHeader));
 }
 inline const LayerDesc* plan_descs(const void* plan, int64_t N) {
     return reinterpret_cast<const LayerDesc*>(static_cast<const char*>(plan) + sizeof(PlanHeader) +
-                                              sizeof(RankInfo) * (size_t)N);
+                                              sizeof(RankInfo) * (size_t)(N + 1));
 }
 
 struct LayerState {                  // per layer, written by the kernels; 64 bytes

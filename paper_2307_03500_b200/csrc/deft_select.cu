@@ -178,31 +178,33 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratc
     return scratch[w] + incl - v;
 }
 
-// CTA-wide: walks a histogram of kBins bins (kBins / kSelThreads consecutive bins per thread,
-// at most 32) from its top bin down and finds the bucket that holds the k-th largest key.
-// out[0] = bucket, out[1] = keys strictly above it.
-template <int kBins, bool kGlobal>
-__device__ __forceinline__ void block_scan_select(const uint32_t* h, uint32_t k, uint32_t* scratch, uint32_t* out) {
-    constexpr int kPer = (kBins + kSelThreads - 1) / kSelThreads;
-    static_assert(kPer <= 32 && (kBins % kPer) == 0, "bins per thread");
-    const int base = kBins - kPer * ((int)threadIdx.x + 1);   // thread order = descending bins
-    uint32_t c[kPer];
+// The searches below run once per layer and step; they are kept out of line and free of
+// unrolled register arrays so that the kernel's straight-line code stays short (at small
+// ranks the kernel is bound by latencies, instruction fetch among them).
+
+// CTA-wide: walks a histogram of `bins` bins (bins / kSelThreads consecutive bins per thread;
+// bins a multiple of kSelThreads) from its top bin down and finds the bucket that holds the
+// k-th largest key.  out[0] = bucket, out[1] = keys strictly above it.  `global`: the histogram
+// is in global memory and was written by other CTAs (read past L1).
+__device__ __noinline__ void block_scan_select(const uint32_t* h, int bins, bool global, uint32_t k,
+                                               uint32_t* scratch, uint32_t* out) {
+    const int per = bins / kSelThreads;
+    const int base = bins - per * ((int)threadIdx.x + 1);   // thread order = descending bins
+    uint32_t c[8];   // all loads in flight together (per <= 8)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c[i] = i < per ? (global ? __ldcg(h + base + i) : h[base + i]) : 0u;
     uint32_t sum = 0;
 #pragma unroll
-    for (int i = 0; i < kPer; ++i) {
-        c[i] = 0;
-        if (base >= 0) c[i] = kGlobal ? __ldcg(h + base + i) : h[base + i];
-        sum += c[i];
-    }
+    for (int i = 0; i < 8; ++i) sum += c[i];
     if (threadIdx.x == 0) { out[0] = 0; out[1] = 0; }
     uint32_t total;
     const uint32_t excl = block_excl_scan(sum, scratch, total);   // keys in bins above mine
-    if (sum != 0 && excl < k && k <= excl + sum) {
+    if (sum != 0 && excl < k && k <= excl + sum) {                // exactly one thread
         uint32_t run = excl;
         bool found = false;
 #pragma unroll
-        for (int i = kPer - 1; i >= 0; --i) {
-            if (!found) {
+        for (int i = 7; i >= 0; --i) {
+            if (!found && i < per) {
                 if (run + c[i] >= k) { out[0] = (uint32_t)(base + i); out[1] = run; found = true; }
                 else run += c[i];
             }
@@ -211,37 +213,33 @@ __device__ __forceinline__ void block_scan_select(const uint32_t* h, uint32_t k,
     __syncthreads();
 }
 
-// One warp: the same search on a histogram of 32 * kPerLane bins in global memory (kPerLane =
-// 8, 16 or 32).  Lane l reads bins [kPerLane * l, kPerLane * (l + 1)); lane 31 holds the top.
-template <int kPerLane>
-__device__ __forceinline__ void warp_scan_select(const uint32_t* __restrict__ h, uint32_t k, int lane,
-                                                 uint32_t& bucket, uint32_t& above) {
-    uint32_t c[kPerLane];
+// One warp: the same search on a histogram of 32 * per bins in global memory (per a multiple
+// of 4, at most 32).  First the lanes' sums (lane l covers bins [per * l, per * (l + 1)), lane 31
+// the top), then the bins of the lane that holds the k-th key, one bin per lane.
+// Returns (bucket, keys strictly above it).
+__device__ __noinline__ uint2 warp_scan_select(const uint32_t* __restrict__ h, int per, uint32_t k) {
+    const int lane = threadIdx.x & 31;
     uint32_t sum = 0;
+    const uint4* h4 = reinterpret_cast<const uint4*>(h + per * lane);
+    uint4 v[8];      // all loads in flight together (per <= 32)
 #pragma unroll
-    for (int i = 0; i < kPerLane / 4; ++i) {
-        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(h + kPerLane * lane) + i);
-        c[4 * i] = v.x; c[4 * i + 1] = v.y; c[4 * i + 2] = v.z; c[4 * i + 3] = v.w;
-        sum += v.x + v.y + v.z + v.w;
-    }
+    for (int i = 0; i < 8; ++i) v[i] = 4 * i < per ? __ldcg(h4 + i) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sum += v[i].x + v[i].y + v[i].z + v[i].w;
     const uint32_t ab = warp_suffix_sum(sum, lane) - sum;   // keys in lanes above mine
     const unsigned hit = __ballot_sync(0xffffffffu, sum != 0 && ab < k && k <= ab + sum);
-    bucket = 0; above = 0;
-    if (hit == 0) return;            // k exceeds the histogram total: cannot happen for a valid plan
+    if (hit == 0) return make_uint2(0u, 0u);   // k exceeds the histogram total: cannot happen for a valid plan
     const int owner = __ffs(hit) - 1;
-    uint32_t b = 0, a = ab;
-    bool found = false;
-#pragma unroll
-    for (int i = kPerLane - 1; i >= 0; --i) {
-        if (!found) {
-            if (a + c[i] >= k) { b = kPerLane * lane + i; found = true; }
-            else a += c[i];
-        }
-    }
-    bucket = __shfl_sync(0xffffffffu, b, owner);
-    above = __shfl_sync(0xffffffffu, a, owner);
+    const uint32_t ab_owner = __shfl_sync(0xffffffffu, ab, owner);
+    const uint32_t c = lane < per ? __ldcg(h + per * owner + lane) : 0u;
+    const uint32_t a = ab_owner + warp_suffix_sum(c, lane) - c;   // keys above this bin
+    const unsigned hit2 = __ballot_sync(0xffffffffu, c != 0 && a < k && k <= a + c);
+    const int b = __ffs(hit2) - 1;
+    return make_uint2((uint32_t)(per * owner + b), __shfl_sync(0xffffffffu, a, b));
 }
-static_assert(kBins2 % 128 == 0 && kBins3 % 128 == 0 && kBins2 <= 1024 && kBins3 <= 1024, "warp_scan_select shapes");
+static_assert(kBins2 % 128 == 0 && kBins3 % 128 == 0 && kBins2 <= 1024 && kBins3 <= 1024 && kBins1 <= 8 * kSelThreads &&
+              kBins1 % kSelThreads == 0 && kDBins1 % kSelThreads == 0 && kDBins2 % kSelThreads == 0 &&
+              kDBins3 % kSelThreads == 0, "search shapes");
 
 // ---------------------------------------------------------------------------------
 // tile workers: one warp holds a whole tile (kTile = 2048 elements) in registers
@@ -313,7 +311,7 @@ __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
 // CTA-wide pass over the CTA's staged entries, in no particular order.  The spilled part is
 // read in batches of kSpillBatch loads per thread so that the pass is not bound by one
 // HBM round trip per entry.
-constexpr int kSpillBatch = 8;
+constexpr int kSpillBatch = 4;
 constexpr int kEmitBatch = 4;
 template <typename F>
 __device__ __forceinline__ void for_each_staged(const Stage& st, uint32_t total, F f) {
@@ -652,8 +650,8 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
             const int cl = c0 + s;
             const int lid = lt->lid[cl];
             __threadfence();
-            block_scan_select<kBins1, true>(p.hist1 + (size_t)lid * kBins1, lt->k[cl],
-                                            misc + kMScratch, misc + kMOut3);
+            block_scan_select(p.hist1 + (size_t)lid * kBins1, kBins1, true, lt->k[cl], misc + kMScratch,
+                              misc + kMOut3);
             if (threadIdx.x == 0) {
                 p.state[lid].b1 = misc[kMOut3];
                 p.state[lid].above1 = misc[kMOut3 + 1];
@@ -717,8 +715,8 @@ __device__ __forceinline__ void step_hist3(const SelParams& p, LayerTable* lt, i
     if (p.timing && threadIdx.x == 0) { atomicMax(p.timing + 14, (unsigned long long)total); atomicAdd(p.timing + 15, (unsigned long long)total); }
     for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer
         const int lid = lt->lid[c];
-        uint32_t b2, above2;
-        warp_scan_select<kBins2 / 32>(p.hist2 + (size_t)lid * kBins2, lt->v1[c], lane, b2, above2);
+        const uint2 s2 = warp_scan_select(p.hist2 + (size_t)lid * kBins2, kBins2 / 32, lt->v1[c]);
+        const uint32_t b2 = s2.x, above2 = s2.y;
         const uint32_t b1 = __ldcg(&p.state[lid].b1);
         __syncwarp();
         if (lane == 0) {
@@ -754,8 +752,8 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t total = misc[kMCursor];
     for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer
-        uint32_t b3, above3;
-        warp_scan_select<kBins3 / 32>(p.hist3 + (size_t)lt->lid[c] * kBins3, lt->v1[c], lane, b3, above3);
+        const uint2 s3 = warp_scan_select(p.hist3 + (size_t)lt->lid[c] * kBins3, kBins3 / 32, lt->v1[c]);
+        const uint32_t b3 = s3.x, above3 = s3.y;
         __syncwarp();
         if (lane == 0) {
             lt->v0[c] = (lt->v0[c] << kShift2) | b3;   // T
@@ -792,7 +790,9 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
 
 // Ordered write of one batch of 32 consecutive staged entries (one per lane).  gt_before /
 // eq_before: entries above / equal to the threshold that precede the batch in the layer.
-__device__ __forceinline__ void emit_batch(const SelParams& p, int64_t out_off, int64_t elem0, bool valid,
+struct EmitOut { float* val; int64_t* idx; float* acc_rw; };
+
+__device__ __forceinline__ void emit_batch(const EmitOut& p, int64_t out_off, int64_t elem0, bool valid,
                                            uint32_t bits, int64_t off, uint32_t T, uint32_t need,
                                            uint32_t& gt_before, uint32_t& eq_before, int lane) {
     const uint32_t lt_mask = (1u << lane) - 1u;
@@ -816,13 +816,17 @@ __device__ __forceinline__ void emit_batch(const SelParams& p, int64_t out_off, 
 // ---------------------------------------------------------------------------------
 // One batch of local tiles [t0, tend): pref[lq - t0] = entries above / equal to T that precede
 // tile lq in its layer.  One warp per tile writes the tile's selected entries.
-__device__ __forceinline__ void emit_tiles(const SelParams& p, const CtaRange& r, const TileTable* tt,
-                                           const Stage& st, const uint2* pref, int t0, int tend, int64_t start,
-                                           int tf, int64_t out_off, uint32_t T, uint32_t need) {
+__device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, const TileTable* tt, uint2* res,
+                                        uint2* spill, const uint2* pref, int t0, int tend, int64_t start, int tf,
+                                        int64_t out_off, uint32_t T, uint32_t need) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Stage st{res, spill};
     for (int lq = t0 + warp; lq < tend; lq += kSelWarps) {
-        const int q = local_tile(p, r, lq);
-        if (q < 0) continue;
+        int q = q0 + lq;
+        if (il) {
+            q = kSuper * ((int)blockIdx.x + (lq / kSuper) * (int)gridDim.x) + lq % kSuper;
+            if (q >= tiles) continue;
+        }
         const uint32_t n = tt->n[lq];
         if (n == 0) continue;
         const uint32_t first = tt->first[lq];
@@ -838,7 +842,7 @@ __device__ __forceinline__ void emit_tiles(const SelParams& p, const CtaRange& r
 #pragma unroll
             for (int u = 0; u < kEmitBatch; ++u) {
                 if (e0 + u * 32 < n)   // uniform over the warp
-                    emit_batch(p, out_off, lo, e0 + u * 32 + lane < n, ent[u].x, (int64_t)y_off(ent[u].y), T, need,
+                    emit_batch(out, out_off, lo, e0 + u * 32 + lane < n, ent[u].x, (int64_t)y_off(ent[u].y), T, need,
                                gt_before, eq_before, lane);
             }
         }
@@ -889,7 +893,8 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             pref[threadIdx.x] = make_uint2(sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
             __syncthreads();
             const int tend = t0 + kSelThreads < r.nloc ? t0 + kSelThreads : r.nloc;
-            emit_tiles(p, r, tt, st, pref, t0, tend, lt->start[0], lt->tf[0], lt->out_off[0], T, need);
+            emit_tiles(EmitOut{p.val, p.idx, p.acc_rw}, p.tiles, 1, 0, tt, st.res, st.spill, pref, t0, tend, lt->start[0],
+                       lt->tf[0], lt->out_off[0], T, need);
             __syncthreads();   // pref is rewritten by the next batch
         }
         return;
@@ -923,7 +928,8 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             pref[threadIdx.x] = make_uint2(base_gt + e_gt, base_eq + e_eq);
             __syncthreads();
             const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
-            emit_tiles(p, r, tt, st, pref, t0, tend, lt->start[c], lt->tf[c], lt->out_off[c], T, need);
+            emit_tiles(EmitOut{p.val, p.idx, p.acc_rw}, p.tiles, 0, r.q0, tt, st.res, st.spill, pref, t0, tend, lt->start[c],
+                       lt->tf[c], lt->out_off[c], T, need);
             base_gt += tot_gt;
             base_eq += tot_eq;
             __syncthreads();   // pref is rewritten by the next batch
@@ -970,7 +976,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
         }
     }
     __syncthreads();
-    block_scan_select<kDBins1, false>(h1, k, scratch, out3);
+    block_scan_select(h1, kDBins1, false, k, scratch, out3);
     const uint32_t b1 = out3[0], above1 = out3[1];
     __syncthreads();
     // level 2 inside bucket b1
@@ -979,7 +985,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
         if ((key >> kDShift1) == b1) atomicAdd(&h[(key >> kDShift2) & (kDBins2 - 1)], 1u);
     }
     __syncthreads();
-    block_scan_select<kDBins2, false>(h, k - above1, scratch, out3);
+    block_scan_select(h, kDBins2, false, k - above1, scratch, out3);
     const uint32_t b2 = out3[0];
     const uint32_t krem2 = k - above1 - out3[1];
     __syncthreads();
@@ -992,7 +998,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
         if ((key >> kDShift2) == prefix) atomicAdd(&h[key & (kDBins3 - 1)], 1u);
     }
     __syncthreads();
-    block_scan_select<kDBins3, false>(h, krem2, scratch, out3);
+    block_scan_select(h, kDBins3, false, krem2, scratch, out3);
     const uint32_t T = (prefix << kDShift2) | out3[0];
     const uint32_t need = krem2 - out3[1];
     __syncthreads();
@@ -1016,7 +1022,8 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
     for (uint32_t fb = f0; fb < f1; fb += 32) {
         const uint32_t f = fb + lane;
         const bool valid = f < f1;
-        emit_batch(p, out_off, start, valid, valid ? skey[f] : 0u, (int64_t)f, T, need, gt_before, eq_before, lane);
+        emit_batch(EmitOut{p.val, p.idx, p.acc_rw}, out_off, start, valid, valid ? skey[f] : 0u, (int64_t)f, T, need,
+                   gt_before, eq_before, lane);
     }
     __syncthreads();   // shared memory is reused by the next layer
 }

@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.deft_plan_upload.argtypes = [vp, vp, vp, sz, vp]
         L.deft_select_planned.restype = i32
         L.deft_select_planned.argtypes = [vp, vp, vp, i32, vp, vp, i64, vp, sz, vp]
+        L.deft_select_update_all.restype = i32
+        L.deft_select_update_all.argtypes = [vp, i64, vp, vp, vp, vp, i64, vp, sz, vp]
         L.deft_select_update_ranks.restype = i32
         L.deft_select_update_ranks.argtypes = [vp, i64, vp, vp, i32, i32, vp, vp, i64, vp, sz, vp, vp]
         L.deft_residual_update.restype = i32
@@ -344,6 +346,16 @@ def deft_select_update_ranks(acc, plan_h: np.ndarray, plan_d, rank_begin: int, r
                                           int(rank_begin), int(rank_end), _dp(val_d, torch.float32),
                                           _dp(idx_d, torch.int64), min(val_d.numel(), idx_d.numel()), _dp(ws),
                                           ws.numel() * ws.element_size(), ev, _stream(stream)))
+
+
+def deft_select_update_all(acc, plan_h: np.ndarray, plan_d, val_d, idx_d, ws, stream=None) -> None:
+    """Selection + residual update for ALL simulated ranks of the plan in one launch."""
+    import torch
+    _check("deft_select_update_all",
+           lib().deft_select_update_all(_dp(acc, torch.float32), acc.numel(), _hp(plan_h), _dp(plan_d),
+                                        _dp(val_d, torch.float32), _dp(idx_d, torch.int64),
+                                        min(val_d.numel(), idx_d.numel()), _dp(ws), ws.numel() * ws.element_size(),
+                                        _stream(stream)))
 
 
 def deft_residual_update(acc, idx_d, count: int, stream=None) -> None:

@@ -88,22 +88,27 @@ class DeftStep:
             deft.deft_select_planned(acc, plan.plan_h, self.plan_d, rank, val, idx, self.ws)
         return val, idx
 
-    def select_and_update_all(self, acc: torch.Tensor, plan: StepPlan, events=None) -> None:
-        """Selection followed by the residual update for every simulated rank, rank after rank (one C call).
+    def select_and_update_all(self, acc: torch.Tensor, plan: StepPlan, events=None, per_rank: bool = False) -> None:
+        """Selection followed by the residual update for every simulated rank (one C call): all ranks in
+        one launch, or — with `per_rank` or `events` — one launch per rank, rank after rank.
         `events`: optional list of (before, between, after) CUDA events per rank, recorded on the stream."""
-        deft.deft_select_update_ranks(acc, plan.plan_h, self.plan_d, 0, self.N, self.val_d, self.idx_d, self.ws,
-                                      events)
+        if events is None and not per_rank:
+            deft.deft_select_update_all(acc, plan.plan_h, self.plan_d, self.val_d, self.idx_d, self.ws)
+        else:
+            deft.deft_select_update_ranks(acc, plan.plan_h, self.plan_d, 0, self.N, self.val_d, self.idx_d, self.ws,
+                                          events)
 
     def residual_update(self, acc: torch.Tensor, idx: torch.Tensor) -> None:
         deft.deft_residual_update(acc, idx, idx.numel())
 
     # -- the whole step for all simulated ranks ---------------------------------------------
-    def step(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, events=None):
+    def step(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, events=None,
+             per_rank: bool = False):
         """accumulate + norms -> plan -> (selection, residual update) for every rank.  Returns the plan and,
         per rank, views of its selected (values, indices)."""
         norms = self.layer_norms(resid, grad)
         plan = self.plan(norms, iteration)
-        self.select_and_update_all(resid, plan, events)
+        self.select_and_update_all(resid, plan, events, per_rank)
         off = plan.rank_out_off
         outs = [(self.val_d[int(off[r]):int(off[r + 1])], self.idx_d[int(off[r]):int(off[r + 1])])
                 for r in range(self.N)]

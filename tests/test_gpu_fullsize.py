@@ -51,11 +51,22 @@ def test_bench_configuration_full_size(deft):
     ds = DeftStep(w.sizes, N, w.density)
     e_d = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
     g_d = torch.from_numpy(g).cuda()
+    # the benchmark's timed path: all ranks in one launch
     plan, outs = ds.step(e_d, g_d, iteration=0)
     torch.cuda.synchronize()
     val_all = ds.val_d[: plan.sum_k].cpu().numpy()
     idx_all = ds.idx_d[: plan.sum_k].cpu().numpy()
     resid = e_d.cpu().numpy()
+    # the per-worker path (one launch per rank, what the worker-view timings use): same bytes
+    e_d.zero_()
+    ds.val_d.zero_()
+    ds.idx_d.zero_()
+    plan2, _ = ds.step(e_d, g_d, iteration=0, per_rank=True)
+    torch.cuda.synchronize()
+    assert plan2.sum_k == plan.sum_k and plan2.k_l.tolist() == plan.k_l.tolist()
+    assert ds.val_d[: plan.sum_k].cpu().numpy().tobytes() == val_all.tobytes()
+    assert np.array_equal(ds.idx_d[: plan.sum_k].cpu().numpy(), idx_all)
+    assert e_d.cpu().numpy().tobytes() == resid.tobytes()
     del g_d
 
     start, _ = oracle.split_layers(w.sizes, N)

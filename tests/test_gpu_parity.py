@@ -139,11 +139,22 @@ def _whole_path(deft, w, steps=1, mode=None, iteration=0):
             seen[want_idx] += 1
             all_idx.append(idx_d)
         assert seen.max() == 1 and int(seen.sum()) == s       # disjoint, density kept
+        # all ranks in one launch (selection + zeroing): same bytes as the per-rank calls
+        val_pr, idx_pr = ds.val_d[:s].clone(), ds.idx_d[:s].clone()
+        e_all = e_gpu.clone()
+        ds.val_d.fill_(7.0)
+        ds.idx_d.fill_(-7)
+        deft.deft_plan_upload(plan.plan_h, ds.plan_d, ds.ws)   # the per-layer scratch state is single-use
+        ds.select_and_update_all(e_all, plan)
+        torch.cuda.synchronize()
+        assert torch.equal(ds.idx_d[:s], idx_pr) and ds.val_d[:s].cpu().numpy().tobytes() == val_pr.cpu().numpy().tobytes()
+        assert torch.all(ds.idx_d[s:] == -7)
         for idx_d in all_idx:
             ds.residual_update(e_gpu, idx_d)
         torch.cuda.synchronize()
         oracle.residual_update(e_cpu, np.nonzero(seen)[0])
         assert e_gpu.cpu().numpy().tobytes() == e_cpu.tobytes()
+        assert e_all.cpu().numpy().tobytes() == e_cpu.tobytes()
 
 
 def test_whole_path_tiny(deft):

@@ -60,11 +60,14 @@ DEFT_API const char* deft_status_string(deft_status s);
 DEFT_API int32_t deft_last_cuda_error(void);
 
 /*
- * Diagnostic: when timing_d (DEVICE, 16 x uint64, zeroed by the caller) is not NULL every
+ * Diagnostic: when timing_d (DEVICE, 1024 x uint64, zeroed by the caller) is not NULL every
  * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs):
- * [0] kernel start, [1] end of histogram pass, [2] after barrier, [3] end of staging pass,
- * [4] after barrier, [5] end of per-layer finish, [6] end of the general path (0 if not
- * taken).  Pass NULL to switch it off.  Not thread-safe; not for production use.
+ * [0] kernel start, [1] end of the level-1 histogram step, [2] end of the staging step,
+ * [3] level-3 histograms done, [4] per-tile counts done, [5] ordered write done, [6] small
+ * layers done; inside the first step [8] histograms zeroed, [9] tiles read, [10] flushed,
+ * [11] tickets taken; [14] / [15] staged entries (max over CTAs / total); [16 + b],
+ * [176 + b], [336 + b] per CTA b: staging-step nanoseconds, staged entries, local layers |
+ * local tiles << 16.  Pass NULL to switch it off.  Not thread-safe; not for production use.
  */
 DEFT_API void deft_debug_select_timing(void* timing_d);
 

@@ -207,7 +207,7 @@ struct SelParams {
     uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output
     int64_t* idx;
-    unsigned long long* timing;      // optional: 16 phase timestamps (ns, max over CTAs); NULL = off
+    unsigned long long* timing;      // optional: 1024 words of phase stamps and per-CTA counters; NULL = off
 };
 
 // Sticky per-thread CUDA error code for deft_last_cuda_error().

@@ -1085,7 +1085,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
         p.timing[16 + 160 + blockIdx.x] = misc[kMCursor];
         p.timing[16 + 320 + blockIdx.x] = (unsigned long long)nl | ((unsigned long long)r.nloc << 16) |
                                           ((unsigned long long)misc[kMCursor + 1] << 32);
-        p.timing[16 + 480 + blockIdx.x] = misc[kMCursor + 2];
+        p.timing[16 + 480 + blockIdx.x] = misc[kMCursor + 2];   // profiling build: cycles in filter_marked
     }
     stamp(p, 2);
     grid.sync();

@@ -258,7 +258,7 @@ def deft_select(acc, layer_start_h, k_l_h, my_layers_h, val_d, idx_d, ws, stream
 
 
 def deft_debug_select_timing(timing_d) -> None:
-    """Diagnostic phase stamps of the selection kernel: a zeroed CUDA uint64/int64 tensor of 16, or None."""
+    """Diagnostic phase stamps of the selection kernel: a zeroed CUDA uint64/int64 tensor of 1024, or None."""
     lib().deft_debug_select_timing(None if timing_d is None else _dp(timing_d))
 
 

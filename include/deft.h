@@ -213,6 +213,22 @@ DEFT_API deft_status deft_layer_norms_static(float* resid_acc_d, const float* gr
                                              void* stream);
 
 /*
+ * One step's host work in one call: Algorithm 3 (deft_allocate_k on the layer sizes implied by
+ * layer_start_h), Algorithm 4 (deft_partition), deft_plan_build and deft_plan_upload, in that
+ * order, with the same results as the four separate calls.  norms_h: HOST [L], this step's
+ * norms.  Outputs (HOST): k_l_h [L], *sum_k_out (may be NULL), bin_of_layer_h [L],
+ * bin_load_h [N] (may be NULL), plan_h (plan_bytes_cap >= deft_plan_bytes(L, N); pinned
+ * memory lets the upload overlap).  plan_d / ws_d: DEVICE, as for deft_plan_upload.
+ * Returns DEFT_OK or DEFT_WARN_K_INEXACT (PAPER mode, sum of k_l differs from k; the plan is
+ * built and uploaded all the same); errors as the four calls.
+ */
+DEFT_API deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
+                                    int64_t k, int32_t mode, int64_t iteration, int64_t* k_l_h,
+                                    int64_t* sum_k_out, int32_t* bin_of_layer_h, double* bin_load_h,
+                                    void* plan_h, size_t plan_bytes_cap, void* plan_d, void* ws_d,
+                                    size_t ws_bytes, void* stream);
+
+/*
  * The per-step plan — Algorithm 4, lines 1-2 and 20 for every rank at once.
  * Once k_l (Algorithm 3) and the bins (Algorithm 4) of a step are known, the layer
  * lists of all N ranks are laid out in one position-independent blob: rank r owns the

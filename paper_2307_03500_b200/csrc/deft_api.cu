@@ -297,6 +297,25 @@ deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
     return fill_plan(plan_h, plan_bytes_cap, L, iteration, ranks);
 }
 
+deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
+                           int64_t k, int32_t mode, int64_t iteration, int64_t* k_l_h, int64_t* sum_k_out,
+                           int32_t* bin_of_layer_h, double* bin_load_h, void* plan_h, size_t plan_bytes_cap,
+                           void* plan_d, void* ws_d, size_t ws_bytes, void* stream) {
+    if (!norms_h || !layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || !plan_d || !ws_d || L < 1)
+        return DEFT_ERR_INVALID_ARG;
+    std::vector<int64_t> size((size_t)L);
+    for (int32_t l = 0; l < L; ++l) size[l] = layer_start_h[l + 1] - layer_start_h[l];
+    const deft_status sa = deft_allocate_k(norms_h, size.data(), L, k, mode, k_l_h, sum_k_out);
+    if (sa < 0) return sa;
+    deft_status s = deft_partition(size.data(), k_l_h, L, N, bin_of_layer_h, bin_load_h);
+    if (s != DEFT_OK) return s;
+    s = deft_plan_build(layer_start_h, k_l_h, bin_of_layer_h, L, N, iteration, plan_h, plan_bytes_cap);
+    if (s != DEFT_OK) return s;
+    s = deft_plan_upload(plan_h, plan_d, ws_d, ws_bytes, stream);
+    if (s != DEFT_OK) return s;
+    return sa;   // DEFT_OK, or the Algorithm 3 warning
+}
+
 deft_status deft_plan_rank_info(const void* plan_h, int32_t rank, int32_t* n_layers_out,
                                 int64_t* elems_out, int64_t* k_out, int64_t* out_off_out) {
     if (!plan_ok(plan_h)) return DEFT_ERR_INVALID_ARG;

@@ -313,6 +313,7 @@ __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
 // HBM round trip per entry.
 constexpr int kSpillBatch = 4;
 constexpr int kEmitBatch = 4;
+constexpr uint32_t kThreadEmit = 12;   // tiles with at most this many staged entries are written by one thread
 template <typename F>
 __device__ __forceinline__ void for_each_staged(const Stage& st, uint32_t total, F f) {
     const uint32_t nres = total < (uint32_t)kResident ? total : (uint32_t)kResident;
@@ -828,7 +829,7 @@ __device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, 
             if (q >= tiles) continue;
         }
         const uint32_t n = tt->n[lq];
-        if (n == 0) continue;
+        if (n <= kThreadEmit) continue;   // nothing staged, or written by the tile's own thread
         const uint32_t first = tt->first[lq];
         const int64_t lo = (start / kTile + (q - tf)) * kTile;
         uint32_t gt_before = pref[lq - t0].x, eq_before = pref[lq - t0].y;
@@ -846,6 +847,27 @@ __device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, 
                                gt_before, eq_before, lane);
             }
         }
+    }
+}
+
+// Tiles with at most kThreadEmit staged entries are written by ONE thread each (thread i of a
+// batch owns tile t0 + i, whose prefix it has just computed): at a few entries per tile a warp
+// per tile leaves most lanes idle and is bound by its own instruction latency.
+__device__ __forceinline__ void emit_small_tile(const EmitOut& out, const Stage& st, uint32_t first, uint32_t n,
+                                                int64_t out_off, int64_t lo, uint32_t T, uint32_t need,
+                                                uint32_t gt_before, uint32_t eq_before) {
+    for (uint32_t e = 0; e < n; ++e) {
+        const uint2 ent = stage_get(st, first + e);
+        const uint32_t key = key_of(ent.x);
+        if (key > T || (key == T && eq_before < need)) {
+            const int64_t pos = out_off + gt_before + (eq_before < need ? eq_before : need);
+            const int64_t elem = lo + (int64_t)y_off(ent.y);
+            out.val[pos] = __uint_as_float(ent.x);
+            out.idx[pos] = elem;
+            if (out.acc_rw) out.acc_rw[elem] = 0.0f;
+        }
+        gt_before += key > T;
+        eq_before += key == T;
     }
 }
 
@@ -891,6 +913,14 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             const uint32_t ex = incl - v;
             const uint2 sb = i < r.nloc ? sbase[i / kSuper] : make_uint2(0u, 0u);
             pref[threadIdx.x] = make_uint2(sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
+            {
+                const int q = i < r.nloc ? local_tile(p, r, i) : -1;
+                const uint32_t n = q >= 0 ? tt->n[i] : 0u;
+                if (n != 0 && n <= kThreadEmit)
+                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw}, st, tt->first[i], n, lt->out_off[0],
+                                    (lt->start[0] / kTile + (q - lt->tf[0])) * kTile, T, need,
+                                    sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
+            }
             __syncthreads();
             const int tend = t0 + kSelThreads < r.nloc ? t0 + kSelThreads : r.nloc;
             emit_tiles(EmitOut{p.val, p.idx, p.acc_rw}, p.tiles, 1, 0, tt, st.res, st.spill, pref, t0, tend, lt->start[0],
@@ -926,6 +956,13 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             const uint32_t e_gt = block_excl_scan(v & 0xffffu, scratch, tot_gt);
             const uint32_t e_eq = block_excl_scan(v >> 16, scratch, tot_eq);
             pref[threadIdx.x] = make_uint2(base_gt + e_gt, base_eq + e_eq);
+            {
+                const uint32_t n = i < tb ? tt->n[i] : 0u;
+                if (n != 0 && n <= kThreadEmit)
+                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw}, st, tt->first[i], n, lt->out_off[c],
+                                    (lt->start[c] / kTile + (r.q0 + i - lt->tf[c])) * kTile, T, need,
+                                    base_gt + e_gt, base_eq + e_eq);
+            }
             __syncthreads();
             const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
             emit_tiles(EmitOut{p.val, p.idx, p.acc_rw}, p.tiles, 0, r.q0, tt, st.res, st.spill, pref, t0, tend, lt->start[c],
@@ -1095,7 +1132,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     step_count(p, r, lt, nl, tt, st, smem);
     stamp(p, 4);
     grid.sync();
+    unsigned long long te0 = 0;
+    if (p.timing && threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(te0));
     step_emit(p, r, lt, nl, tt, st, smem);
+    if (p.timing && threadIdx.x == 0) {
+        unsigned long long te1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(te1));
+        p.timing[16 + 640 + blockIdx.x] = te1 - te0;
+    }
     stamp(p, 5);
     __syncthreads();
     for (int j = blockIdx.x; j < p.n_my; j += gridDim.x)

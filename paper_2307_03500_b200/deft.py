@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.deft_plan_rank_info.argtypes = [vp, i32, vp, vp, vp, vp]
         L.deft_plan_rank_table.restype = i32
         L.deft_plan_rank_table.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.deft_plan_step.restype = i32
+        L.deft_plan_step.argtypes = [vp, vp, i32, i32, i64, i32, i64, vp, vp, vp, vp, vp, sz, vp, vp, sz, vp]
         L.deft_plan_upload.restype = i32
         L.deft_plan_upload.argtypes = [vp, vp, vp, sz, vp]
         L.deft_select_planned.restype = i32
@@ -312,6 +314,30 @@ def deft_plan_upload(plan_h: np.ndarray, plan_d, ws, stream=None) -> None:
         raise ValueError("plan_d smaller than the plan")
     _check("deft_plan_upload", lib().deft_plan_upload(_hp(plan_h), _dp(plan_d), _dp(ws),
                                                       ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_plan_step(norms, layer_start_h, n_workers: int, k: int, mode: int, iteration: int, plan_h: np.ndarray,
+                   plan_d, ws, stream=None):
+    """Algorithm 3 + Algorithm 4 + plan build + plan upload in one call.
+    Returns (k_l int64[L], sum_k, bin_of_layer int32[L], bin_load float64[N], status)."""
+    nr = _np(norms, np.float64)
+    ls = _np(layer_start_h, np.int64)
+    L = nr.size
+    if ls.size != L + 1:
+        raise ValueError("norms and layer_start_h disagree")
+    if plan_d.numel() * plan_d.element_size() < deft_plan_bytes(L, n_workers) or plan_h.dtype != np.uint8 or \
+            not plan_h.flags.c_contiguous:
+        raise ValueError("plan buffers too small or not contiguous uint8")
+    k_l = np.empty(L, dtype=np.int64)
+    bins = np.empty(L, dtype=np.int32)
+    load = np.empty(int(n_workers), dtype=np.float64)
+    s = ctypes.c_int64(0)
+    st = _check("deft_plan_step",
+                lib().deft_plan_step(_hp(nr), _hp(ls), L, int(n_workers), int(k), int(mode), int(iteration), _hp(k_l),
+                                     ctypes.byref(s), _hp(bins), _hp(load), _hp(plan_h), plan_h.size, _dp(plan_d),
+                                     _dp(ws), ws.numel() * ws.element_size(), _stream(stream)),
+                allow_warn=True)
+    return k_l, int(s.value), bins, load, st
 
 
 def deft_select_planned(acc, plan_h: np.ndarray, plan_d, rank: int, val_d, idx_d, ws, stream=None) -> None:

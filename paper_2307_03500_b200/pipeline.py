@@ -67,10 +67,8 @@ class DeftStep:
     # -- steps 2 and 3: local k and bins (host) ---------------------------------------------
     def plan(self, norms: np.ndarray, iteration: int = 0) -> StepPlan:
         """Algorithm 3, Algorithm 4, then the plan of all N ranks built on the host and uploaded."""
-        k_l, sum_k, _ = deft.deft_allocate_k(norms, self.layer_size, self.k, self.mode)
-        bins, load = deft.deft_partition(self.layer_size, k_l, self.N)
-        deft.deft_plan_build(self.layer_start, k_l, bins, self.N, iteration, out=self.plan_h)
-        deft.deft_plan_upload(self.plan_h, self.plan_d, self.ws)
+        k_l, sum_k, bins, load, _ = deft.deft_plan_step(norms, self.layer_start, self.N, self.k, self.mode, iteration,
+                                                        self.plan_h, self.plan_d, self.ws)
         n_layers, elems, rank_k, out_off = deft.deft_plan_rank_table(self.plan_h, self.N)
         off = np.zeros(self.N + 1, dtype=np.int64)
         off[:-1] = out_off

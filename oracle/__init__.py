@@ -155,6 +155,34 @@ def residual_update(acc, idx):
     return acc
 
 
+def threshold_select(acc, threshold):
+    """Hard-threshold sparsifier (Section 3.2): entries with magnitude > threshold, ascending index."""
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    lib = _load()
+    lib.oracle_threshold_select.restype = ctypes.c_int64
+    n = lib.oracle_threshold_select(_p(acc), _i64(acc.size), ctypes.c_float(threshold), None, None, _i64(0))
+    val = np.empty(n, dtype=np.float32)
+    idx = np.empty(n, dtype=np.int64)
+    lib.oracle_threshold_select(_p(acc), _i64(acc.size), ctypes.c_float(threshold), _p(val), _p(idx), _i64(n))
+    return val, idx
+
+
+def clt_leader(iteration, n_workers):
+    """CLT-k (Section 3.1): the worker that selects in this iteration."""
+    lib = _load()
+    lib.oracle_clt_leader.restype = ctypes.c_int64
+    return int(lib.oracle_clt_leader(_i64(iteration), _i64(n_workers)))
+
+
+def gather_update(acc, idx):
+    """CLT-k follower: own values at the leader's indices, then cleared (in place).  Returns the values."""
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    ix = np.ascontiguousarray(idx, dtype=np.int64)
+    val = np.empty(ix.size, dtype=np.float32)
+    _load().oracle_gather_update(_p(acc), _p(ix), _i64(ix.size), _p(val))
+    return val
+
+
 def my_layers(bin_of_layer, iteration, rank, n_workers):
     """Layer ids (ascending) whose bin is the one ``rank`` reads this iteration."""
     b = rank_bin(iteration, rank, n_workers)

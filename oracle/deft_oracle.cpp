@@ -299,4 +299,42 @@ void oracle_residual_update(float* acc, const int64_t* idx, int64_t count) {
     for (int64_t j = 0; j < count; ++j) acc[idx[j]] = 0.0f;
 }
 
+// ---------------------------------------------------------------------------
+// Comparison sparsifiers (Section 3; not part of DEFT itself).
+// ---------------------------------------------------------------------------
+// Hard-threshold sparsifier (Section 3.2): every entry whose magnitude is larger than a fixed
+// threshold is selected, one O(n_g) check per entry.  "Larger" is read as strict, and the
+// magnitudes are compared in the same order Algorithm 5's selection uses (IEEE bit pattern
+// with the sign cleared), so a NaN entry counts as larger than any threshold.  Output in
+// ascending index.  Returns the number of selected entries; writes at most cap of them.
+int64_t oracle_threshold_select(const float* acc, int64_t n, float threshold, float* val, int64_t* idx,
+                                int64_t cap) {
+    uint32_t tbits;
+    std::memcpy(&tbits, &threshold, 4);
+    tbits &= 0x7fffffffu;
+    int64_t count = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        uint32_t b;
+        std::memcpy(&b, &acc[i], 4);
+        if ((b & 0x7fffffffu) > tbits) {
+            if (count < cap) { val[count] = acc[i]; idx[count] = i; }
+            ++count;
+        }
+    }
+    return count;
+}
+
+// CLT-k (Sections 1 and 3.1): one worker per iteration, the leader, selects the top k of ITS
+// vector (= Algorithm 5 with one layer) and broadcasts the indices; the leaders take turns
+// ("cyclic").  Every worker then contributes its own values at the leader's indices and
+// clears them from its residual.
+int64_t oracle_clt_leader(int64_t iteration, int64_t n_workers) { return iteration % n_workers; }
+
+void oracle_gather_update(float* acc, const int64_t* idx, int64_t count, float* val) {
+    for (int64_t j = 0; j < count; ++j) {
+        val[j] = acc[idx[j]];
+        acc[idx[j]] = 0.0f;
+    }
+}
+
 }  // extern "C"

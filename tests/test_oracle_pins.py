@@ -402,3 +402,63 @@ def test_whole_path_partitions_are_disjoint_and_density_is_kept(wl):
     # per-layer counts
     for l in range(size.size):
         assert int(seen[start[l]:start[l + 1]].sum()) == k_l[l]
+
+
+# ------------------------------------------------------------------------------------------
+# comparison sparsifiers (Section 3): hard threshold, CLT-k
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("kind", ["gauss", "wide_exponent", "few_values", "mostly_zero", "signed_zero", "denormal"])
+def test_threshold_select_equals_numpy_mask(kind):
+    x = W.adversarial_vector(kind, 50_003, seed=21)
+    for lam in (0.0, 1e-30, 0.25, 0.5, 1.0, 3.0, 1e30):
+        val, idx = oracle.threshold_select(x, lam)
+        want = np.nonzero(np.abs(x) > np.float32(lam))[0]       # library routine on finite data
+        assert np.array_equal(idx, want)
+        assert val.tobytes() == x[want].tobytes()
+
+
+def test_threshold_select_hand_cases():
+    x = np.array([0.5, -0.5, 0.25, -0.0, 0.0, np.inf, -np.inf, 1e-45, -3.0], dtype=np.float32)
+    val, idx = oracle.threshold_select(x, 0.5)                    # strict: 0.5 itself is not selected
+    assert idx.tolist() == [5, 6, 8] and val.tolist() == [np.inf, -np.inf, -3.0]
+    val, idx = oracle.threshold_select(x, 0.0)                    # everything but the zeros (the denormal counts)
+    assert idx.tolist() == [0, 1, 2, 5, 6, 7, 8]
+    val, idx = oracle.threshold_select(x, np.inf)
+    assert idx.size == 0
+    y = np.array([1.0, np.nan, 2.0], dtype=np.float32)            # NaN sorts above everything, as in Algorithm 5
+    assert oracle.threshold_select(y, 1e38)[1].tolist() == [1]
+    assert oracle.threshold_select(x, -0.5)[1].tolist() == [5, 6, 8]   # the threshold's sign is ignored
+
+
+def test_threshold_at_the_kth_magnitude_reproduces_topk_when_magnitudes_are_distinct():
+    rng = np.random.default_rng(5)
+    x = np.unique(np.abs(rng.standard_normal(30_000).astype(np.float32)))[:20_001].copy()   # distinct magnitudes
+    rng.shuffle(x)
+    x *= rng.choice(np.array([-1.0, 1.0], dtype=np.float32), size=x.size)
+    mags = np.sort(np.abs(x))[::-1]
+    assert np.unique(mags).size == mags.size == 20_001
+    for k in (1, 17, 2000, 20_000):
+        lam = float(mags[k])                                        # the (k+1)-th largest magnitude
+        val, idx = oracle.threshold_select(x, lam)
+        tv, ti = oracle.topk(x, k)
+        assert np.array_equal(idx, ti) and val.tobytes() == tv.tobytes()
+
+
+def test_clt_leader_cycles_and_gather_update():
+    assert [oracle.clt_leader(t, 4) for t in range(9)] == [0, 1, 2, 3, 0, 1, 2, 3, 0]
+    assert oracle.clt_leader(7, 1) == 0
+    rng = np.random.default_rng(6)
+    x = rng.standard_normal(1000).astype(np.float32)
+    idx = np.sort(rng.choice(1000, size=100, replace=False)).astype(np.int64)
+    y = x.copy()
+    val = oracle.gather_update(y, idx)
+    assert val.tobytes() == x[idx].tobytes()
+    want = x.copy()
+    want[idx] = 0.0
+    assert y.tobytes() == want.tobytes()
+    # a follower's contribution at the leader's indices: leader selects, follower gathers
+    leader_vec = rng.standard_normal(1000).astype(np.float32)
+    _, lidx = oracle.topk(leader_vec, 10)
+    f = x.copy()
+    fv = oracle.gather_update(f, lidx)
+    assert np.array_equal(fv, x[lidx]) and not f[lidx].any() and np.count_nonzero(f != x) == np.count_nonzero(x[lidx])

@@ -307,6 +307,36 @@ DEFT_API deft_status deft_select_update_all(float* acc_d, int64_t n_g, const voi
                                             size_t ws_bytes, void* stream);
 
 /*
+ * Comparison sparsifiers of Section 3 (not part of DEFT; they reuse its selection kernel).
+ *
+ * Hard-threshold sparsifier (Section 3.2): selects every entry of acc_d[0, n) whose magnitude is
+ * larger than |threshold| (strict; magnitudes compare as in Algorithm 5's selection, so a NaN
+ * entry is larger than any threshold), one read of the vector.  Writes the first out_cap of
+ * them in ascending index to val_d / idx_d (DEVICE; may be NULL when out_cap = 0) and the
+ * total number to *count_d (DEVICE int64; may exceed out_cap).  zero_selected != 0 also clears
+ * every selected entry in acc_d (the residual update), whether or not it fitted in out_cap.
+ * ws_d: deft_workspace_bytes(n, 1).  Errors: INVALID_ARG (NaN threshold, NULL, misaligned, n
+ * beyond DEFT_MAX_LAYER_ELEMS), CAPACITY (workspace), CUDA.
+ */
+DEFT_API deft_status deft_threshold_select(float* acc_d, int64_t n, float threshold, int32_t zero_selected,
+                                           float* val_d, int64_t* idx_d, int64_t out_cap, int64_t* count_d,
+                                           void* ws_d, size_t ws_bytes, void* stream);
+
+/*
+ * CLT-k (Sections 1, 3.1): the worker that selects in `iteration` — the leaders take turns —
+ * or -1 for invalid arguments.  The leader's selection is deft_topk_baseline on its own vector.
+ */
+DEFT_API int32_t deft_clt_leader(int64_t iteration, int32_t N);
+
+/*
+ * CLT-k follower step: val_d[i] = acc_d[idx_d[i]], then acc_d[idx_d[i]] = +0, for the `count`
+ * indices the leader broadcast (DEVICE; distinct, each in [0, n_g) — not checked).
+ * Errors: INVALID_ARG, CUDA.
+ */
+DEFT_API deft_status deft_gather_update(float* acc_d, int64_t n_g, const int64_t* idx_d, int64_t count,
+                                        float* val_d, void* stream);
+
+/*
  * Residual update — Algorithm 1 lines 11-12: acc[idx[j]] = +0.0f for j < count; the
  * buffer is then the next step's local error.  Indices must be distinct and < n_g.
  *   idx_d[count] DEVICE.  count may be 0.  Errors: INVALID_ARG, CUDA.

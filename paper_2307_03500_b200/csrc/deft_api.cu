@@ -145,14 +145,21 @@ deft_status upload_plan(const void* plan_h, void* plan_d, void* ws_d, size_t ws_
     return DEFT_OK;
 }
 
+// Hard-threshold mode of the selection kernel (one layer, threshold given).
+struct FixedThreshold {
+    bool on = false;
+    uint32_t key = 0;                       // magnitude key of the threshold
+    unsigned long long* count_d = nullptr;  // receives the number of entries above it
+};
+
 deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan_d, int32_t rank,
                         float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
-                        cudaStream_t stream, bool zero_selected = false) {
+                        cudaStream_t stream, bool zero_selected = false, FixedThreshold fixed = FixedThreshold()) {
     const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
     if (rank < 0 || rank > hdr->N) return DEFT_ERR_INVALID_ARG;   // rank N = all ranks' layers as one list
     const RankInfo& R = plan_ranks(plan_h)[rank];
     if (R.n_my == 0) return DEFT_OK;
-    if (out_cap < R.k) return DEFT_ERR_CAPACITY;
+    if (!fixed.on && out_cap < R.k) return DEFT_ERR_CAPACITY;
     const WsLayout w = ws_layout(hdr->total_elems, hdr->L, hdr->total_tiles);
     if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
     char* ws = static_cast<char*>(ws_d);
@@ -171,6 +178,10 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.val = val_d;
     p.idx = idx_d;
     p.timing = g_select_timing;
+    p.fixed_thr = fixed.on ? 1 : 0;
+    p.thr_key = fixed.key;
+    p.out_cap = out_cap;
+    p.count_out = fixed.count_d;
     // one CTA per SM at most (co-resident by construction); fewer when the rank is small
     const int sms = sm_count();
     int want = (R.tiles + 1) / 2;
@@ -431,6 +442,48 @@ deft_status deft_topk_baseline(const float* acc_d, int64_t n, int64_t k, float* 
     if (!aligned16(acc_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
     std::vector<LayerItem> items(1, LayerItem{0, n, k, 0});
     return select_once(acc_d, items, val_d, idx_d, k, ws_d, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+deft_status deft_threshold_select(float* acc_d, int64_t n, float threshold, int32_t zero_selected, float* val_d,
+                                  int64_t* idx_d, int64_t out_cap, int64_t* count_d, void* ws_d, size_t ws_bytes,
+                                  void* stream) {
+    if (!acc_d || !count_d || !ws_d || n < 1 || n > DEFT_MAX_LAYER_ELEMS || out_cap < 0 ||
+        (out_cap > 0 && (!val_d || !idx_d)) || threshold != threshold)
+        return DEFT_ERR_INVALID_ARG;
+    if (!aligned16(acc_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<std::vector<LayerItem>> ranks(1, std::vector<LayerItem>(1, LayerItem{0, n, 1, 0}));
+    std::vector<char> blob(plan_bytes(1, 1));
+    deft_status s = fill_plan(blob.data(), blob.size(), 1, 0, ranks);
+    if (s != DEFT_OK) return s;
+    const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(blob.data());
+    const WsLayout w = ws_layout(hdr->total_elems, hdr->L, hdr->total_tiles);
+    if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
+    void* plan_d = static_cast<char*>(ws_d) + w.plan;
+    s = upload_plan(blob.data(), plan_d, ws_d, ws_bytes, st);
+    if (s != DEFT_OK) return s;
+    DEFT_CUDA_TRY(cudaMemsetAsync(count_d, 0, sizeof(int64_t), st));
+    FixedThreshold fixed;
+    fixed.on = true;
+    uint32_t bits;
+    std::memcpy(&bits, &threshold, 4);
+    fixed.key = bits & 0x7fffffffu;
+    fixed.count_d = reinterpret_cast<unsigned long long*>(count_d);
+    return select_rank(acc_d, blob.data(), plan_d, 0, val_d, idx_d, out_cap, ws_d, ws_bytes, st, zero_selected != 0,
+                       fixed);
+}
+
+int32_t deft_clt_leader(int64_t iteration, int32_t N) {
+    if (N < 1 || iteration < 0) return -1;
+    return (int32_t)(iteration % N);
+}
+
+deft_status deft_gather_update(float* acc_d, int64_t n_g, const int64_t* idx_d, int64_t count, float* val_d,
+                               void* stream) {
+    if (count < 0 || n_g < 1 || count > n_g) return DEFT_ERR_INVALID_ARG;
+    if (count == 0) return DEFT_OK;
+    if (!acc_d || !idx_d || !val_d) return DEFT_ERR_INVALID_ARG;
+    return launch_gather_update(acc_d, idx_d, count, val_d, static_cast<cudaStream_t>(stream));
 }
 
 deft_status deft_residual_update(float* acc_d, int64_t n_g, const int64_t* idx_d, int64_t count,

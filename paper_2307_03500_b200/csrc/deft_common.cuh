@@ -207,6 +207,11 @@ struct SelParams {
     uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output
     int64_t* idx;
+    // hard-threshold mode (one layer, no search): every entry whose key exceeds thr_key is selected
+    int32_t fixed_thr;               // 1: hard-threshold mode
+    uint32_t thr_key;                // magnitude key of the threshold
+    int64_t out_cap;                 // entries val / idx can take (positions beyond it are not written)
+    unsigned long long* count_out;   // hard-threshold mode: number of entries above the threshold (zeroed before launch)
     unsigned long long* timing;      // optional: 1024 words of phase stamps and per-CTA counters; NULL = off
 };
 
@@ -230,5 +235,7 @@ deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t 
 deft_status launch_select(const SelParams& p, cudaStream_t stream);
 deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t count,
                                    cudaStream_t stream);
+deft_status launch_gather_update(float* acc_d, const int64_t* idx_d, int64_t count, float* val_d,
+                                 cudaStream_t stream);
 
 }  // namespace deft

@@ -68,7 +68,7 @@ enum MiscOff : int {   // word offsets inside the misc area
     kMOut3 = 64,       // 4: result of block_scan_select
     kMLast = 72,       // kSlots: this CTA flushed the layer's last tiles
     kMCursor = 80,     // 1: staged entries of this CTA
-    kMTab = 96,        // kBSlots: per-slot b1 in step B
+    kMTab = 96,        // 2 * kBSlots: per-slot staging threshold, then per-slot b1 in step B
     kMWarpCnt = 128,   // 32: per-warp packed counts (direct layers)
 };
 static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4 && kSlots <= 8 && kBSlots <= 32, "misc area");
@@ -401,13 +401,12 @@ __device__ __noinline__ uint2 filter_marked(const uint32_t* __restrict__ tile, u
 
 // Staging pass over one tile: marks the entries with bucket >= b1; tiles without any cost a
 // compare per element.
-__device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t b1,
-                                             uint32_t* h2, const Stage& st, uint32_t ytag, uint32_t* cursor,
-                                             uint32_t* wbase, int lane) {
+__device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t thr,
+                                             uint32_t b1, uint32_t* h2, const Stage& st, uint32_t ytag,
+                                             uint32_t* cursor, uint32_t* wbase, int lane) {
     TileRegs t;
     uint32_t vm[2];
-    load_tile(acc, ts, lane, t, vm);
-    const uint32_t thr = b1 << kShift1;          // key >= thr  <=>  bucket >= b1
+    load_tile(acc, ts, lane, t, vm);             // entries with key >= thr are staged
     uint32_t keep[2] = {0u, 0u};                 // bit (4*(i%8) + c) of keep[i/8]
 #pragma unroll
     for (int i = 0; i < 16; ++i) keep[i >> 3] |= keep4(t.v[i], thr) << (4 * (i & 7));
@@ -568,7 +567,7 @@ __device__ __forceinline__ uint32_t own_tiles(const SelParams& p, const CtaRange
 }
 
 __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
-    return p.desc[j].end - p.desc[j].start <= kDirectElems;
+    return !p.fixed_thr && p.desc[j].end - p.desc[j].start <= kDirectElems;
 }
 
 // Fills the table of the CTA's streamed layers; returns how many there are (at most
@@ -676,8 +675,15 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
         const int ns = nl - c0 < kBSlots ? nl - c0 : kBSlots;
         if ((int)threadIdx.x < ns) {
             const LayerState* ls = p.state + lt->lid[c0 + threadIdx.x];
-            misc[kMTab + threadIdx.x] = __ldcg(&ls->b1);
-            lt->v1[c0 + threadIdx.x] = lt->k[c0 + threadIdx.x] - __ldcg(&ls->above1);   // krem1
+            if (p.fixed_thr) {
+                misc[kMTab + threadIdx.x] = p.thr_key + 1u;     // key >= thr_key + 1  <=>  key > thr_key
+                misc[kMTab + kBSlots + threadIdx.x] = 0xffffffffu;   // no bucket feeds the level-2 histogram
+            } else {
+                const uint32_t b1 = __ldcg(&ls->b1);
+                misc[kMTab + threadIdx.x] = b1 << kShift1;      // key >= thr  <=>  bucket >= b1
+                misc[kMTab + kBSlots + threadIdx.x] = b1;
+                lt->v1[c0 + threadIdx.x] = lt->k[c0 + threadIdx.x] - __ldcg(&ls->above1);   // krem1
+            }
         }
         for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) hist2s[i] = 0;
         __syncthreads();
@@ -690,7 +696,8 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
             const int cl = tile_layer(lt, c0 + ns, q, c);
             if (cl < 0) continue;
             const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-            const uint2 fn = filter_tile(p.acc, ts, misc[kMTab + cl - c0], hist2s + (cl - c0) * kBins2, st,
+            const uint2 fn = filter_tile(p.acc, ts, misc[kMTab + cl - c0], misc[kMTab + kBSlots + cl - c0],
+                                         hist2s + (cl - c0) * kBins2, st,
                                          pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
                                          reinterpret_cast<uint32_t*>(smem + kSmWBase) + 16 * warp, lane);
             if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
@@ -752,7 +759,14 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
     const uint32_t* misc = reinterpret_cast<const uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t total = misc[kMCursor];
-    for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer
+    if (p.fixed_thr) {
+        // the threshold is given: every staged entry is selected, a tile's count is what it staged
+        if (threadIdx.x == 0 && nl > 0) { lt->v0[0] = p.thr_key; lt->v1[0] = 0u; }
+        for (int i = threadIdx.x; i < r.nloc; i += kSelThreads) tt->ge[i] = local_tile(p, r, i) >= 0 ? tt->n[i] : 0u;
+        if (threadIdx.x == 0 && total) atomicAdd(p.count_out, (unsigned long long)total);
+        __syncthreads();
+    }
+    for (int c = warp; c < nl && !p.fixed_thr; c += kSelWarps) {   // one warp per layer
         const uint2 s3 = warp_scan_select(p.hist3 + (size_t)lt->lid[c] * kBins3, kBins3 / 32, lt->v1[c]);
         const uint32_t b3 = s3.x, above3 = s3.y;
         __syncwarp();
@@ -761,14 +775,16 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
             lt->v1[c] = lt->v1[c] - above3;            // need
         }
     }
-    for (int i = threadIdx.x; i < r.nloc; i += kSelThreads) tt->ge[i] = 0;
-    __syncthreads();
-    for_each_staged(st, total, [&](const uint2 ent) {
-        const uint32_t key = key_of(ent.x), T = lt->v0[y_layer(ent.y)];
-        if (key > T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u);
-        else if (key == T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u << 16);
-    });
-    __syncthreads();
+    if (!p.fixed_thr) {
+        for (int i = threadIdx.x; i < r.nloc; i += kSelThreads) tt->ge[i] = 0;
+        __syncthreads();
+        for_each_staged(st, total, [&](const uint2 ent) {
+            const uint32_t key = key_of(ent.x), T = lt->v0[y_layer(ent.y)];
+            if (key > T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u);
+            else if (key == T) atomicAdd(&tt->ge[y_tile(ent.y)], 1u << 16);
+        });
+        __syncthreads();
+    }
     if (r.il) {   // totals per own super-tile, published under the super-tile's id
         for (int m = threadIdx.x; m < r.nloc / kSuper; m += kSelThreads) {
             uint32_t gt = 0, eq = 0;
@@ -791,7 +807,7 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
 
 // Ordered write of one batch of 32 consecutive staged entries (one per lane).  gt_before /
 // eq_before: entries above / equal to the threshold that precede the batch in the layer.
-struct EmitOut { float* val; int64_t* idx; float* acc_rw; };
+struct EmitOut { float* val; int64_t* idx; float* acc_rw; int64_t cap; };
 
 __device__ __forceinline__ void emit_batch(const EmitOut& p, int64_t out_off, int64_t elem0, bool valid,
                                            uint32_t bits, int64_t off, uint32_t T, uint32_t need,
@@ -804,8 +820,10 @@ __device__ __forceinline__ void emit_batch(const EmitOut& p, int64_t out_off, in
     if (gt || (eq && my_eq < need)) {
         // selected entries before me: every larger key, and the first `need` equal ones
         const int64_t pos = out_off + my_gt + (my_eq < need ? my_eq : need);
-        p.val[pos] = __uint_as_float(bits);
-        p.idx[pos] = elem0 + off;
+        if (pos < p.cap) {
+            p.val[pos] = __uint_as_float(bits);
+            p.idx[pos] = elem0 + off;
+        }
         if (p.acc_rw) p.acc_rw[elem0 + off] = 0.0f;
     }
     gt_before += __popc(gt_b);
@@ -862,8 +880,10 @@ __device__ __forceinline__ void emit_small_tile(const EmitOut& out, const Stage&
         if (key > T || (key == T && eq_before < need)) {
             const int64_t pos = out_off + gt_before + (eq_before < need ? eq_before : need);
             const int64_t elem = lo + (int64_t)y_off(ent.y);
-            out.val[pos] = __uint_as_float(ent.x);
-            out.idx[pos] = elem;
+            if (pos < out.cap) {
+                out.val[pos] = __uint_as_float(ent.x);
+                out.idx[pos] = elem;
+            }
             if (out.acc_rw) out.acc_rw[elem] = 0.0f;
         }
         gt_before += key > T;
@@ -917,13 +937,13 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
                 const int q = i < r.nloc ? local_tile(p, r, i) : -1;
                 const uint32_t n = q >= 0 ? tt->n[i] : 0u;
                 if (n != 0 && n <= kThreadEmit)
-                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw}, st, tt->first[i], n, lt->out_off[0],
+                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, st, tt->first[i], n, lt->out_off[0],
                                     (lt->start[0] / kTile + (q - lt->tf[0])) * kTile, T, need,
                                     sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
             }
             __syncthreads();
             const int tend = t0 + kSelThreads < r.nloc ? t0 + kSelThreads : r.nloc;
-            emit_tiles(EmitOut{p.val, p.idx, p.acc_rw}, p.tiles, 1, 0, tt, st.res, st.spill, pref, t0, tend, lt->start[0],
+            emit_tiles(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, p.tiles, 1, 0, tt, st.res, st.spill, pref, t0, tend, lt->start[0],
                        lt->tf[0], lt->out_off[0], T, need);
             __syncthreads();   // pref is rewritten by the next batch
         }
@@ -959,13 +979,13 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             {
                 const uint32_t n = i < tb ? tt->n[i] : 0u;
                 if (n != 0 && n <= kThreadEmit)
-                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw}, st, tt->first[i], n, lt->out_off[c],
+                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, st, tt->first[i], n, lt->out_off[c],
                                     (lt->start[c] / kTile + (r.q0 + i - lt->tf[c])) * kTile, T, need,
                                     base_gt + e_gt, base_eq + e_eq);
             }
             __syncthreads();
             const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
-            emit_tiles(EmitOut{p.val, p.idx, p.acc_rw}, p.tiles, 0, r.q0, tt, st.res, st.spill, pref, t0, tend, lt->start[c],
+            emit_tiles(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, p.tiles, 0, r.q0, tt, st.res, st.spill, pref, t0, tend, lt->start[c],
                        lt->tf[c], lt->out_off[c], T, need);
             base_gt += tot_gt;
             base_eq += tot_eq;
@@ -1059,7 +1079,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
     for (uint32_t fb = f0; fb < f1; fb += 32) {
         const uint32_t f = fb + lane;
         const bool valid = f < f1;
-        emit_batch(EmitOut{p.val, p.idx, p.acc_rw}, out_off, start, valid, valid ? skey[f] : 0u, (int64_t)f, T, need,
+        emit_batch(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, out_off, start, valid, valid ? skey[f] : 0u, (int64_t)f, T, need,
                    gt_before, eq_before, lane);
     }
     __syncthreads();   // shared memory is reused by the next layer
@@ -1103,9 +1123,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     st.res = reinterpret_cast<uint2*>(smem + kSmMain);
     st.spill = spill_base(p, r);
 
-    step_hist1(p, r, lt, nl, smem);
-    stamp(p, 1);
-    grid.sync();
+    if (!p.fixed_thr) {   // uniform over the grid
+        step_hist1(p, r, lt, nl, smem);
+        stamp(p, 1);
+        grid.sync();
+    }
     if (p.weighted) {   // from here on: contiguous runs of equal estimated cost
         r = weighted_range(p, reinterpret_cast<uint32_t*>(smem + kSmMain), reinterpret_cast<int*>(smem + kSmTf),
                            misc + kMScratch);
@@ -1125,9 +1147,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
         p.timing[16 + 480 + blockIdx.x] = misc[kMCursor + 2];   // profiling build: cycles in filter_marked
     }
     stamp(p, 2);
-    grid.sync();
-    step_hist3(p, lt, nl, st, smem);
-    stamp(p, 3);
+    if (!p.fixed_thr) {
+        grid.sync();
+        step_hist3(p, lt, nl, st, smem);
+        stamp(p, 3);
+    }
     grid.sync();
     step_count(p, r, lt, nl, tt, st, smem);
     stamp(p, 4);
@@ -1151,6 +1175,17 @@ __global__ void k_zero_at(float* __restrict__ acc, const int64_t* __restrict__ i
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
          i += (int64_t)gridDim.x * blockDim.x)
         acc[idx[i]] = 0.0f;
+}
+
+// CLT-k follower: own values at the leader's indices, then cleared.
+__global__ void k_gather_zero(float* __restrict__ acc, const int64_t* __restrict__ idx, int64_t count,
+                              float* __restrict__ val) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t j = idx[i];
+        val[i] = acc[j];
+        acc[j] = 0.0f;
+    }
 }
 
 }  // namespace
@@ -1177,6 +1212,16 @@ deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t c
     const int64_t want = (count + 255) / 256;
     const int64_t cap = (int64_t)sm_count() * 16;
     k_zero_at<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(acc_d, idx_d, count);
+    DEFT_CUDA_TRY(cudaGetLastError());
+    return DEFT_OK;
+}
+
+deft_status launch_gather_update(float* acc_d, const int64_t* idx_d, int64_t count, float* val_d,
+                                 cudaStream_t stream) {
+    if (count == 0) return DEFT_OK;
+    const int64_t want = (count + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    k_gather_zero<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(acc_d, idx_d, count, val_d);
     DEFT_CUDA_TRY(cudaGetLastError());
     return DEFT_OK;
 }

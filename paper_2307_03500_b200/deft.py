@@ -80,6 +80,12 @@ def lib() -> ctypes.CDLL:
         L.deft_plan_rank_info.argtypes = [vp, i32, vp, vp, vp, vp]
         L.deft_plan_rank_table.restype = i32
         L.deft_plan_rank_table.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.deft_threshold_select.restype = i32
+        L.deft_threshold_select.argtypes = [vp, i64, ctypes.c_float, i32, vp, vp, i64, vp, vp, sz, vp]
+        L.deft_clt_leader.restype = i32
+        L.deft_clt_leader.argtypes = [i64, i32]
+        L.deft_gather_update.restype = i32
+        L.deft_gather_update.argtypes = [vp, i64, vp, i64, vp, vp]
         L.deft_plan_step.restype = i32
         L.deft_plan_step.argtypes = [vp, vp, i32, i32, i64, i32, i64, vp, vp, vp, vp, vp, sz, vp, vp, sz, vp]
         L.deft_plan_upload.restype = i32
@@ -382,6 +388,36 @@ def deft_select_update_all(acc, plan_h: np.ndarray, plan_d, val_d, idx_d, ws, st
                                         _dp(val_d, torch.float32), _dp(idx_d, torch.int64),
                                         min(val_d.numel(), idx_d.numel()), _dp(ws), ws.numel() * ws.element_size(),
                                         _stream(stream)))
+
+
+def deft_threshold_select(acc, threshold: float, val_d, idx_d, count_d, ws, zero_selected: bool = False,
+                          stream=None) -> None:
+    """Hard-threshold sparsifier (Section 3.2): entries with magnitude > threshold, ascending index.
+    count_d: CUDA int64 tensor of one element that receives the total count."""
+    import torch
+    cap = 0 if val_d is None or idx_d is None else min(val_d.numel(), idx_d.numel())
+    _check("deft_threshold_select",
+           lib().deft_threshold_select(_dp(acc, torch.float32), acc.numel(), float(threshold), int(bool(zero_selected)),
+                                       _dp(val_d, torch.float32) if cap else None,
+                                       _dp(idx_d, torch.int64) if cap else None, cap, _dp(count_d, torch.int64),
+                                       _dp(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_clt_leader(iteration: int, n_workers: int) -> int:
+    r = int(lib().deft_clt_leader(int(iteration), int(n_workers)))
+    if r < 0:
+        raise DeftError("deft_clt_leader", ERR_INVALID_ARG)
+    return r
+
+
+def deft_gather_update(acc, idx_d, count: int, val_d, stream=None) -> None:
+    """CLT-k follower: val_d[i] = acc[idx_d[i]], then that entry is cleared."""
+    import torch
+    if count > idx_d.numel() or count > val_d.numel():
+        raise ValueError("count exceeds idx_d / val_d")
+    _check("deft_gather_update",
+           lib().deft_gather_update(_dp(acc, torch.float32), acc.numel(), _dp(idx_d, torch.int64), int(count),
+                                    _dp(val_d, torch.float32), _stream(stream)))
 
 
 def deft_residual_update(acc, idx_d, count: int, stream=None) -> None:

@@ -388,6 +388,25 @@ def run_ours(args):
             tk.append(a.elapsed_time(b))
     t_topk = float(np.median(tk))
 
+    # the comparison sparsifiers of Section 3 on the same vector: hard threshold at the magnitude of the
+    # Top-k result's smallest entry (so that it selects k - 1 entries), and the CLT-k follower step
+    lam = float(tk_val.abs().min().item())
+    cnt_d = torch.zeros(1, dtype=torch.int64, device=dev)
+    th, ga = [], []
+    for i in range(3 + 10):
+        a, b, c = ev(), ev(), ev()
+        a.record(stream)
+        deft.deft_threshold_select(e, lam, tk_val, tk_idx, cnt_d, ds.ws)
+        b.record(stream)
+        deft.deft_gather_update(g, tk_idx, k - 1, tk_val)      # a follower's values at broadcast indices
+        c.record(stream)
+        stream.synchronize()
+        if i >= 3:
+            th.append(a.elapsed_time(b))
+            ga.append(b.elapsed_time(c))
+    t_thr, t_gather, n_thr = float(np.median(th)), float(np.median(ga)), int(cnt_d.item())
+    g.copy_(g_host)                                             # the gather cleared entries of g
+
     # end to end through the public call with HOST buffers: gradient from pinned host memory,
     # selected (value, index) pairs and norms back to the host, every step
     out_val_h = torch.empty(ds.val_d.numel(), dtype=torch.float32).pin_memory()
@@ -491,6 +510,11 @@ def run_ours(args):
                               "speedup_vs_slowest_rank": t_topk / float(sel_med.max()),
                               "model_f_n": n_g * lnk / cost_max if cost_max > 0 else None,
                               "model_f_trivial_n": N * lnk / math.log(k / N) if k > N else None},
+            "comparison_selectors": {
+                "hard_threshold": {"ms": t_thr, "selected": n_thr, "bytes_per_elem": 4, "bytes_per_selected": 12,
+                                   "gbs": (4.0 * n_g + 12.0 * n_thr) / (t_thr * 1e-3) / 1e9,
+                                   "frac": (4.0 * n_g + 12.0 * n_thr) / (t_thr * 1e-3) / 1e9 / peak},
+                "clt_k": {"leader_select_ms": t_topk, "follower_gather_ms": t_gather, "entries": k - 1}},
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))

@@ -108,6 +108,15 @@ def partition(layer_size, k_l, n_workers):
     return bins, load
 
 
+def partition_by_size(layer_size, n_workers):
+    """Algorithm 4's packing with cost = layer size (load-model ablation). Returns (bins, loads)."""
+    sz = np.ascontiguousarray(layer_size, dtype=np.int64)
+    bins = np.zeros(sz.size, dtype=np.int32)
+    load = np.zeros(int(n_workers), dtype=np.float64)
+    _load().oracle_partition_by_size(_p(sz), _i64(sz.size), _i64(n_workers), _p(bins), _p(load))
+    return bins, load
+
+
 def rank_bin(iteration, rank, n_workers):
     """Algorithm 4 lines 1-2."""
     return int(_load().oracle_rank_bin(_i64(iteration), _i64(rank), _i64(n_workers)))

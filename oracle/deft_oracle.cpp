@@ -220,6 +220,28 @@ void oracle_partition(const int64_t* layer_size, const int64_t* k_l, int64_t L, 
     }
 }
 
+// Variant of Algorithm 4 for hardware whose selection time follows the bytes a worker scans
+// rather than size * ln(k) (a linear-time selection): the same greedy packing with
+// cost_l = size_l.  Not in the paper; an ablation of the load model of Eq. 3.
+void oracle_partition_by_size(const int64_t* layer_size, int64_t L, int64_t n_workers,
+                              int32_t* bin_of_layer, double* size_bin /* n_workers */) {
+    std::vector<double> cost(L);
+    for (int64_t i = 0; i < L; ++i) cost[i] = (double)layer_size[i];
+    for (int64_t b = 0; b < n_workers; ++b) size_bin[b] = 0.0;
+    for (int64_t it = 0; it < L; ++it) {
+        int64_t idx_max = 0;
+        for (int64_t i = 1; i < L; ++i)
+            if (cost[i] > cost[idx_max]) idx_max = i;
+        const double val_max = cost[idx_max];
+        int64_t bin_min = 0;
+        for (int64_t b = 1; b < n_workers; ++b)
+            if (size_bin[b] < size_bin[bin_min]) bin_min = b;
+        bin_of_layer[idx_max] = (int32_t)bin_min;
+        size_bin[bin_min] = size_bin[bin_min] + val_max;
+        cost[idx_max] = -1.0;
+    }
+}
+
 // Algorithm 4, lines 1-2: the bin a rank reads in a given iteration.
 int64_t oracle_rank_bin(int64_t iteration, int64_t rank, int64_t n_workers) {
     const int64_t cycle = iteration % n_workers;

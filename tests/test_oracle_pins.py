@@ -274,6 +274,28 @@ def test_partition_equal_costs_divide_evenly():
     assert np.allclose(load, 30 * math.log(4))
 
 
+def test_partition_by_size_hand_case_and_bounds():
+    # sizes 5,4,3,3,3 on two bins, largest first into the lighter bin (first bin on ties):
+    # 5->b0, 4->b1, 3->b1 (4<5), 3->b0 (5<7), 3->b1 (7<8): loads 8 | 10
+    bins, load = oracle.partition_by_size([5, 4, 3, 3, 3], 2)
+    assert bins.tolist() == [0, 1, 1, 0, 1] and load.tolist() == [8.0, 10.0]
+    rng = np.random.default_rng(23)
+    for trial in range(40):
+        L = int(rng.integers(1, 10))
+        N = int(rng.integers(1, 5))
+        sizes = rng.integers(1, 1000, size=L)
+        bins, load = oracle.partition_by_size(sizes, N)
+        for b in range(N):
+            assert load[b] == float(sizes[bins == b].sum())             # integer-valued doubles: exact
+        opt = oracle.partition_optimum(sizes.astype(np.float64), N)
+        assert opt - 1e-9 <= load.max() <= (4.0 / 3.0 - 1.0 / (3.0 * N)) * opt + 1e-9
+    # with equal k_l the two load models rank the layers alike and pack identically
+    sizes = rng.integers(100, 10_000, size=25)
+    b_eq3, _ = oracle.partition(sizes, np.full(25, 7), 4)
+    b_size, _ = oracle.partition_by_size(sizes, 4)
+    assert b_eq3.tolist() == b_size.tolist()
+
+
 # --------------------------------------------------------------------------
 # Algorithm 5 / Top-k
 # --------------------------------------------------------------------------

@@ -374,6 +374,20 @@ def run_ours(args):
     sel_med = np.median(t_sel, axis=0)
     worker_ms = float(np.median(t_acc) + np.median(t_host) + np.max(sel_med))
 
+    # load-model ablation: the same per-worker passes with layers packed by size instead of Eq. 3
+    ds.cost_model = deft.COST_SIZE
+    size_recs = []
+    for it in range(max(3, min(args.steps, 20))):
+        tri = [(ev(), ev(), ev()) for _ in range(N)]
+        for t3 in tri:
+            for x in t3:
+                x.record(stream)
+        one_step(args.warmup + 2 * args.steps + it, size_recs, g, tri)
+    stream.synchronize()
+    ds.cost_model = deft.COST_EQ3
+    t_sel_size = np.median(np.array([[a.elapsed_time(b) for (a, b, c) in r["ranks"]] for r in size_recs]), axis=0)
+    plan_s = size_recs[-1]["plan"]
+
     # full-vector Top-k on the same GPU (comparison sparsifier), timed alone
     tk_val = torch.empty(k, dtype=torch.float32, device=dev)
     tk_idx = torch.empty(k, dtype=torch.int64, device=dev)
@@ -510,6 +524,12 @@ def run_ours(args):
                               "speedup_vs_slowest_rank": t_topk / float(sel_med.max()),
                               "model_f_n": n_g * lnk / cost_max if cost_max > 0 else None,
                               "model_f_trivial_n": N * lnk / math.log(k / N) if k > N else None},
+            "load_model_ablation": {
+                "eq3": {"select_ms_max": float(sel_med.max()), "select_ms_mean": float(sel_med[busy].mean()),
+                        "rank_elems_max_over_mean": float(plan_w.rank_elems.max() / plan_w.rank_elems.mean())},
+                "size": {"select_ms_max": float(t_sel_size.max()), "select_ms_mean": float(t_sel_size.mean()),
+                         "rank_elems_max_over_mean": float(plan_s.rank_elems.max() / plan_s.rank_elems.mean()),
+                         "rank_k_min": int(plan_s.rank_k.min()), "rank_k_max": int(plan_s.rank_k.max())}},
             "comparison_selectors": {
                 "hard_threshold": {"ms": t_thr, "selected": n_thr, "bytes_per_elem": 4, "bytes_per_selected": 12,
                                    "gbs": (4.0 * n_g + 12.0 * n_thr) / (t_thr * 1e-3) / 1e9,

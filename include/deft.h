@@ -50,6 +50,10 @@ typedef int32_t deft_status;
 #define DEFT_MODE_PAPER 0  /* Algorithm 3 exactly as listed                                      */
 #define DEFT_MODE_EXACT 1  /* Algorithm 3 followed by an integer repair so that sum k_l == k     */
 
+/* Load model of the bin packing (Algorithm 4). */
+#define DEFT_COST_EQ3  0   /* cost_l = size_l * ln(k_l): Eq. 3                                     */
+#define DEFT_COST_SIZE 1   /* cost_l = size_l: the bytes a worker scans (no counterpart in the paper) */
+
 /* Largest layer (and largest n for deft_topk_baseline) the selection kernels accept. */
 #define DEFT_MAX_LAYER_ELEMS 2147483647LL
 
@@ -121,6 +125,16 @@ DEFT_API deft_status deft_allocate_k(const double* norms_h, const int64_t* layer
  */
 DEFT_API deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L,
                            int32_t N, int32_t* bin_of_layer_h, double* bin_load_h);
+
+/*
+ * Algorithm 4's packing under a chosen load model.  DEFT_COST_EQ3 is deft_partition().
+ * DEFT_COST_SIZE packs by layer size alone: the paper's model (Eq. 3) prices a sort-based
+ * selection; the selection kernel here is linear in the elements a worker scans, so its time
+ * follows bytes, and Eq. 3's cost-0 layers (k_l = 1) pile up in one bin.  k_l_h may be NULL for
+ * DEFT_COST_SIZE.  Outputs and errors as deft_partition(); INVALID_ARG for an unknown model.
+ */
+DEFT_API deft_status deft_partition_model(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L, int32_t N,
+                                          int32_t cost_model, int32_t* bin_of_layer_h, double* bin_load_h);
 
 /*
  * Which bin a rank reads in a given iteration — Algorithm 4, lines 1-2:
@@ -214,8 +228,8 @@ DEFT_API deft_status deft_layer_norms_static(float* resid_acc_d, const float* gr
 
 /*
  * One step's host work in one call: Algorithm 3 (deft_allocate_k on the layer sizes implied by
- * layer_start_h), Algorithm 4 (deft_partition), deft_plan_build and deft_plan_upload, in that
- * order, with the same results as the four separate calls.  norms_h: HOST [L], this step's
+ * layer_start_h), Algorithm 4 (deft_partition_model with cost_model), deft_plan_build and
+ * deft_plan_upload, in that order, with the same results as the four separate calls.  norms_h: HOST [L], this step's
  * norms.  Outputs (HOST): k_l_h [L], *sum_k_out (may be NULL), bin_of_layer_h [L],
  * bin_load_h [N] (may be NULL), plan_h (plan_bytes_cap >= deft_plan_bytes(L, N); pinned
  * memory lets the upload overlap).  plan_d / ws_d: DEVICE, as for deft_plan_upload.
@@ -223,8 +237,8 @@ DEFT_API deft_status deft_layer_norms_static(float* resid_acc_d, const float* gr
  * built and uploaded all the same); errors as the four calls.
  */
 DEFT_API deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
-                                    int64_t k, int32_t mode, int64_t iteration, int64_t* k_l_h,
-                                    int64_t* sum_k_out, int32_t* bin_of_layer_h, double* bin_load_h,
+                                    int64_t k, int32_t mode, int32_t cost_model, int64_t iteration,
+                                    int64_t* k_l_h, int64_t* sum_k_out, int32_t* bin_of_layer_h, double* bin_load_h,
                                     void* plan_h, size_t plan_bytes_cap, void* plan_d, void* ws_d,
                                     size_t ws_bytes, void* stream);
 

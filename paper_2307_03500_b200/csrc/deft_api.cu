@@ -309,7 +309,8 @@ deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
 }
 
 deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
-                           int64_t k, int32_t mode, int64_t iteration, int64_t* k_l_h, int64_t* sum_k_out,
+                           int64_t k, int32_t mode, int32_t cost_model, int64_t iteration, int64_t* k_l_h,
+                           int64_t* sum_k_out,
                            int32_t* bin_of_layer_h, double* bin_load_h, void* plan_h, size_t plan_bytes_cap,
                            void* plan_d, void* ws_d, size_t ws_bytes, void* stream) {
     if (!norms_h || !layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || !plan_d || !ws_d || L < 1)
@@ -318,7 +319,7 @@ deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, 
     for (int32_t l = 0; l < L; ++l) size[l] = layer_start_h[l + 1] - layer_start_h[l];
     const deft_status sa = deft_allocate_k(norms_h, size.data(), L, k, mode, k_l_h, sum_k_out);
     if (sa < 0) return sa;
-    deft_status s = deft_partition(size.data(), k_l_h, L, N, bin_of_layer_h, bin_load_h);
+    deft_status s = deft_partition_model(size.data(), k_l_h, L, N, cost_model, bin_of_layer_h, bin_load_h);
     if (s != DEFT_OK) return s;
     s = deft_plan_build(layer_start_h, k_l_h, bin_of_layer_h, L, N, iteration, plan_h, plan_bytes_cap);
     if (s != DEFT_OK) return s;

@@ -144,15 +144,20 @@ deft_status deft_allocate_k(const double* norms_h, const int64_t* layer_size_h, 
     return (sum == k) ? DEFT_OK : DEFT_WARN_K_INEXACT;
 }
 
-// Algorithm 4 (packing part) with the load model of Eq. 3.
-deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L,
-                           int32_t N, int32_t* bin_of_layer_h, double* bin_load_h) {
-    if (!layer_size_h || !k_l_h || !bin_of_layer_h || L < 1 || N < 1) return DEFT_ERR_INVALID_ARG;
+// Algorithm 4 (packing part).  cost_model: DEFT_COST_EQ3 = size * ln(k) (Eq. 3),
+// DEFT_COST_SIZE = size (the bytes a worker scans).
+deft_status deft_partition_model(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L, int32_t N,
+                                 int32_t cost_model, int32_t* bin_of_layer_h, double* bin_load_h) {
+    if (!layer_size_h || !bin_of_layer_h || L < 1 || N < 1 ||
+        (cost_model != DEFT_COST_EQ3 && cost_model != DEFT_COST_SIZE) || (cost_model == DEFT_COST_EQ3 && !k_l_h))
+        return DEFT_ERR_INVALID_ARG;
     for (int32_t l = 0; l < L; ++l)
-        if (layer_size_h[l] < 1 || k_l_h[l] < 1) return DEFT_ERR_INVALID_ARG;
+        if (layer_size_h[l] < 1 || (cost_model == DEFT_COST_EQ3 && k_l_h[l] < 1)) return DEFT_ERR_INVALID_ARG;
 
     std::vector<double> c(L);
-    for (int32_t l = 0; l < L; ++l) c[l] = (double)layer_size_h[l] * std::log((double)k_l_h[l]);
+    for (int32_t l = 0; l < L; ++l)
+        c[l] = cost_model == DEFT_COST_EQ3 ? (double)layer_size_h[l] * std::log((double)k_l_h[l])
+                                           : (double)layer_size_h[l];
     // "largest remaining cost, lowest id on ties" L times = one stable pass over the layers
     // sorted by descending cost; "smallest load, lowest id on ties" = a min-heap on (load, bin).
     // Each bin receives its costs in the same order as in the listing, so the fp64 sums are the same.
@@ -174,6 +179,13 @@ deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, in
     if (bin_load_h)
         for (int32_t b = 0; b < N; ++b) bin_load_h[b] = load[b];
     return DEFT_OK;
+}
+
+// Algorithm 4 (packing part) with the load model of Eq. 3.
+deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, int32_t L,
+                           int32_t N, int32_t* bin_of_layer_h, double* bin_load_h) {
+    if (!k_l_h) return DEFT_ERR_INVALID_ARG;
+    return deft_partition_model(layer_size_h, k_l_h, L, N, DEFT_COST_EQ3, bin_of_layer_h, bin_load_h);
 }
 
 int32_t deft_rank_bin(int64_t iteration, int32_t rank, int32_t N) {

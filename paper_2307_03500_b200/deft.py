@@ -87,7 +87,9 @@ def lib() -> ctypes.CDLL:
         L.deft_gather_update.restype = i32
         L.deft_gather_update.argtypes = [vp, i64, vp, i64, vp, vp]
         L.deft_plan_step.restype = i32
-        L.deft_plan_step.argtypes = [vp, vp, i32, i32, i64, i32, i64, vp, vp, vp, vp, vp, sz, vp, vp, sz, vp]
+        L.deft_plan_step.argtypes = [vp, vp, i32, i32, i64, i32, i32, i64, vp, vp, vp, vp, vp, sz, vp, vp, sz, vp]
+        L.deft_partition_model.restype = i32
+        L.deft_partition_model.argtypes = [vp, vp, i32, i32, i32, vp, vp]
         L.deft_plan_upload.restype = i32
         L.deft_plan_upload.argtypes = [vp, vp, vp, sz, vp]
         L.deft_select_planned.restype = i32
@@ -174,6 +176,23 @@ def deft_allocate_k(norms, layer_size, k: int, mode: int = MODE_EXACT) -> Tuple[
                 lib().deft_allocate_k(_hp(nr), _hp(sz), sz.size, int(k), int(mode), _hp(k_l), ctypes.byref(s)),
                 allow_warn=True)
     return k_l, int(s.value), st
+
+
+COST_EQ3 = 0
+COST_SIZE = 1
+
+
+def deft_partition_model(layer_size, k_l, n_workers: int, cost_model: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 4's packing under a load model (COST_EQ3 / COST_SIZE) -> (bins int32[L], loads float64[N])."""
+    sz = _np(layer_size, np.int64)
+    kl = None if k_l is None else _np(k_l, np.int64)
+    if kl is not None and kl.size != sz.size:
+        raise ValueError("k_l and layer_size differ in length")
+    bins = np.zeros(sz.size, dtype=np.int32)
+    load = np.zeros(int(n_workers), dtype=np.float64)
+    _check("deft_partition_model", lib().deft_partition_model(_hp(sz), _hp(kl), sz.size, int(n_workers),
+                                                              int(cost_model), _hp(bins), _hp(load)))
+    return bins, load
 
 
 def deft_partition(layer_size, k_l, n_workers: int) -> Tuple[np.ndarray, np.ndarray]:
@@ -323,7 +342,7 @@ def deft_plan_upload(plan_h: np.ndarray, plan_d, ws, stream=None) -> None:
 
 
 def deft_plan_step(norms, layer_start_h, n_workers: int, k: int, mode: int, iteration: int, plan_h: np.ndarray,
-                   plan_d, ws, stream=None):
+                   plan_d, ws, stream=None, cost_model: int = 0):
     """Algorithm 3 + Algorithm 4 + plan build + plan upload in one call.
     Returns (k_l int64[L], sum_k, bin_of_layer int32[L], bin_load float64[N], status)."""
     nr = _np(norms, np.float64)
@@ -339,7 +358,8 @@ def deft_plan_step(norms, layer_start_h, n_workers: int, k: int, mode: int, iter
     load = np.empty(int(n_workers), dtype=np.float64)
     s = ctypes.c_int64(0)
     st = _check("deft_plan_step",
-                lib().deft_plan_step(_hp(nr), _hp(ls), L, int(n_workers), int(k), int(mode), int(iteration), _hp(k_l),
+                lib().deft_plan_step(_hp(nr), _hp(ls), L, int(n_workers), int(k), int(mode), int(cost_model),
+                                     int(iteration), _hp(k_l),
                                      ctypes.byref(s), _hp(bins), _hp(load), _hp(plan_h), plan_h.size, _dp(plan_d),
                                      _dp(ws), ws.numel() * ws.element_size(), _stream(stream)),
                 allow_warn=True)

@@ -33,10 +33,11 @@ class StepPlan:
 
 class DeftStep:
     def __init__(self, tensor_sizes, n_workers: int, density: float, device="cuda:0",
-                 mode: int = deft.MODE_EXACT, k: Optional[int] = None):
+                 mode: int = deft.MODE_EXACT, k: Optional[int] = None, cost_model: int = deft.COST_EQ3):
         self.device = torch.device(device)
         self.N = int(n_workers)
         self.mode = mode
+        self.cost_model = cost_model
         self.layer_start, self.layer_tensor = deft.deft_split_layers(tensor_sizes, n_workers)
         self.layer_size = np.diff(self.layer_start)
         self.L = int(self.layer_size.size)
@@ -68,7 +69,7 @@ class DeftStep:
     def plan(self, norms: np.ndarray, iteration: int = 0) -> StepPlan:
         """Algorithm 3, Algorithm 4, then the plan of all N ranks built on the host and uploaded."""
         k_l, sum_k, bins, load, _ = deft.deft_plan_step(norms, self.layer_start, self.N, self.k, self.mode, iteration,
-                                                        self.plan_h, self.plan_d, self.ws)
+                                                        self.plan_h, self.plan_d, self.ws, cost_model=self.cost_model)
         n_layers, elems, rank_k, out_off = deft.deft_plan_rank_table(self.plan_h, self.N)
         off = np.zeros(self.N + 1, dtype=np.int64)
         off[:-1] = out_off

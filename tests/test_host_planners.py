@@ -128,6 +128,25 @@ def test_partition_matches_oracle_bit_for_bit():
         assert sorted(seen) == list(range(L))
 
 
+def test_partition_by_size_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(4)
+    for _ in range(200):
+        norms, sizes, k, L, n_g = _random_case(rng)
+        N = int(rng.integers(1, 70))
+        a, la = deft.deft_partition_model(sizes, None, N, deft.COST_SIZE)
+        b, lb = oracle.partition_by_size(sizes, N)
+        assert a.tolist() == b.tolist()
+        assert la.tobytes() == lb.tobytes()
+        k_l, _ = oracle.allocate_k(norms, sizes, k, oracle.MODE_PAPER)
+        c, lc = deft.deft_partition_model(sizes, k_l, N, deft.COST_EQ3)      # the Eq. 3 model through the same call
+        d, ld = oracle.partition(sizes, k_l, N)
+        assert c.tolist() == d.tolist() and lc.tobytes() == ld.tobytes()
+    with pytest.raises(deft.DeftError):
+        deft.deft_partition_model([5, 5], [1, 1], 2, 7)
+    with pytest.raises(deft.DeftError):
+        deft.deft_partition_model([5, 5], None, 2, deft.COST_EQ3)
+
+
 def test_partition_errors():
     with pytest.raises(deft.DeftError):
         deft.deft_partition([5, 5], [1, 0], 2)

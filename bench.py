@@ -244,6 +244,58 @@ def run_sweep(args, dev):
     print(json.dumps(rows))
 
 
+def run_trace(args, dev):
+    """Actual density (Section 5.2) and error (Eq. 2) over a stream of steps for N simulated workers
+    with different gradients (shared signal + per-worker noise), per sparsifier: the synthetic
+    analogue of the paper's Figures 4-6.  One table row per step to stderr, a JSON object to stdout."""
+    import torch
+    from paper_2307_03500_b200.simulate import MultiWorkerSim
+
+    w = make_workload(args)
+    N, d = w.n_workers, w.density
+    steps = args.steps
+    sims = {"deft": MultiWorkerSim(w.sizes, N, d, "deft", device=dev),
+            "topk": MultiWorkerSim(w.sizes, N, d, "topk", device=dev),
+            "cltk": MultiWorkerSim(w.sizes, N, d, "cltk", device=dev)}
+    gen = torch.Generator(device=dev)
+    rows = []
+    topk_density = []
+    print("%4s | %-22s | %-22s | %-22s" % ("step", "deft dens / err", "topk dens / err", "cltk dens / err"), file=sys.stderr)
+    for t in range(steps):
+        base = torch.from_numpy(w.gradient(t)).to(dev)
+        grads = []
+        for r in range(N):
+            gen.manual_seed((w.seed << 20) + t * 4096 + r)
+            noise = torch.randn(base.numel(), generator=gen, device=dev, dtype=torch.float32)
+            grads.append(base + 0.5 * base.abs() * noise)
+        row = {"step": t}
+        for name, sim in sims.items():
+            dens, err = sim.step(grads)
+            row[name] = {"density": dens, "error": err}
+        topk_density.append(row["topk"]["density"])
+        rows.append(row)
+        print("%4d | %10.6f %11.5g | %10.6f %11.5g | %10.6f %11.5g" % (
+            t, row["deft"]["density"], row["deft"]["error"], row["topk"]["density"], row["topk"]["error"],
+            row["cltk"]["density"], row["cltk"]["error"]), file=sys.stderr)
+    # DEFT at the density Top-k actually reached (the paper's Figure 6 comparison)
+    d_match = float(np.mean(topk_density))
+    sim2 = MultiWorkerSim(w.sizes, N, d_match, "deft", device=dev)
+    matched = []
+    for t in range(steps):
+        base = torch.from_numpy(w.gradient(t)).to(dev)
+        grads = []
+        for r in range(N):
+            gen.manual_seed((w.seed << 20) + t * 4096 + r)
+            noise = torch.randn(base.numel(), generator=gen, device=dev, dtype=torch.float32)
+            grads.append(base + 0.5 * base.abs() * noise)
+        dens, err = sim2.step(grads)
+        matched.append({"step": t, "density": dens, "error": err})
+    print("DEFT at density %.6f (mean actual density of Top-k): final error %.5g vs Top-k %.5g" % (
+        d_match, matched[-1]["error"], rows[-1]["topk"]["error"]), file=sys.stderr)
+    print(json.dumps({"workload": w.name, "n_workers": N, "density": d, "steps": steps, "rows": rows,
+                      "deft_at_topk_density": {"density": d_match, "rows": matched}}))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -305,6 +357,9 @@ def run_ours(args):
 
     if args.mode == "sweep":
         run_sweep(args, dev)
+        return
+    if args.mode == "trace":
+        run_trace(args, dev)
         return
 
     if args.mode != "step":
@@ -553,8 +608,9 @@ def main():
     ap.add_argument("--density", type=float, default=0.0)
     ap.add_argument("--cpu-ranks", type=int, default=4, help="ranks the oracle runs for the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select", "sweep"],
+    ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select", "sweep", "trace"],
                     help="step = the benchmark; sweep = selection vs Top-k over N and d for --workload; "
+                         "trace = density and error over --steps steps, N workers with different gradients; "
                          "the others repeat one call only, for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -195,7 +195,10 @@ def run_sweep(args, dev):
             ds = DeftStep(base.sizes, N, d, device=dev)
             e = torch.zeros_like(g)
             reps, warm = 5, 3
-            sel, acc, host = [], [], []
+            sel, acc, host, tk = [], [], [], []
+            tk_val = torch.empty(ds.k, dtype=torch.float32, device=dev)
+            tk_idx = torch.empty(ds.k, dtype=torch.int64, device=dev)
+            tk_ws = deft.alloc_workspace(ds.n_g, 1, dev)    # Top-k keeps its own remembered cut
             for it in range(warm + reps):
                 tri = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(N)]
                 for t3 in tri:
@@ -205,6 +208,10 @@ def run_sweep(args, dev):
                 a0.record(stream)
                 deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)
                 a1.record(stream)
+                b0 = torch.cuda.Event(enable_timing=True); b1 = torch.cuda.Event(enable_timing=True)
+                b0.record(stream)
+                deft.deft_topk_baseline(e, ds.k, tk_val, tk_idx, tk_ws)   # Top-k on this step's accumulated vector
+                b1.record(stream)
                 ds.norms_h.copy_(ds.norms_d, non_blocking=True)
                 stream.synchronize()
                 t0 = time.perf_counter()
@@ -215,19 +222,9 @@ def run_sweep(args, dev):
                 if it >= warm:
                     sel.append([a.elapsed_time(b) for (a, b, c) in tri])
                     acc.append(a0.elapsed_time(a1))
+                    tk.append(b0.elapsed_time(b1))
                     host.append((t1 - t0) * 1e3)
             sel_med = np.median(np.array(sel), axis=0)
-            tk_val = torch.empty(ds.k, dtype=torch.float32, device=dev)
-            tk_idx = torch.empty(ds.k, dtype=torch.int64, device=dev)
-            tk = []
-            for i in range(3 + 5):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                deft.deft_topk_baseline(e, ds.k, tk_val, tk_idx, ds.ws)
-                b.record(stream)
-                stream.synchronize()
-                if i >= 3:
-                    tk.append(a.elapsed_time(b))
             t_topk = float(np.median(tk))
             cost_max = float(plan.bin_load.max())
             row = {"workload": base.name, "density": d, "n_workers": N, "k": ds.k, "layers": ds.L,
@@ -239,7 +236,7 @@ def run_sweep(args, dev):
             print("%-12s %7g %4d %9d %5d | %9.1f %9.1f %9.1f %9.1f | %9.1f %8.2f %8.2f" % (
                 base.name, d, N, ds.k, ds.L, row["norms_us"], row["host_us"], row["select_us_max"],
                 row["select_us_sum"], row["topk_us"], row["speedup_vs_topk"], row["model_f_n"] or 0.0), file=sys.stderr)
-            del ds, e, tk_val, tk_idx
+            del ds, e, tk_val, tk_idx, tk_ws
             torch.cuda.empty_cache()
     print(json.dumps(rows))
 
@@ -323,6 +320,16 @@ def run_ours(args):
     g = g_host.to(dev)
     e = torch.zeros(n_g, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
+    # The gradient stream: an independent seeded draw for every step (SGD gradients differ from step
+    # to step), generated on the device BEFORE the timed region and kept resident; at most
+    # args.pool draws (memory), cycled beyond that.
+    pool = []
+    if args.mode == "step":
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        fit = int(max(1, (free_b - 24e9) // (4 * n_g)))
+        n_pool = max(1, min(args.pool, args.warmup + args.steps, fit))
+        pool = [W.device_gradient(w, t, dev) for t in range(n_pool)]
+        torch.cuda.synchronize()
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -334,13 +341,26 @@ def run_ours(args):
 
     launches = {"n": 0}
 
-    def one_step(it, rec=None, grad=g, marks=None):
+    tk_val = torch.empty(k, dtype=torch.float32, device=dev)
+    tk_idx = torch.empty(k, dtype=torch.int64, device=dev)
+    tk_ws = deft.alloc_workspace(n_g, 1, dev)       # its own workspace: Top-k keeps its own remembered cut
+    tk_times = []
+
+    def one_step(it, rec=None, grad=None, marks=None, with_topk=False):
         """The whole path for all N simulated ranks: accumulate + norms, D2H norms, host planner, plan
         upload, then every rank's selection + residual update — in ONE launch, or, with `marks`
         (per-rank event triples), one launch per rank for per-worker timings."""
+        if grad is None:
+            grad = pool[it % len(pool)]
         e0 = ev(); e0.record(stream)
         deft.deft_layer_norms(e, grad, ds.layer_start_d, ds.norms_d, ds.ws)
         e1 = ev(); e1.record(stream)
+        if with_topk:   # the comparison sparsifier on this step's accumulated vector (selects, does not zero)
+            ta, tb = ev(), ev()
+            ta.record(stream)
+            deft.deft_topk_baseline(e, k, tk_val, tk_idx, tk_ws)
+            tb.record(stream)
+            tk_times.append((ta, tb))
         ds.norms_h.copy_(ds.norms_d, non_blocking=True)
         stream.synchronize()
         th0 = time.perf_counter()
@@ -422,7 +442,7 @@ def run_ours(args):
         for t3 in tri:
             for x in t3:
                 x.record(stream)
-        one_step(args.warmup + args.steps + it, rank_recs, g, tri)
+        one_step(args.warmup + args.steps + it, rank_recs, None, tri, with_topk=True)
     stream.synchronize()
     t_sel = np.array([[a.elapsed_time(b) for (a, b, c) in r["ranks"]] for r in rank_recs])      # [steps, N]
     plan_w = rank_recs[-1]["plan"]
@@ -437,25 +457,15 @@ def run_ours(args):
         for t3 in tri:
             for x in t3:
                 x.record(stream)
-        one_step(args.warmup + 2 * args.steps + it, size_recs, g, tri)
+        one_step(args.warmup + 2 * args.steps + it, size_recs, None, tri)
     stream.synchronize()
     ds.cost_model = deft.COST_EQ3
     t_sel_size = np.median(np.array([[a.elapsed_time(b) for (a, b, c) in r["ranks"]] for r in size_recs]), axis=0)
     plan_s = size_recs[-1]["plan"]
 
-    # full-vector Top-k on the same GPU (comparison sparsifier), timed alone
-    tk_val = torch.empty(k, dtype=torch.float32, device=dev)
-    tk_idx = torch.empty(k, dtype=torch.int64, device=dev)
-    tk = []
-    for i in range(3 + 10):
-        a, b = ev(), ev()
-        a.record(stream)
-        deft.deft_topk_baseline(e, k, tk_val, tk_idx, ds.ws)
-        b.record(stream)
-        stream.synchronize()
-        if i >= 3:
-            tk.append(a.elapsed_time(b))
-    t_topk = float(np.median(tk))
+    # full-vector Top-k on the same GPU (comparison sparsifier): timed inside the per-worker steps above,
+    # each time on that step's accumulated vector
+    t_topk = float(np.median([a.elapsed_time(b) for (a, b) in tk_times[1:]]))
 
     # the comparison sparsifiers of Section 3 on the same vector: hard threshold at the magnitude of the
     # Top-k result's smallest entry (so that it selects k - 1 entries), and the CLT-k follower step
@@ -465,7 +475,7 @@ def run_ours(args):
     for i in range(3 + 10):
         a, b, c = ev(), ev(), ev()
         a.record(stream)
-        deft.deft_threshold_select(e, lam, tk_val, tk_idx, cnt_d, ds.ws)
+        deft.deft_threshold_select(e, lam, tk_val, tk_idx, cnt_d, tk_ws)
         b.record(stream)
         deft.deft_gather_update(g, tk_idx, k - 1, tk_val)      # a follower's values at broadcast indices
         c.record(stream)
@@ -547,6 +557,9 @@ def run_ours(args):
             "config": {"workload": w.name, "n_g": n_g, "layers": L, "n_workers": N, "density": w.density, "k": k,
                        "sum_k": int(plan.sum_k), "seed": w.seed, "k_mode": "EXACT",
                        "l2": "inputs larger than L2 (%.2f GB vector, no flush)" % (4.0 * n_g / 1e9),
+                       "gradient_stream": "%d independent seeded draws generated on the device before timing, "
+                                          "one per step%s" % (len(pool), "" if len(pool) >= args.warmup + args.steps
+                                                              else ", cycled"),
                        "multi_gpu": "replicas only"},
             "clocks": clocks,
             "e2e": {"value": world * n_g / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
@@ -608,6 +621,8 @@ def main():
     ap.add_argument("--density", type=float, default=0.0)
     ap.add_argument("--cpu-ranks", type=int, default=4, help="ranks the oracle runs for the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pool", type=int, default=105,
+                    help="independent gradient draws kept on the device (one per step; cycled beyond that)")
     ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select", "sweep", "trace"],
                     help="step = the benchmark; sweep = selection vs Top-k over N and d for --workload; "
                          "trace = density and error over --steps steps, N workers with different gradients; "

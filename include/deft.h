@@ -162,6 +162,16 @@ DEFT_API deft_status deft_bin_layers(const int32_t* bin_of_layer_h, int32_t L, i
 DEFT_API size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers);
 
 /*
+ * Clears the one part of a workspace that is carried from call to call: per layer, the
+ * first-level bucket the previous selection found, from which the next selection of a model
+ * with n_layers layers takes its speculative cut (see deft_select_planned).  Call it once
+ * after allocating the workspace.  What that area holds never changes a result: stale or
+ * arbitrary contents only decide whether a selection reads the vector once or twice (or, for
+ * absurdly low cuts, how much it stages).  Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+DEFT_API deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_layers, void* stream);
+
+/*
  * Error-feedback accumulate fused with the per-layer gradient norms —
  * Algorithm 1 line 5 and the per-layer L2 norm that Section 4.2 ranks layers by.
  *   resid_acc_d[n_g]  in/out  on entry the local error e; on exit acc = e + grad

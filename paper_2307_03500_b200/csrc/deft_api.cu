@@ -33,7 +33,7 @@ namespace {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
-struct LayerItem { int64_t start, end, k; int32_t layer_id; };
+struct LayerItem { int64_t start, end, k; int32_t layer_id; double norm = 0.0; };
 
 // Writes the plan blob for `ranks` lists of layers (each ascending in address).
 deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteration,
@@ -68,6 +68,7 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
             D.elem_off = elems_all + elems;
             D.tile_first = (int32_t)tiles;
             D.layer_id = it.layer_id;
+            D.norm = it.norm;
             tiles += (it.end - 1) / kTile - it.start / kTile + 1;
             elems += it.end - it.start;
             k += it.k;
@@ -173,6 +174,8 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.hist1 = reinterpret_cast<uint32_t*>(ws + w.hist1);
     p.hist2 = reinterpret_cast<uint32_t*>(ws + w.hist2);
     p.hist3 = reinterpret_cast<uint32_t*>(ws + w.hist3);
+    p.spec_ctl = reinterpret_cast<uint32_t*>(ws + w.hint);
+    p.hint = reinterpret_cast<uint2*>(ws + w.hint + 256);
     p.runge = reinterpret_cast<uint2*>(ws + w.runge) + 2 * ((size_t)R.tile_base + (size_t)rank);
     p.staging = reinterpret_cast<uint2*>(ws + w.staging);
     p.val = val_d;
@@ -266,6 +269,15 @@ int32_t deft_last_cuda_error(void) { return g_last_cuda_error; }
 
 void deft_debug_select_timing(void* timing_d) { g_select_timing = static_cast<unsigned long long*>(timing_d); }
 
+deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_layers, void* stream) {
+    if (!ws_d || n_layers < 1 || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    const WsLayout w = ws_layout(1, n_layers, 1);   // the kept area's place depends on the layer count only
+    const size_t bytes = 256 + sizeof(uint2) * (size_t)n_layers;
+    if (w.hint + bytes > ws_bytes) return DEFT_ERR_CAPACITY;
+    DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + w.hint, 0, bytes, static_cast<cudaStream_t>(stream)));
+    return DEFT_OK;
+}
+
 size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers) {
     if (max_elems < 1 || max_layers < 1) return 0;
     const size_t a = ws_layout(max_elems, max_layers, max_tiles(max_elems, max_layers)).total;
@@ -290,9 +302,9 @@ size_t deft_plan_bytes(int32_t L, int32_t N) {
     return plan_bytes(L, N);
 }
 
-deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
-                            const int32_t* bin_of_layer_h, int32_t L, int32_t N, int64_t iteration,
-                            void* plan_h, size_t plan_bytes_cap) {
+static deft_status plan_build_impl(const int64_t* layer_start_h, const int64_t* k_l_h,
+                                   const int32_t* bin_of_layer_h, const double* norms_h, int32_t L, int32_t N,
+                                   int64_t iteration, void* plan_h, size_t plan_bytes_cap) {
     if (!layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || L < 1 || N < 1 || N > kMaxRanks ||
         iteration < 0)
         return DEFT_ERR_INVALID_ARG;
@@ -303,9 +315,15 @@ deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
         if (b < 0 || b >= N) return DEFT_ERR_INVALID_ARG;
         // rank r reads bin (cycle + r) % N  <=>  bin b is read by rank (b - cycle) mod N
         const int32_t r = ((b - cycle) % N + N) % N;
-        ranks[r].push_back(LayerItem{layer_start_h[l], layer_start_h[l + 1], k_l_h[l], l});
+        ranks[r].push_back(LayerItem{layer_start_h[l], layer_start_h[l + 1], k_l_h[l], l, norms_h ? norms_h[l] : 0.0});
     }
     return fill_plan(plan_h, plan_bytes_cap, L, iteration, ranks);
+}
+
+deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
+                            const int32_t* bin_of_layer_h, int32_t L, int32_t N, int64_t iteration,
+                            void* plan_h, size_t plan_bytes_cap) {
+    return plan_build_impl(layer_start_h, k_l_h, bin_of_layer_h, nullptr, L, N, iteration, plan_h, plan_bytes_cap);
 }
 
 deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
@@ -321,7 +339,8 @@ deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, 
     if (sa < 0) return sa;
     deft_status s = deft_partition_model(size.data(), k_l_h, L, N, cost_model, bin_of_layer_h, bin_load_h);
     if (s != DEFT_OK) return s;
-    s = deft_plan_build(layer_start_h, k_l_h, bin_of_layer_h, L, N, iteration, plan_h, plan_bytes_cap);
+    // the plan also carries the norms: the selection kernel scales its speculative cuts with them
+    s = plan_build_impl(layer_start_h, k_l_h, bin_of_layer_h, norms_h, L, N, iteration, plan_h, plan_bytes_cap);
     if (s != DEFT_OK) return s;
     s = deft_plan_upload(plan_h, plan_d, ws_d, ws_bytes, stream);
     if (s != DEFT_OK) return s;

@@ -20,7 +20,7 @@ namespace deft {
 constexpr int kTile = 2048;          // elements per tile
 constexpr int kSelThreads = 512;     // one persistent CTA per SM (128 registers per thread)
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kSlots = 8;            // level-1 shared-memory histograms live at once per CTA
+constexpr int kSlots = 4;            // level-1 shared-memory histograms live at once per CTA
 
 // Radix digits over the 31-bit magnitude key (IEEE bits with the sign cleared):
 // level 1 = bits 30..19 (exponent + 4 mantissa bits), level 2 = bits 18..9, level 3 = bits 8..0.
@@ -33,7 +33,7 @@ constexpr int kDShift1 = 19, kDShift2 = 9;
 // Layers of at most kDirectElems elements are not streamed: one CTA loads each of them whole.
 constexpr int kDirectElems = 16384;
 // Staged entries a CTA keeps in shared memory; the rest spills to the staging stream in HBM.
-constexpr int kResident = 16384;
+constexpr int kResident = 8192;
 // Limits of one CTA's share of a rank (checked on the host before launch).
 constexpr int kMaxLocalTiles = 4096;    // tiles per CTA
 constexpr int kMaxLocalLayers = 256;    // streamed layers per CTA
@@ -129,7 +129,8 @@ struct LayerDesc {                   // 64 bytes
     int64_t elem_off;                // absolute staging index of the layer's first slot
     int32_t tile_first;              // rank-local id of the layer's first tile
     int32_t layer_id;                // id in the model's layer table (state / histogram index)
-    int64_t reserved[2];
+    double norm;                     // this step's L2 norm of the layer, or 0 if the plan was built without norms
+    int64_t reserved;
 };
 static_assert(sizeof(LayerDesc) == 64, "LayerDesc layout");
 
@@ -162,6 +163,7 @@ struct WsLayout {
     size_t zero_begin, zero_end;     // [state | hist1 | hist2 | hist3]: cleared at plan upload
     size_t state, hist1, hist2, hist3;
     size_t runge, staging;
+    size_t hint;                     // per layer: what the previous call found (see SelParams::hint); kept across calls
     size_t total;
 };
 
@@ -175,6 +177,7 @@ inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
     w.hist2 = off;    off += sizeof(uint32_t) * (size_t)kBins2 * (size_t)L;
     w.hist3 = off;    off += sizeof(uint32_t) * (size_t)kBins3 * (size_t)L;
     w.zero_end = off;
+    w.hint = off;     off += 256 + align_up(sizeof(uint2) * (size_t)L, 256);   // control words, then one entry per layer
     const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
     w.runge = off;    off += align_up(sizeof(uint2) * slots, 256);
     // + slack: the interleaved split rounds a rank up to whole super-tiles
@@ -203,6 +206,10 @@ struct SelParams {
     uint32_t* hist1;                 // [L][kBins1]
     uint32_t* hist2;                 // [L][kBins2]
     uint32_t* hist3;                 // [L][kBins3]
+    uint32_t* spec_ctl;              // kept across calls: [0] calls left without speculation, [1] CTAs that had to
+                                     // read twice in this call, [2] CTAs that have finished this call
+    uint2* hint;                     // [L] (first-level bucket of the previous call + 1 or 0 = none, that call's
+                                     // layer norm as float bits); read and updated
     uint2* runge;                    // this rank's (CTA, layer) pairs (slot = CTA + layer position): totals
     uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output

@@ -1,25 +1,32 @@
 // Layer-wise top-k selection for one worker (Algorithm 5) as ONE persistent cooperative
 // kernel: a segmented radix select over magnitude bit patterns followed by an ordered
 // compaction.  One CTA of 512 threads per SM; five steps separated by grid barriers.  Every
-// CTA owns the same contiguous run of the rank's tiles in every step and keeps what it
-// stages for them (in shared memory; overflow spills to HBM), so after the second read of the
-// vector all work is local to the CTA that staged the data.
+// CTA owns the same tiles of the call in every step and keeps what it stages for them (in
+// shared memory; overflow spills to HBM), so after the reading steps all work is local to the
+// CTA that staged the data.
 //
 //   A   read 1: per-layer histogram of key bits 30..19 in shared memory, flushed with integer
 //       atomics; the CTA that flushes a layer's last tiles finds the bucket b1 holding the
-//       k-th largest key
-//   B   read 2: one warp per tile keeps the whole tile in registers and moves every entry
-//       with bucket >= b1, in index order, behind the CTA's staging cursor; bucket-b1 entries
-//       feed the level-2 histogram (bits 18..9)
+//       k-th largest key.  In the same pass every entry at or above a SPECULATIVE cut — the
+//       bucket the previous call found for the layer, lowered by a margin — is moved, in
+//       index order, behind the CTA's staging cursor.
+//   B   a CTA whose cuts were all at or below the true b1 already holds everything it needs
+//       and reads nothing; any other CTA drops what it staged and reads its tiles a second
+//       time with the true cut.  Then the staged entries of bucket b1 feed the level-2
+//       histogram (bits 18..9).
 //   S2  every CTA finds bucket b2 of its layers from the level-2 histograms, then adds the
 //       level-3 histogram (bits 8..0) of its staged entries of bucket (b1, b2)
 //   S3  every CTA fixes the exact threshold key T and the number of entries equal to T to
 //       take, counts its staged entries above / equal to T per tile, publishes its totals
-//   S4  every CTA adds up the totals of the CTAs before it, scans its own tiles, and writes
-//       (value, int64 index) in ascending index (equal keys: lowest indices first);
+//   S4  every CTA adds up the totals of the tiles before its own, scans its own tiles, and
+//       writes (value, int64 index) in ascending index (equal keys: lowest indices first);
 //       optionally zeroes the selected entries of the vector (residual update)
 // Layers of at most kDirectElems elements take no part in this: at the end one CTA loads
 // each of them whole and finishes it from shared memory.
+//
+// The speculative cut only decides whether step B has to read: the staged set is always a
+// superset of what the true cut keeps, so the result does not depend on it.  In a training
+// loop the cut of a layer moves little from step to step and the vector is read once.
 //
 // Determinism: histograms use integer atomics (order-free); the staging order inside a CTA
 // depends on warp timing but every output position is a function of counts and of the tile
@@ -33,18 +40,23 @@ namespace cg = cooperative_groups;
 namespace deft {
 namespace {
 
-constexpr int kS2Chunk = 8;       // layers whose level-3 histograms are built at once
-constexpr int kBSlots = 4;        // layers whose level-2 histograms are built at once
+#ifndef DEFT_SPEC_MARGIN
+#define DEFT_SPEC_MARGIN 1
+#endif
+constexpr int kSpecMargin = DEFT_SPEC_MARGIN;   // buckets (of 1/16 octave) the speculative cut lies below the predicted b1
+constexpr uint32_t kSpecBudgetPerTile = 64;   // speculative staging stops at this many entries per tile of the CTA
+constexpr int kSpecDensity = 8;
+constexpr uint32_t kSpecCooldown = 8;   // calls without speculation after a call in which a speculative cut failed   // no speculation for layers that select more than 1 / kSpecDensity of their entries
 
 // shared-memory carve-up (bytes)
-constexpr int kSmMain = 0;   // A: kSlots level-1 histograms | B..S4: resident entries | direct: keys
+constexpr int kSmMain = 0;   // A: kSlots level-1 histograms, then resident entries | direct: keys
 constexpr int kSmMainBytes = 128 * 1024;
-static_assert(kSlots * kBins1 * 4 <= kSmMainBytes && kResident * 8 <= kSmMainBytes &&
-              kDirectElems * 4 <= kSmMainBytes, "main region");
-constexpr int kSmAux = kSmMain + kSmMainBytes;   // B: level-2 slots | S2: level-3 slots | direct: its histograms
+constexpr int kSmRes = kSmMain + kSlots * kBins1 * 4;   // resident staged entries (live from step A on)
+static_assert(kSlots * kBins1 * 4 + kResident * 8 <= kSmMainBytes && kDirectElems * 4 <= kSmMainBytes &&
+              3 * (kMaxWeightedLayers + 1) * 4 <= kSmMainBytes, "main region");
+constexpr int kSmAux = kSmMain + kSmMainBytes;   // direct layers: their histograms
 constexpr int kSmAuxBytes = 20 * 1024;
-static_assert(kBSlots * kBins2 * 4 <= kSmAuxBytes && kS2Chunk * kBins3 * 4 <= kSmAuxBytes &&
-              kDBins1 * 4 + kDBins2 * 4 <= kSmAuxBytes && kDBins2 >= kDBins3, "aux region");
+static_assert(kDBins1 * 4 + kDBins2 * 4 <= kSmAuxBytes && kDBins2 >= kDBins3, "aux region");
 constexpr int kSmTile = kSmAux + kSmAuxBytes;    // per local tile: first entry, entries, counts
 constexpr int kSmTileBytes = kMaxLocalTiles * 10;
 constexpr int kSmLayer = kSmTile + kSmTileBytes; // per local streamed layer, see LayerTable
@@ -68,10 +80,11 @@ enum MiscOff : int {   // word offsets inside the misc area
     kMOut3 = 64,       // 4: result of block_scan_select
     kMLast = 72,       // kSlots: this CTA flushed the layer's last tiles
     kMCursor = 80,     // 1: staged entries of this CTA
-    kMTab = 96,        // 2 * kBSlots: per-slot staging threshold, then per-slot b1 in step B
+    kMFlag = 96,       // 1: this CTA has to read its tiles again
+    kMTried = 97,      // 1: at least one layer of this CTA had a speculative cut
     kMWarpCnt = 128,   // 32: per-warp packed counts (direct layers)
 };
-static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4 && kSlots <= 8 && kBSlots <= 32, "misc area");
+static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4 && kSlots <= 8, "misc area");
 
 // Facts about the CTA's streamed layers (shared memory, struct of arrays).
 struct LayerTable {
@@ -83,6 +96,7 @@ struct LayerTable {
     int64_t end[kMaxLocalLayers];
     int64_t out_off[kMaxLocalLayers];
     uint32_t k[kMaxLocalLayers];     // entries to select
+    uint32_t sthr[kMaxLocalLayers];  // entries with key >= sthr are staged (0xffffffff: none)
     uint32_t v0[kMaxLocalLayers];    // step value: prefix (b1, b2) | T
     uint32_t v1[kMaxLocalLayers];    // step value: krem1 | krem2 | need
     uint32_t base_gt[kMaxLocalLayers];
@@ -280,22 +294,6 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ acc, const T
     }
 }
 
-__device__ __forceinline__ void hist_tile(const float* __restrict__ acc, const TileSpan& ts,
-                                          uint32_t* h, int lane) {
-    TileRegs t;
-    uint32_t vm[2];
-    load_tile(acc, ts, lane, t, vm);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        atomicAdd(&h[key_of(t.v[i].x) >> kShift1], 1u);
-        atomicAdd(&h[key_of(t.v[i].y) >> kShift1], 1u);
-        atomicAdd(&h[key_of(t.v[i].z) >> kShift1], 1u);
-        atomicAdd(&h[key_of(t.v[i].w) >> kShift1], 1u);
-    }
-    // the components outside the layer were counted as zeros
-    if (lane == 0 && ts.e - ts.s != kTile) atomicSub(&h[0], (uint32_t)(kTile - (ts.e - ts.s)));
-}
-
 // Where a CTA's staged entry number `pos` lives.
 struct Stage {
     uint2* res;      // shared memory, kResident entries
@@ -344,19 +342,15 @@ __device__ __forceinline__ uint32_t pick4(uint32_t a, uint32_t b, uint32_t c, ui
     return (sel & 2) ? cd : ab;
 }
 
-// The rare part of the staging pass, kept out of line and small (the hot loop around it must
+// The rare part of a reading pass, kept out of line and small (the hot loop around it must
 // stay resident in the instruction cache): moves the tile's marked entries behind the CTA's
 // cursor in index order (load, lane, component = ascending offset).  k0 / k1: bit (4 * (i % 8)
 // + c) of word i / 8 marks component c of this lane's load i.  The values are read again from
 // the vector (the tile has just been loaded: they come from L1 / L2).  wbase: 16 words of
 // shared memory private to the warp.  Returns (first entry, entries).
-__device__ __noinline__ uint2 filter_marked(const uint32_t* __restrict__ tile, uint32_t k0, uint32_t k1, uint32_t b1,
-                                            uint32_t* h2, uint2* res, uint2* spill, uint32_t ytag,
-                                            uint32_t* cursor, uint32_t* wbase) {
+__device__ __noinline__ uint2 stage_marked(const uint32_t* __restrict__ tile, uint32_t k0, uint32_t k1, uint2* res,
+                                           uint2* spill, uint32_t ytag, uint32_t* cursor, uint32_t* wbase) {
     const int lane = threadIdx.x & 31;
-#ifdef DEFT_PROFILE_FILTER
-    const long long pf0 = clock64();
-#endif
     // per-load counts of this lane, 8 bits each, four loads per word; scanned over the lanes
     uint32_t excl[4], tot[4];
 #pragma unroll
@@ -387,34 +381,46 @@ __device__ __noinline__ uint2 filter_marked(const uint32_t* __restrict__ tile, u
         const uint32_t before_lanes = (pick4(excl[0], excl[1], excl[2], excl[3], i >> 2) >> (8 * (i & 3))) & 0xffu;
         const uint32_t before_mine = __popc((uint32_t)(all >> (4 * i)) & ((1u << c) - 1u));
         const uint32_t off = (uint32_t)((i * 32 + lane) * 4 + c);
-        const uint32_t bits = __ldg(tile + off);
-        const uint32_t key = key_of(bits);
-        if ((key >> kShift1) == b1) atomicAdd(&h2[(key >> kShift2) & (kBins2 - 1)], 1u);
-        stage_put(st, wbase[i] + before_lanes + before_mine, make_uint2(bits, ytag | off));
+        stage_put(st, wbase[i] + before_lanes + before_mine, make_uint2(__ldg(tile + off), ytag | off));
     }
     __syncwarp();   // wbase is rewritten by the warp's next tile
-#ifdef DEFT_PROFILE_FILTER
-    if (lane == 0) { atomicAdd(cursor + 1, 1u); atomicAdd(cursor + 2, (uint32_t)(clock64() - pf0)); }
-#endif
     return make_uint2(first, n);
 }
 
-// Staging pass over one tile: marks the entries with bucket >= b1; tiles without any cost a
-// compare per element.
-__device__ __forceinline__ uint2 filter_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t thr,
-                                             uint32_t b1, uint32_t* h2, const Stage& st, uint32_t ytag,
-                                             uint32_t* cursor, uint32_t* wbase, int lane) {
-    TileRegs t;
-    uint32_t vm[2];
-    load_tile(acc, ts, lane, t, vm);             // entries with key >= thr are staged
-    uint32_t keep[2] = {0u, 0u};                 // bit (4*(i%8) + c) of keep[i/8]
+// keep[]: bit (4 * (i % 8) + c) of keep[i / 8] = component c of load i has key >= thr and lies in the layer.
+__device__ __forceinline__ void mark_tile(const TileRegs& t, const uint32_t (&vm)[2], uint32_t thr, uint32_t (&keep)[2]) {
+    keep[0] = keep[1] = 0u;
 #pragma unroll
     for (int i = 0; i < 16; ++i) keep[i >> 3] |= keep4(t.v[i], thr) << (4 * (i & 7));
     keep[0] &= vm[0];
     keep[1] &= vm[1];
+}
+
+// Reading pass over one tile.  kHist: count every element in the level-1 histogram h.
+// Entries with key >= thr are staged (thr = 0xffffffff: none).  Returns (first entry, entries).
+template <bool kHist>
+__device__ __forceinline__ uint2 read_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t* h,
+                                           uint32_t thr, const Stage& st, uint32_t ytag, uint32_t* cursor,
+                                           uint32_t* wbase, int lane) {
+    TileRegs t;
+    uint32_t vm[2];
+    load_tile(acc, ts, lane, t, vm);
+    if (kHist) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            atomicAdd(&h[key_of(t.v[i].x) >> kShift1], 1u);
+            atomicAdd(&h[key_of(t.v[i].y) >> kShift1], 1u);
+            atomicAdd(&h[key_of(t.v[i].z) >> kShift1], 1u);
+            atomicAdd(&h[key_of(t.v[i].w) >> kShift1], 1u);
+        }
+        // the components outside the layer were loaded as zeros
+        if (lane == 0 && ts.e - ts.s != kTile) atomicSub(&h[0], (uint32_t)(kTile - (ts.e - ts.s)));
+    }
+    uint32_t keep[2];
+    mark_tile(t, vm, thr, keep);
     if (!__any_sync(0xffffffffu, (keep[0] | keep[1]) != 0)) return make_uint2(0u, 0u);
-    return filter_marked(reinterpret_cast<const uint32_t*>(acc + ts.lo), keep[0], keep[1], b1, h2, st.res, st.spill,
-                         ytag, cursor, wbase);
+    return stage_marked(reinterpret_cast<const uint32_t*>(acc + ts.lo), keep[0], keep[1], st.res, st.spill, ytag,
+                        cursor, wbase);
 }
 
 // ---------------------------------------------------------------------------------
@@ -575,6 +581,10 @@ __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
 __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRange& r, LayerTable* lt,
                                                  uint32_t* scratch) {
     int nl = 0;
+    // scratch[kMTried - kMScratch] is the CTA's "speculated" flag (same misc area)
+    const bool spec_on = !p.fixed_thr && __ldcg(p.spec_ctl) == 0u;
+    if (threadIdx.x == 0) scratch[kMTried - kMScratch] = 0u;
+    __syncthreads();
     for (int j0 = r.jA; j0 <= r.jB; j0 += kSelThreads) {
         const int j = j0 + (int)threadIdx.x;
         const bool streamed = j <= r.jB && !is_direct(p, j);
@@ -589,6 +599,24 @@ __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRa
             lt->end[c] = p.desc[j].end;
             lt->out_off[c] = p.desc[j].out_off;
             lt->k[c] = (uint32_t)p.desc[j].k;
+            // speculative cut: the bucket the previous call found for this layer, moved by as many
+            // buckets (16 per octave) as the layer's norm has changed, lowered by a margin
+            uint32_t sthr = 0xffffffffu;
+            if (p.fixed_thr) {
+                sthr = p.thr_key + 1u;                       // key >= thr_key + 1  <=>  key > thr_key
+            } else if (spec_on && p.desc[j].k * kSpecDensity <= p.desc[j].end - p.desc[j].start) {
+                const uint2 hint = __ldcg(p.hint + p.desc[j].layer_id);
+                if (hint.x != 0 && hint.x <= (uint32_t)kBins1) {
+                    int pb = (int)hint.x - 1 - kSpecMargin;
+                    const float was = __uint_as_float(hint.y), now = (float)p.desc[j].norm;
+                    if (was > 0.0f && now > 0.0f && was < 3.0e38f && now < 3.0e38f)
+                        pb += (int)floorf(16.0f * log2f(now / was));
+                    pb = pb < 0 ? 0 : (pb > kBins1 - 1 ? kBins1 - 1 : pb);
+                    sthr = (uint32_t)pb << kShift1;
+                    scratch[kMTried - kMScratch] = 1u;
+                }
+            }
+            lt->sthr[c] = sthr;
         }
         nl += (int)tot;
     }
@@ -604,13 +632,16 @@ __device__ __forceinline__ int tile_layer(const LayerTable* lt, int nl, int q, i
 }
 
 // ---------------------------------------------------------------------------------
-// step A: level-1 histograms, kSlots layers at a time
+// step A: level-1 histograms (kSlots layers at a time) and speculative staging
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r, const LayerTable* lt, int nl,
-                                           unsigned char* smem) {
+__device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r, const LayerTable* lt, int nl,
+                                           TileTable* tt, const Stage& st, unsigned char* smem) {
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem + kSmMain);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
+    uint32_t* wbase = reinterpret_cast<uint32_t*>(smem + kSmWBase);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMFlag] = 0; }
+    const uint32_t budget = (uint32_t)r.nloc * kSpecBudgetPerTile + 1024u;
     for (int c0 = 0; c0 < nl; c0 += kSlots) {
         const int ns = nl - c0 < kSlots ? nl - c0 : kSlots;
         for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) hist[i] = 0;
@@ -625,7 +656,17 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
             const int cl = tile_layer(lt, c0 + ns, q, c);
             if (cl < 0) continue;
             const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-            hist_tile(p.acc, ts, hist + (cl - c0) * kBins1, lane);
+            // a cut that turns out far too low must not flood the staging area: past the budget the
+            // CTA stops staging and reads a second time in step B
+            uint32_t thr = lt->sthr[cl];
+            if (*reinterpret_cast<volatile uint32_t*>(misc + kMCursor) > budget) {
+                thr = 0xffffffffu;
+                if (lane == 0) misc[kMFlag] = 1u;
+            }
+            const uint2 fn = read_tile<true>(p.acc, ts, hist + (cl - c0) * kBins1, thr, st,
+                                             pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
+                                             wbase + 16 * warp, lane);
+            if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
         }
         __syncthreads();
         stamp(p, 9);
@@ -655,6 +696,8 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
             if (threadIdx.x == 0) {
                 p.state[lid].b1 = misc[kMOut3];
                 p.state[lid].above1 = misc[kMOut3 + 1];
+                // the next call's speculative cut starts from here
+                p.hint[lid] = make_uint2(misc[kMOut3] + 1u, __float_as_uint((float)p.desc[lt->j[cl]].norm));
             }
             __syncthreads();
         }
@@ -663,52 +706,62 @@ __device__ __forceinline__ void step_hist1(const SelParams& p, const CtaRange& r
 }
 
 // ---------------------------------------------------------------------------------
-// step B: staging pass + level-2 histograms, kBSlots layers at a time
+// step B: second read where the speculative cut was too high, then level-2 histograms
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
-                                            TileTable* tt, const Stage& st, unsigned char* smem) {
-    uint32_t* hist2s = reinterpret_cast<uint32_t*>(smem + kSmAux);
+__device__ __forceinline__ void step_read2(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
+                                           TileTable* tt, const Stage& st, unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
+    uint32_t* wbase = reinterpret_cast<uint32_t*>(smem + kSmWBase);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMCursor + 1] = 0; misc[kMCursor + 2] = 0; }   // +1, +2: profiling build
-    for (int c0 = 0; c0 < nl; c0 += kBSlots) {
-        const int ns = nl - c0 < kBSlots ? nl - c0 : kBSlots;
-        if ((int)threadIdx.x < ns) {
-            const LayerState* ls = p.state + lt->lid[c0 + threadIdx.x];
-            if (p.fixed_thr) {
-                misc[kMTab + threadIdx.x] = p.thr_key + 1u;     // key >= thr_key + 1  <=>  key > thr_key
-                misc[kMTab + kBSlots + threadIdx.x] = 0xffffffffu;   // no bucket feeds the level-2 histogram
-            } else {
-                const uint32_t b1 = __ldcg(&ls->b1);
-                misc[kMTab + threadIdx.x] = b1 << kShift1;      // key >= thr  <=>  bucket >= b1
-                misc[kMTab + kBSlots + threadIdx.x] = b1;
-                lt->v1[c0 + threadIdx.x] = lt->k[c0 + threadIdx.x] - __ldcg(&ls->above1);   // krem1
+    if (threadIdx.x == 0 && p.fixed_thr) misc[kMFlag] = 1u;   // else: set in step A if the CTA ran over its budget
+    __syncthreads();
+    if (!p.fixed_thr) {
+        for (int c = threadIdx.x; c < nl; c += kSelThreads) {
+            const LayerState* ls = p.state + lt->lid[c];
+            const uint32_t b1 = __ldcg(&ls->b1);
+            lt->v0[c] = b1;
+            lt->v1[c] = lt->k[c] - __ldcg(&ls->above1);          // krem1
+            const uint32_t need_thr = b1 << kShift1;             // key >= need_thr  <=>  bucket >= b1
+            if (lt->sthr[c] > need_thr) {                        // staged too little (or nothing) for this layer
+                lt->sthr[c] = need_thr;
+                misc[kMFlag] = 1u;
             }
-        }
-        for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) hist2s[i] = 0;
-        __syncthreads();
-        int la, lb;
-        local_span(r, lt, c0, c0 + ns - 1, la, lb);
-        int c = c0;
-        for (int lq = la + warp; lq < lb; lq += kSelWarps) {
-            const int q = local_tile(p, r, lq);
-            if (q < 0) continue;
-            const int cl = tile_layer(lt, c0 + ns, q, c);
-            if (cl < 0) continue;
-            const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-            const uint2 fn = filter_tile(p.acc, ts, misc[kMTab + cl - c0], misc[kMTab + kBSlots + cl - c0],
-                                         hist2s + (cl - c0) * kBins2, st,
-                                         pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
-                                         reinterpret_cast<uint32_t*>(smem + kSmWBase) + 16 * warp, lane);
-            if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
-        }
-        __syncthreads();
-        for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) {
-            const uint32_t cnt = hist2s[i];
-            if (cnt) atomicAdd(p.hist2 + (size_t)lt->lid[c0 + i / kBins2] * kBins2 + (i % kBins2), cnt);
         }
         __syncthreads();
     }
+    if (misc[kMFlag]) {   // uniform over the CTA: drop what was staged, read the CTA's tiles with the true cuts
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            misc[kMCursor] = 0;
+            if (!p.fixed_thr && misc[kMTried]) atomicAdd(p.spec_ctl + 1, 1u);   // a speculative cut failed
+        }
+        __syncthreads();
+        int la, lb;
+        if (nl > 0) {
+            local_span(r, lt, 0, nl - 1, la, lb);
+            int c = 0;
+            for (int lq = la + warp; lq < lb; lq += kSelWarps) {
+                const int q = local_tile(p, r, lq);
+                if (q < 0) continue;
+                const int cl = tile_layer(lt, nl, q, c);
+                if (cl < 0) continue;
+                const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
+                const uint2 fn = read_tile<false>(p.acc, ts, nullptr, lt->sthr[cl], st,
+                                                  pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
+                                                  wbase + 16 * warp, lane);
+                if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
+            }
+        }
+        __syncthreads();
+    }
+    if (p.fixed_thr) return;
+    const uint32_t total = misc[kMCursor];
+    for_each_staged(st, total, [&](const uint2 ent) {
+        const int c = (int)y_layer(ent.y);
+        const uint32_t key = key_of(ent.x);
+        if ((key >> kShift1) == lt->v0[c])
+            atomicAdd(p.hist2 + (size_t)lt->lid[c] * kBins2 + ((key >> kShift2) & (kBins2 - 1)), 1u);
+    });
 }
 
 // ---------------------------------------------------------------------------------
@@ -716,7 +769,6 @@ __device__ __forceinline__ void step_filter(const SelParams& p, const CtaRange& 
 // ---------------------------------------------------------------------------------
 __device__ __forceinline__ void step_hist3(const SelParams& p, LayerTable* lt, int nl, const Stage& st,
                                            unsigned char* smem) {
-    uint32_t* h3 = reinterpret_cast<uint32_t*>(smem + kSmAux);
     const uint32_t* misc = reinterpret_cast<const uint32_t*>(smem + kSmMisc);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t total = misc[kMCursor];
@@ -724,31 +776,20 @@ __device__ __forceinline__ void step_hist3(const SelParams& p, LayerTable* lt, i
     for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer
         const int lid = lt->lid[c];
         const uint2 s2 = warp_scan_select(p.hist2 + (size_t)lid * kBins2, kBins2 / 32, lt->v1[c]);
-        const uint32_t b2 = s2.x, above2 = s2.y;
-        const uint32_t b1 = __ldcg(&p.state[lid].b1);
         __syncwarp();
         if (lane == 0) {
-            lt->v0[c] = (b1 << (kShift1 - kShift2)) | b2;   // key >> kShift2 of the candidates
-            lt->v1[c] = lt->v1[c] - above2;                 // krem2
+            lt->v0[c] = (lt->v0[c] << (kShift1 - kShift2)) | s2.x;   // key >> kShift2 of the candidates
+            lt->v1[c] = lt->v1[c] - s2.y;                            // krem2
         }
     }
-    for (int c0 = 0; c0 < nl; c0 += kS2Chunk) {
-        const int ns = nl - c0 < kS2Chunk ? nl - c0 : kS2Chunk;
-        for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) h3[i] = 0;
-        __syncthreads();
-        for_each_staged(st, total, [&](const uint2 ent) {
-            const int c = (int)y_layer(ent.y);
-            const uint32_t key = key_of(ent.x);
-            if (c >= c0 && c < c0 + ns && (key >> kShift2) == lt->v0[c])
-                atomicAdd(&h3[(c - c0) * kBins3 + (key & (kBins3 - 1))], 1u);
-        });
-        __syncthreads();
-        for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) {
-            const uint32_t cnt = h3[i];
-            if (cnt) atomicAdd(p.hist3 + (size_t)lt->lid[c0 + i / kBins3] * kBins3 + (i % kBins3), cnt);
-        }
-        __syncthreads();
-    }
+    __syncthreads();
+    // the candidates of bucket (b1, b2) are a small fraction of k: straight to the global histograms
+    for_each_staged(st, total, [&](const uint2 ent) {
+        const int c = (int)y_layer(ent.y);
+        const uint32_t key = key_of(ent.x);
+        if ((key >> kShift2) == lt->v0[c])
+            atomicAdd(p.hist3 + (size_t)lt->lid[c] * kBins3 + (key & (kBins3 - 1)), 1u);
+    });
 }
 
 // ---------------------------------------------------------------------------------
@@ -1118,33 +1159,29 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     TileTable* tt = reinterpret_cast<TileTable*>(smem + kSmTile);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     CtaRange r = cta_range(p, reinterpret_cast<int*>(smem + kSmTf));
-    int nl = build_layer_table(p, r, lt, misc + kMScratch);
+    if (p.weighted)   // contiguous runs of equal estimated cost instead of equal length
+        r = weighted_range(p, reinterpret_cast<uint32_t*>(smem + kSmMain), reinterpret_cast<int*>(smem + kSmTf),
+                           misc + kMScratch);
+    const int nl = build_layer_table(p, r, lt, misc + kMScratch);
     Stage st;
-    st.res = reinterpret_cast<uint2*>(smem + kSmMain);
+    st.res = reinterpret_cast<uint2*>(smem + kSmRes);
     st.spill = spill_base(p, r);
 
     if (!p.fixed_thr) {   // uniform over the grid
-        step_hist1(p, r, lt, nl, smem);
+        step_read1(p, r, lt, nl, tt, st, smem);
         stamp(p, 1);
         grid.sync();
     }
-    if (p.weighted) {   // from here on: contiguous runs of equal estimated cost
-        r = weighted_range(p, reinterpret_cast<uint32_t*>(smem + kSmMain), reinterpret_cast<int*>(smem + kSmTf),
-                           misc + kMScratch);
-        nl = build_layer_table(p, r, lt, misc + kMScratch);
-        st.spill = spill_base(p, r);
-    }
     unsigned long long tb0 = 0;
     if (p.timing && threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tb0));
-    step_filter(p, r, lt, nl, tt, st, smem);
+    step_read2(p, r, lt, nl, tt, st, smem);
     if (p.timing && threadIdx.x == 0) {
         unsigned long long tb1;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tb1));
         p.timing[16 + blockIdx.x] = tb1 - tb0;
         p.timing[16 + 160 + blockIdx.x] = misc[kMCursor];
         p.timing[16 + 320 + blockIdx.x] = (unsigned long long)nl | ((unsigned long long)r.nloc << 16) |
-                                          ((unsigned long long)misc[kMCursor + 1] << 32);
-        p.timing[16 + 480 + blockIdx.x] = misc[kMCursor + 2];   // profiling build: cycles in filter_marked
+                                          ((unsigned long long)misc[kMFlag] << 32);
     }
     stamp(p, 2);
     if (!p.fixed_thr) {
@@ -1169,6 +1206,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     for (int j = blockIdx.x; j < p.n_my; j += gridDim.x)
         if (is_direct(p, j)) resolve_direct(p, j, smem);   // uniform over the CTA
     stamp(p, 6);
+    if (!p.fixed_thr && threadIdx.x == 0) {
+        // the last CTA to finish settles whether the next calls speculate: after a call with a failed
+        // cut, the next kSpecCooldown calls read twice as a matter of course
+        __threadfence();
+        if (atomicAdd(p.spec_ctl + 2, 1u) == gridDim.x - 1) {
+            const uint32_t cool = __ldcg(p.spec_ctl), failed = __ldcg(p.spec_ctl + 1);
+            p.spec_ctl[0] = cool > 0 ? cool - 1 : (failed > 0 ? kSpecCooldown : 0u);
+            p.spec_ctl[1] = 0u;
+            p.spec_ctl[2] = 0u;
+        }
+    }
 }
 
 __global__ void k_zero_at(float* __restrict__ acc, const int64_t* __restrict__ idx, int64_t count) {

@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.deft_plan_rank_info.argtypes = [vp, i32, vp, vp, vp, vp]
         L.deft_plan_rank_table.restype = i32
         L.deft_plan_rank_table.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.deft_workspace_init.restype = i32
+        L.deft_workspace_init.argtypes = [vp, sz, i32, vp]
         L.deft_threshold_select.restype = i32
         L.deft_threshold_select.argtypes = [vp, i64, ctypes.c_float, i32, vp, vp, i64, vp, vp, sz, vp]
         L.deft_clt_leader.restype = i32
@@ -233,7 +235,10 @@ def deft_workspace_bytes(max_elems: int, max_layers: int) -> int:
 def alloc_workspace(max_elems: int, max_layers: int, device="cuda"):
     """A torch uint8 tensor of deft_workspace_bytes() bytes (torch allocations are 512-byte aligned)."""
     import torch
-    return torch.empty(deft_workspace_bytes(max_elems, max_layers), dtype=torch.uint8, device=device)
+    ws = torch.empty(deft_workspace_bytes(max_elems, max_layers), dtype=torch.uint8, device=device)
+    with torch.cuda.device(ws.device):
+        _check("deft_workspace_init", lib().deft_workspace_init(_dp(ws), ws.numel(), int(max_layers), _stream(None)))
+    return ws
 
 
 def deft_layer_norms(resid_acc, grad, layer_start_d, norms_d, ws, stream=None) -> None:

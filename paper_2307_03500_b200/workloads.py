@@ -137,6 +137,32 @@ class Workload:
         return g
 
 
+def device_gradient(w: "Workload", step: int, device, out=None):
+    """The same distribution as ``Workload.gradient`` drawn on the GPU with torch's generator
+    (seeded by (seed, step); NOT the same numbers as the host draw): a benchmark needs a fresh
+    vector every step and the host generator takes seconds per draw at full size.  Input
+    generation only — nothing of the method is computed here."""
+    import torch
+    gen = torch.Generator(device=device)
+    gen.manual_seed(((w.seed & 0xFFFF) << 32) + 0xD00D0000 + int(step))
+    g = out if out is not None else torch.empty(w.n_g, dtype=torch.float32, device=device)
+    scales = w.scales()
+    pos = 0
+    for t, size in enumerate(w.sizes):
+        view = g[pos:pos + size]
+        if w.dist == "laplace":
+            u = torch.rand(size, generator=gen, device=device, dtype=torch.float32) - 0.5
+            view.copy_(-float(scales[t]) * torch.sign(u) * torch.log1p(-2.0 * u.abs()).clamp_(min=-80.0))
+        else:
+            view.normal_(0.0, float(scales[t]), generator=gen)
+            if w.dist == "lstm_rows" and t in w.sparse_tensors:
+                rows = size // w.row_len
+                keep = torch.rand(rows, generator=gen, device=device) < w.row_keep
+                view.view(rows, w.row_len).mul_(keep.to(torch.float32).unsqueeze(1))
+        pos += size
+    return g
+
+
 def tiny() -> Workload:
     return Workload("tiny", tiny_sizes(), 4, 0.01, 0, "gauss", 1e-4, 1e-1)
 

@@ -297,6 +297,35 @@ def test_large_multi_layer_rank_cost_weighted_split(deft):
     assert val.tobytes() == want_val.tobytes()
 
 
+@pytest.mark.parametrize("scale_first", [1.0, 16.0, 1.0 / 16.0, 1e-6, 1e6])
+def test_speculative_cut_from_previous_call_never_changes_the_result(deft, scale_first):
+    """The kernel stages entries above a cut remembered from the previous call on the same
+    workspace.  Whatever that cut is — exact, far too high (second read needed), far too low
+    (nearly everything staged) — the selection must equal the oracle's."""
+    w = W.scaled_down(W.gpt2_medium(4, 0.01), 32)
+    x = w.gradient(0)
+    start, _ = oracle.split_layers(w.sizes, 4)
+    size = np.diff(start)
+    k_l = np.maximum(1, size // 97)
+    k_l[::5] = np.maximum(1, size[::5] // 3)                    # some layers too dense for a speculative cut
+    my = np.arange(size.size, dtype=np.int32)
+    ws = deft.alloc_workspace(int(start[-1]), size.size)
+    first = (x * np.float32(scale_first)).astype(np.float32)
+    first[start[3]:start[4]] = x[start[3]:start[4]] * np.float32(1e3)      # one layer's cut moves the other way
+    got0 = _gpu_select(deft, _dev(first), start, k_l, my, ws=ws)
+    want0 = oracle.select_rank(first, start, k_l, my)
+    assert np.array_equal(got0[1], want0[1]) and got0[0].tobytes() == want0[0].tobytes()
+    want = oracle.select_rank(x, start, k_l, my)
+    for _ in range(2):                                           # second call: cuts from `first`; third: from x itself
+        got = _gpu_select(deft, _dev(x), start, k_l, my, ws=ws)
+        assert np.array_equal(got[1], want[1]) and got[0].tobytes() == want[0].tobytes()
+    # a subset of the layers, Top-k and a hard threshold share the workspace (and its remembered cuts)
+    sub = my[1::2]
+    got = _gpu_select(deft, _dev(x), start, k_l, sub, ws=ws)
+    wsub = oracle.select_rank(x, start, k_l, sub)
+    assert np.array_equal(got[1], wsub[1]) and got[0].tobytes() == wsub[0].tobytes()
+
+
 def test_select_is_bit_deterministic_run_to_run(deft):
     w = W.scaled_down(W.gpt2_medium(4, 0.01), 16)
     x = w.gradient(0)

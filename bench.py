@@ -185,7 +185,7 @@ def run_sweep(args, dev):
 
     stream = torch.cuda.current_stream()
     base = W.WORKLOADS[args.workload]()
-    g = torch.from_numpy(base.gradient(0)).to(dev)
+    g = torch.empty(base.n_g, dtype=torch.float32, device=dev)
     rows = []
     print("%-12s %7s %4s %9s %5s | %9s %9s %9s %9s | %9s %8s %8s" % (
         "workload", "d", "N", "k", "L", "norms_us", "host_us", "sel_max", "sel_sum", "topk_us", "speedup", "model"),
@@ -194,7 +194,7 @@ def run_sweep(args, dev):
         for N in ([args.n_workers] if args.n_workers else [1, 2, 4, 8, 16, 32, 64]):
             ds = DeftStep(base.sizes, N, d, device=dev)
             e = torch.zeros_like(g)
-            reps, warm = 5, 3
+            reps, warm = 6, 12
             sel, acc, host, tk = [], [], [], []
             tk_val = torch.empty(ds.k, dtype=torch.float32, device=dev)
             tk_idx = torch.empty(ds.k, dtype=torch.int64, device=dev)
@@ -204,6 +204,7 @@ def run_sweep(args, dev):
                 for t3 in tri:
                     for x in t3:
                         x.record(stream)
+                W.device_gradient(base, it, dev, out=g)          # an independent draw every step
                 a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
                 a0.record(stream)
                 deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)

@@ -46,7 +46,7 @@ namespace {
 constexpr int kSpecMargin = DEFT_SPEC_MARGIN;   // buckets (of 1/16 octave) the speculative cut lies below the predicted b1
 constexpr uint32_t kSpecBudgetPerTile = 64;   // speculative staging stops at this many entries per tile of the CTA
 constexpr int kSpecDensity = 8;
-constexpr uint32_t kSpecCooldown = 8;   // calls without speculation after a call in which a speculative cut failed   // no speculation for layers that select more than 1 / kSpecDensity of their entries
+constexpr uint32_t kSpecCooldown = 4;   // calls without speculation after a call in which a speculative cut failed   // no speculation for layers that select more than 1 / kSpecDensity of their entries
 
 // shared-memory carve-up (bytes)
 constexpr int kSmMain = 0;   // A: kSlots level-1 histograms, then resident entries | direct: keys
@@ -54,9 +54,11 @@ constexpr int kSmMainBytes = 128 * 1024;
 constexpr int kSmRes = kSmMain + kSlots * kBins1 * 4;   // resident staged entries (live from step A on)
 static_assert(kSlots * kBins1 * 4 + kResident * 8 <= kSmMainBytes && kDirectElems * 4 <= kSmMainBytes &&
               3 * (kMaxWeightedLayers + 1) * 4 <= kSmMainBytes, "main region");
-constexpr int kSmAux = kSmMain + kSmMainBytes;   // direct layers: their histograms
+constexpr int kSmAux = kSmMain + kSmMainBytes;   // B: level-2 slots | S2: level-3 slots | direct: its histograms
 constexpr int kSmAuxBytes = 20 * 1024;
-static_assert(kDBins1 * 4 + kDBins2 * 4 <= kSmAuxBytes && kDBins2 >= kDBins3, "aux region");
+constexpr int kH2Slots = 4, kH3Slots = 8;        // layers whose level-2 / level-3 histograms are built at once
+static_assert(kH2Slots * kBins2 * 4 <= kSmAuxBytes && kH3Slots * kBins3 * 4 <= kSmAuxBytes &&
+              kDBins1 * 4 + kDBins2 * 4 <= kSmAuxBytes && kDBins2 >= kDBins3, "aux region");
 constexpr int kSmTile = kSmAux + kSmAuxBytes;    // per local tile: first entry, entries, counts
 constexpr int kSmTileBytes = kMaxLocalTiles * 10;
 constexpr int kSmLayer = kSmTile + kSmTileBytes; // per local streamed layer, see LayerTable
@@ -309,7 +311,7 @@ __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
 // CTA-wide pass over the CTA's staged entries, in no particular order.  The spilled part is
 // read in batches of kSpillBatch loads per thread so that the pass is not bound by one
 // HBM round trip per entry.
-constexpr int kSpillBatch = 4;
+constexpr int kSpillBatch = 8;
 constexpr int kEmitBatch = 4;
 constexpr uint32_t kThreadEmit = 12;   // tiles with at most this many staged entries are written by one thread
 template <typename F>
@@ -349,7 +351,8 @@ __device__ __forceinline__ uint32_t pick4(uint32_t a, uint32_t b, uint32_t c, ui
 // the vector (the tile has just been loaded: they come from L1 / L2).  wbase: 16 words of
 // shared memory private to the warp.  Returns (first entry, entries).
 __device__ __noinline__ uint2 stage_marked(const uint32_t* __restrict__ tile, uint32_t k0, uint32_t k1, uint2* res,
-                                           uint2* spill, uint32_t ytag, uint32_t* cursor, uint32_t* wbase) {
+                                           uint2* spill, uint32_t ytag, uint32_t* cursor, uint32_t* wbase,
+                                           uint32_t* h2, uint32_t b1) {
     const int lane = threadIdx.x & 31;
     // per-load counts of this lane, 8 bits each, four loads per word; scanned over the lanes
     uint32_t excl[4], tot[4];
@@ -375,13 +378,30 @@ __device__ __noinline__ uint2 stage_marked(const uint32_t* __restrict__ tile, ui
     unsigned long long m = (unsigned long long)k0 | ((unsigned long long)k1 << 32);
     const unsigned long long all = m;
     while (m) {
-        const int bit = __ffsll((long long)m) - 1;
-        m &= m - 1;
-        const int i = bit >> 2, c = bit & 3;
-        const uint32_t before_lanes = (pick4(excl[0], excl[1], excl[2], excl[3], i >> 2) >> (8 * (i & 3))) & 0xffu;
-        const uint32_t before_mine = __popc((uint32_t)(all >> (4 * i)) & ((1u << c) - 1u));
-        const uint32_t off = (uint32_t)((i * 32 + lane) * 4 + c);
-        stage_put(st, wbase[i] + before_lanes + before_mine, make_uint2(__ldg(tile + off), ytag | off));
+        // up to four of this lane's entries per round: their reloads are in flight together
+        int bit[4];
+        uint32_t bits[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            bit[u] = -1;
+            bits[u] = 0u;
+            if (m) {
+                bit[u] = __ffsll((long long)m) - 1;
+                m &= m - 1;
+                bits[u] = __ldg(tile + (((bit[u] >> 2) * 32 + lane) * 4 + (bit[u] & 3)));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (bit[u] < 0) continue;
+            const int i = bit[u] >> 2, c = bit[u] & 3;
+            const uint32_t before_lanes = (pick4(excl[0], excl[1], excl[2], excl[3], i >> 2) >> (8 * (i & 3))) & 0xffu;
+            const uint32_t before_mine = __popc((uint32_t)(all >> (4 * i)) & ((1u << c) - 1u));
+            const uint32_t off = (uint32_t)((i * 32 + lane) * 4 + c);
+            if (h2 != nullptr && (key_of(bits[u]) >> kShift1) == b1)   // second read: b1 is known, feed level 2 on the way
+                atomicAdd(&h2[(key_of(bits[u]) >> kShift2) & (kBins2 - 1)], 1u);
+            stage_put(st, wbase[i] + before_lanes + before_mine, make_uint2(bits[u], ytag | off));
+        }
     }
     __syncwarp();   // wbase is rewritten by the warp's next tile
     return make_uint2(first, n);
@@ -401,7 +421,7 @@ __device__ __forceinline__ void mark_tile(const TileRegs& t, const uint32_t (&vm
 template <bool kHist>
 __device__ __forceinline__ uint2 read_tile(const float* __restrict__ acc, const TileSpan& ts, uint32_t* h,
                                            uint32_t thr, const Stage& st, uint32_t ytag, uint32_t* cursor,
-                                           uint32_t* wbase, int lane) {
+                                           uint32_t* wbase, int lane, uint32_t* h2 = nullptr, uint32_t b1 = 0) {
     TileRegs t;
     uint32_t vm[2];
     load_tile(acc, ts, lane, t, vm);
@@ -420,7 +440,7 @@ __device__ __forceinline__ uint2 read_tile(const float* __restrict__ acc, const 
     mark_tile(t, vm, thr, keep);
     if (!__any_sync(0xffffffffu, (keep[0] | keep[1]) != 0)) return make_uint2(0u, 0u);
     return stage_marked(reinterpret_cast<const uint32_t*>(acc + ts.lo), keep[0], keep[1], st.res, st.spill, ytag,
-                        cursor, wbase);
+                        cursor, wbase, h2, b1);
 }
 
 // ---------------------------------------------------------------------------------
@@ -729,6 +749,7 @@ __device__ __forceinline__ void step_read2(const SelParams& p, const CtaRange& r
         }
         __syncthreads();
     }
+    uint32_t* h2 = reinterpret_cast<uint32_t*>(smem + kSmAux);
     if (misc[kMFlag]) {   // uniform over the CTA: drop what was staged, read the CTA's tiles with the true cuts
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -736,32 +757,57 @@ __device__ __forceinline__ void step_read2(const SelParams& p, const CtaRange& r
             if (!p.fixed_thr && misc[kMTried]) atomicAdd(p.spec_ctl + 1, 1u);   // a speculative cut failed
         }
         __syncthreads();
-        int la, lb;
-        if (nl > 0) {
-            local_span(r, lt, 0, nl - 1, la, lb);
-            int c = 0;
+        // kH2Slots layers at a time: their level-2 histograms are built in the same pass
+        for (int c0 = 0; c0 < nl; c0 += kH2Slots) {
+            const int ns = nl - c0 < kH2Slots ? nl - c0 : kH2Slots;
+            for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) h2[i] = 0;
+            __syncthreads();
+            int la, lb;
+            local_span(r, lt, c0, c0 + ns - 1, la, lb);
+            int c = c0;
             for (int lq = la + warp; lq < lb; lq += kSelWarps) {
                 const int q = local_tile(p, r, lq);
                 if (q < 0) continue;
-                const int cl = tile_layer(lt, nl, q, c);
+                const int cl = tile_layer(lt, c0 + ns, q, c);
                 if (cl < 0) continue;
                 const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
                 const uint2 fn = read_tile<false>(p.acc, ts, nullptr, lt->sthr[cl], st,
                                                   pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
-                                                  wbase + 16 * warp, lane);
+                                                  wbase + 16 * warp, lane,
+                                                  p.fixed_thr ? nullptr : h2 + (cl - c0) * kBins2, lt->v0[cl]);
                 if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
             }
+            __syncthreads();
+            if (!p.fixed_thr) {
+                for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) {
+                    const uint32_t cnt = h2[i];
+                    if (cnt) atomicAdd(p.hist2 + (size_t)lt->lid[c0 + i / kBins2] * kBins2 + (i % kBins2), cnt);
+                }
+                __syncthreads();
+            }
+        }
+        return;
+    }
+    if (p.fixed_thr) return;
+    // level-2 histograms of the staged entries of bucket b1: kH2Slots layers at a time in shared memory
+    const uint32_t total = misc[kMCursor];
+    for (int c0 = 0; c0 < nl; c0 += kH2Slots) {
+        const int ns = nl - c0 < kH2Slots ? nl - c0 : kH2Slots;
+        for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) h2[i] = 0;
+        __syncthreads();
+        for_each_staged(st, total, [&](const uint2 ent) {
+            const int c = (int)y_layer(ent.y);
+            const uint32_t key = key_of(ent.x);
+            if (c >= c0 && c < c0 + ns && (key >> kShift1) == lt->v0[c])
+                atomicAdd(&h2[(c - c0) * kBins2 + ((key >> kShift2) & (kBins2 - 1))], 1u);
+        });
+        __syncthreads();
+        for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) {
+            const uint32_t cnt = h2[i];
+            if (cnt) atomicAdd(p.hist2 + (size_t)lt->lid[c0 + i / kBins2] * kBins2 + (i % kBins2), cnt);
         }
         __syncthreads();
     }
-    if (p.fixed_thr) return;
-    const uint32_t total = misc[kMCursor];
-    for_each_staged(st, total, [&](const uint2 ent) {
-        const int c = (int)y_layer(ent.y);
-        const uint32_t key = key_of(ent.x);
-        if ((key >> kShift1) == lt->v0[c])
-            atomicAdd(p.hist2 + (size_t)lt->lid[c] * kBins2 + ((key >> kShift2) & (kBins2 - 1)), 1u);
-    });
 }
 
 // ---------------------------------------------------------------------------------
@@ -783,13 +829,25 @@ __device__ __forceinline__ void step_hist3(const SelParams& p, LayerTable* lt, i
         }
     }
     __syncthreads();
-    // the candidates of bucket (b1, b2) are a small fraction of k: straight to the global histograms
-    for_each_staged(st, total, [&](const uint2 ent) {
-        const int c = (int)y_layer(ent.y);
-        const uint32_t key = key_of(ent.x);
-        if ((key >> kShift2) == lt->v0[c])
-            atomicAdd(p.hist3 + (size_t)lt->lid[c] * kBins3 + (key & (kBins3 - 1)), 1u);
-    });
+    // level-3 histograms of the staged entries of bucket (b1, b2): kH3Slots layers at a time
+    uint32_t* h3 = reinterpret_cast<uint32_t*>(smem + kSmAux);
+    for (int c0 = 0; c0 < nl; c0 += kH3Slots) {
+        const int ns = nl - c0 < kH3Slots ? nl - c0 : kH3Slots;
+        for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) h3[i] = 0;
+        __syncthreads();
+        for_each_staged(st, total, [&](const uint2 ent) {
+            const int c = (int)y_layer(ent.y);
+            const uint32_t key = key_of(ent.x);
+            if (c >= c0 && c < c0 + ns && (key >> kShift2) == lt->v0[c])
+                atomicAdd(&h3[(c - c0) * kBins3 + (key & (kBins3 - 1))], 1u);
+        });
+        __syncthreads();
+        for (int i = threadIdx.x; i < ns * kBins3; i += kSelThreads) {
+            const uint32_t cnt = h3[i];
+            if (cnt) atomicAdd(p.hist3 + (size_t)lt->lid[c0 + i / kBins3] * kBins3 + (i % kBins3), cnt);
+        }
+        __syncthreads();
+    }
 }
 
 // ---------------------------------------------------------------------------------

@@ -293,6 +293,11 @@ DEFT_API deft_status deft_plan_upload(const void* plan_h, void* plan_d, void* ws
  * (the rank's own output; out_cap entries available).  A rank without layers writes
  * nothing.  plan_h is read on the host for the rank's sizes; plan_d is what the kernel
  * reads.  Errors: INVALID_ARG, CAPACITY (out_cap or workspace), CUDA.
+ *
+ * Speed, not results, depends on the workspace's history: the kernel remembers per layer the
+ * first-level bucket it found and, in the next call on the same workspace, stages everything
+ * above a cut derived from it while it builds the histogram.  If every cut of a CTA turns
+ * out low enough, the CTA never reads its part of the vector a second time.
  */
 DEFT_API deft_status deft_select_planned(const float* acc_d, const void* plan_h, const void* plan_d,
                                          int32_t rank, float* val_d, int64_t* idx_d, int64_t out_cap,

@@ -66,12 +66,14 @@ DEFT_API int32_t deft_last_cuda_error(void);
 /*
  * Diagnostic: when timing_d (DEVICE, 1024 x uint64, zeroed by the caller) is not NULL every
  * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs):
- * [0] kernel start, [1] end of the level-1 histogram step, [2] end of the staging step,
- * [3] level-3 histograms done, [4] per-tile counts done, [5] ordered write done, [6] small
- * layers done; inside the first step [8] histograms zeroed, [9] tiles read, [10] flushed,
- * [11] tickets taken; [14] / [15] staged entries (max over CTAs / total); [16 + b],
- * [176 + b], [336 + b] per CTA b: staging-step nanoseconds, staged entries, local layers |
- * local tiles << 16.  Pass NULL to switch it off.  Not thread-safe; not for production use.
+ * [0] kernel start, [1] end of the first read (level-1 histogram + speculative staging),
+ * [2] end of the second read / level-2 histograms, [3] level-3 histograms done, [4] per-tile
+ * counts done, [5] ordered write done, [6] small layers done; inside the first step
+ * [8] histograms zeroed, [9] tiles read, [10] flushed, [11] tickets taken; [14] / [15] staged
+ * entries (max over CTAs / total); per CTA b: [16 + b] nanoseconds in the second step,
+ * [176 + b] staged entries, [336 + b] local layers | local tiles << 16 | read-twice flag << 32,
+ * [656 + b] nanoseconds in the ordered write, [816 + b] nanoseconds in the first read.
+ * Pass NULL to switch it off.  Not thread-safe; not for production use.
  */
 DEFT_API void deft_debug_select_timing(void* timing_d);
 

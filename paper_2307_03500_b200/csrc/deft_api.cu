@@ -98,7 +98,21 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
                 D.out_off += ri[r].out_off;
                 all.push_back(D);
             }
-        std::sort(all.begin(), all.end(), [](const LayerDesc& a, const LayerDesc& b) { return a.start < b.start; });
+        auto by_start = [](const LayerDesc& a, const LayerDesc& b) { return a.start < b.start; };
+        if ((int64_t)all.size() == (int64_t)L) {   // layer ids that are address order: place, do not sort
+            std::vector<LayerDesc> placed((size_t)L);
+            std::vector<char> seen((size_t)L, 0);
+            bool ok = true;
+            for (const LayerDesc& D : all) {
+                if (D.layer_id < 0 || D.layer_id >= L || seen[D.layer_id]) { ok = false; break; }
+                seen[D.layer_id] = 1;
+                placed[D.layer_id] = D;
+            }
+            if (ok && std::is_sorted(placed.begin(), placed.end(), by_start)) all.swap(placed);
+            else std::sort(all.begin(), all.end(), by_start);
+        } else {
+            std::sort(all.begin(), all.end(), by_start);
+        }
         bool disjoint = (int64_t)all.size() <= (int64_t)L;
         for (size_t i = 1; i < all.size() && disjoint; ++i) disjoint = all[i].start >= all[i - 1].end;
         M.desc_first = (int32_t)d;
@@ -309,6 +323,7 @@ static deft_status plan_build_impl(const int64_t* layer_start_h, const int64_t* 
         iteration < 0)
         return DEFT_ERR_INVALID_ARG;
     std::vector<std::vector<LayerItem>> ranks((size_t)N);
+    for (auto& v : ranks) v.reserve((size_t)(L / N + 8));
     const int32_t cycle = (int32_t)(iteration % N);
     for (int32_t l = 0; l < L; ++l) {
         const int32_t b = bin_of_layer_h[l];

@@ -63,7 +63,7 @@ constexpr int kSmTile = kSmAux + kSmAuxBytes;    // per local tile: first entry,
 constexpr int kSmTileBytes = kMaxLocalTiles * 10;
 constexpr int kSmLayer = kSmTile + kSmTileBytes; // per local streamed layer, see LayerTable
 constexpr int kSmLayerBytes = kMaxLocalLayers * 64;   // >= sizeof(LayerTable)
-constexpr int kSmPref = kSmLayer + kSmLayerBytes;   // S4: totals / prefixes of the runs of 32 tiles of one layer
+constexpr int kSmPref = kSmLayer + kSmLayerBytes;   // prefixes of one batch of tiles in S4
 constexpr int kSmPrefBytes = kSelThreads * 8;
 constexpr int kSmMisc = kSmPref + kSmPrefBytes;
 constexpr int kSmMiscBytes = 1024;
@@ -312,6 +312,8 @@ __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
 // read in batches of kSpillBatch loads per thread so that the pass is not bound by one
 // HBM round trip per entry.
 constexpr int kSpillBatch = 8;
+constexpr int kEmitBatch = 4;
+constexpr uint32_t kThreadEmit = 12;   // tiles with at most this many staged entries are written by one thread
 
 template <typename F>
 __device__ __forceinline__ void for_each_staged(const Stage& st, uint32_t total, F f) {
@@ -675,38 +677,13 @@ __device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r
         stamp(p, 8);
         int la, lb;
         local_span(r, lt, c0, c0 + ns - 1, la, lb);
-        // The warp's tiles, software-pipelined: as soon as a tile's registers have been consumed
-        // (histogram, marks) the next tile's loads are issued, and the staging of the marked
-        // entries — which reads them again from L1 / L2 — runs while those loads are in flight.
         int c = c0;
-        int lq = la + warp - kSelWarps, cl = -1;
-        TileSpan ts;
-        auto next_tile = [&]() {   // advances (lq, cl, ts) to the warp's next tile; false when there is none
-            for (lq += kSelWarps; lq < lb; lq += kSelWarps) {
-                const int q = local_tile(p, r, lq);
-                if (q < 0) continue;
-                cl = tile_layer(lt, c0 + ns, q, c);
-                if (cl < 0) continue;
-                ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-                return true;
-            }
-            return false;
-        };
-        TileRegs t;
-        uint32_t vm[2];
-        bool have = next_tile();
-        if (have) load_tile(p.acc, ts, lane, t, vm);
-        while (have) {
-            uint32_t* h = hist + (cl - c0) * kBins1;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                atomicAdd(&h[key_of(t.v[i].x) >> kShift1], 1u);
-                atomicAdd(&h[key_of(t.v[i].y) >> kShift1], 1u);
-                atomicAdd(&h[key_of(t.v[i].z) >> kShift1], 1u);
-                atomicAdd(&h[key_of(t.v[i].w) >> kShift1], 1u);
-            }
-            // the components outside the layer were loaded as zeros
-            if (lane == 0 && ts.e - ts.s != kTile) atomicSub(&h[0], (uint32_t)(kTile - (ts.e - ts.s)));
+        for (int lq = la + warp; lq < lb; lq += kSelWarps) {
+            const int q = local_tile(p, r, lq);
+            if (q < 0) continue;
+            const int cl = tile_layer(lt, c0 + ns, q, c);
+            if (cl < 0) continue;
+            const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
             // a cut that turns out far too low must not flood the staging area: past the budget the
             // CTA stops staging and reads a second time in step B
             uint32_t thr = lt->sthr[cl];
@@ -714,18 +691,10 @@ __device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r
                 thr = 0xffffffffu;
                 if (lane == 0) misc[kMFlag] = 1u;
             }
-            uint32_t keep[2];
-            mark_tile(t, vm, thr, keep);
-            const uint32_t* tile = reinterpret_cast<const uint32_t*>(p.acc + ts.lo);
-            const uint32_t ytag = pack_y(0u, (uint32_t)cl, (uint32_t)lq);
-            const int lq_cur = lq;
-            have = next_tile();
-            if (have) load_tile(p.acc, ts, lane, t, vm);          // in flight during the staging below
-            uint2 fn = make_uint2(0u, 0u);
-            if (__any_sync(0xffffffffu, (keep[0] | keep[1]) != 0))
-                fn = stage_marked_body(tile, keep[0], keep[1], st.res, st.spill, ytag, misc + kMCursor,
-                                       wbase + 16 * warp, nullptr, 0u);
-            if (lane == 0) { tt->first[lq_cur] = fn.x; tt->n[lq_cur] = (uint16_t)fn.y; }
+            const uint2 fn = read_tile<true>(p.acc, ts, hist + (cl - c0) * kBins1, thr, st,
+                                             pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
+                                             wbase + 16 * warp, lane);
+            if (lane == 0) { tt->first[lq] = fn.x; tt->n[lq] = (uint16_t)fn.y; }
         }
         __syncthreads();
         stamp(p, 9);
@@ -971,59 +940,70 @@ __device__ __forceinline__ void emit_batch(const EmitOut& p, int64_t out_off, in
 // ---------------------------------------------------------------------------------
 // step S4: totals of the tiles before this CTA's, scan of the own tiles, ordered write
 // ---------------------------------------------------------------------------------
-// One warp writes the selected entries of a RUN of up to 32 consecutive tiles of a layer (local
-// tiles lq0 .. lq0 + nt - 1, tile ids q_first ..).  Consecutive tiles hold consecutive index
-// ranges and every tile's staged entries are in index order, so the run's entries, tile after
-// tile, are in index order: the warp walks them 32 at a time, whatever tile they come from, and
-// every output position is the count of selected entries before it.  gt_before / eq_before:
-// entries above / equal to T that precede the run in the layer.
-__device__ __noinline__ void emit_run(EmitOut out, const TileTable* tt, uint2* res, uint2* spill, int lq0, int nt,
-                                      int64_t lo_first, int64_t out_off, uint32_t T, uint32_t need,
-                                      uint32_t gt_before, uint32_t eq_before) {
-    const int lane = threadIdx.x & 31;
+// One batch of local tiles [t0, tend): pref[lq - t0] = entries above / equal to T that precede
+// tile lq in its layer.  One warp per tile writes the tile's selected entries.
+__device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, const TileTable* tt, uint2* res,
+                                        uint2* spill, const uint2* pref, int t0, int tend, int64_t start, int tf,
+                                        int64_t out_off, uint32_t T, uint32_t need) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Stage st{res, spill};
-    const uint32_t n_l = lane < nt ? tt->n[lq0 + lane] : 0u;          // lane <-> tile of the run
-    const uint32_t first_l = lane < nt ? tt->first[lq0 + lane] : 0u;
-    const uint32_t incl = warp_incl_scan(n_l, lane);
-    const uint32_t off_l = incl - n_l;                                  // entries of the run before this tile
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    constexpr int kU = 4;   // batches of 32 entries whose loads are in flight together
-    for (uint32_t x0 = 0; x0 < total; x0 += 32 * kU) {
-        uint2 ent[kU];
-        int ti[kU];
+    for (int lq = t0 + warp; lq < tend; lq += kSelWarps) {
+        int q = q0 + lq;
+        if (il) {
+            q = kSuper * ((int)blockIdx.x + (lq / kSuper) * (int)gridDim.x) + lq % kSuper;
+            if (q >= tiles) continue;
+        }
+        const uint32_t n = tt->n[lq];
+        if (n <= kThreadEmit) continue;   // nothing staged, or written by the tile's own thread
+        const uint32_t first = tt->first[lq];
+        const int64_t lo = (start / kTile + (q - tf)) * kTile;
+        uint32_t gt_before = pref[lq - t0].x, eq_before = pref[lq - t0].y;
+        for (uint32_t e0 = 0; e0 < n; e0 += 32 * kEmitBatch) {   // loads of a round are in flight together
+            uint2 ent[kEmitBatch];
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            const uint32_t x = x0 + 32 * u + lane;
-            // the tile of entry x: the last lane whose offset is <= x (empty tiles share the next tile's offset)
-            ti[u] = 0;
-            if (x0 + 32 * u < total) {   // uniform over the warp
+            for (int u = 0; u < kEmitBatch; ++u) {
+                const uint32_t e = e0 + u * 32 + lane;
+                ent[u] = e < n ? stage_get(st, first + e) : make_uint2(0u, 0u);
+            }
 #pragma unroll
-                for (int step = 16; step >= 1; step >>= 1) {
-                    const int cand = ti[u] + step;
-                    const uint32_t o = __shfl_sync(0xffffffffu, off_l, cand & 31);
-                    if (cand < 32 && o <= x) ti[u] = cand;
-                }
-                const uint32_t first_t = __shfl_sync(0xffffffffu, first_l, ti[u]);
-                const uint32_t off_t = __shfl_sync(0xffffffffu, off_l, ti[u]);
-                ent[u] = x < total ? stage_get(st, first_t + (x - off_t)) : make_uint2(0u, 0u);
+            for (int u = 0; u < kEmitBatch; ++u) {
+                if (e0 + u * 32 < n)   // uniform over the warp
+                    emit_batch(out, out_off, lo, e0 + u * 32 + lane < n, ent[u].x, (int64_t)y_off(ent[u].y), T, need,
+                               gt_before, eq_before, lane);
             }
         }
-#pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            if (x0 + 32 * u < total)   // uniform over the warp
-                emit_batch(out, out_off, lo_first + (int64_t)ti[u] * kTile, x0 + 32 * u + lane < total, ent[u].x,
-                           (int64_t)y_off(ent[u].y), T, need, gt_before, eq_before, lane);
+    }
+}
+
+// Tiles with at most kThreadEmit staged entries are written by ONE thread each (thread i of a
+// batch owns tile t0 + i, whose prefix it has just computed): at a few entries per tile a warp
+// per tile leaves most lanes idle and is bound by its own instruction latency.
+__device__ __forceinline__ void emit_small_tile(const EmitOut& out, const Stage& st, uint32_t first, uint32_t n,
+                                                int64_t out_off, int64_t lo, uint32_t T, uint32_t need,
+                                                uint32_t gt_before, uint32_t eq_before) {
+    for (uint32_t e = 0; e < n; ++e) {
+        const uint2 ent = stage_get(st, first + e);
+        const uint32_t key = key_of(ent.x);
+        if (key > T || (key == T && eq_before < need)) {
+            const int64_t pos = out_off + gt_before + (eq_before < need ? eq_before : need);
+            const int64_t elem = lo + (int64_t)y_off(ent.y);
+            if (pos < out.cap) {
+                out.val[pos] = __uint_as_float(ent.x);
+                out.idx[pos] = elem;
+            }
+            if (out.acc_rw) out.acc_rw[elem] = 0.0f;
         }
+        gt_before += key > T;
+        eq_before += key == T;
     }
 }
 
 __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r, LayerTable* lt, int nl,
                                           const TileTable* tt, const Stage& st, unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
-    uint2* runs = reinterpret_cast<uint2*>(smem + kSmPref);   // per run: totals, then prefixes
+    uint2* pref = reinterpret_cast<uint2*>(smem + kSmPref);
     uint32_t* scratch = misc + kMScratch;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const EmitOut out{p.val, p.idx, p.acc_rw, p.out_cap};
     if (r.il) {
         if (nl == 0) return;
         // Prefix at each own super-tile b + mG: the totals of all super-tiles are summed in
@@ -1047,12 +1027,34 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
             if ((int)threadIdx.x < nm) sbase[threadIdx.x] = make_uint2(e_gt + w.x, e_eq + w.y);
         }
         __syncthreads();
-        // one run = one super-tile (consecutive tiles of the layer); sbase[m] = what precedes it
-        for (int m = warp; m < nm; m += kSelWarps) {
-            const int q_first = kSuper * (b + m * G);
-            const int nt = p.tiles - q_first < kSuper ? p.tiles - q_first : kSuper;
-            emit_run(out, tt, st.res, st.spill, m * kSuper, nt, (lt->start[0] / kTile + (q_first - lt->tf[0])) * kTile,
-                     lt->out_off[0], lt->v0[0], lt->v1[0], sbase[m].x, sbase[m].y);
+        const uint32_t T = lt->v0[0], need = lt->v1[0];
+        for (int t0 = 0; t0 < r.nloc; t0 += kSelThreads) {
+            const int i = t0 + (int)threadIdx.x;
+            const uint32_t v = i < r.nloc ? tt->ge[i] : 0u;   // counts <= kTile each: 16 of them fit 16 bits
+            uint32_t incl = v;
+#pragma unroll
+            for (int o = 1; o < kSuper; o <<= 1) {
+                const uint32_t x = __shfl_up_sync(0xffffffffu, incl, o, kSuper);
+                if ((lane & (kSuper - 1)) >= o) incl += x;
+            }
+            const uint32_t ex = incl - v;
+            const uint2 sb = i < r.nloc ? sbase[i / kSuper] : make_uint2(0u, 0u);
+            pref[threadIdx.x] = make_uint2(sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
+            bool big = false;
+            {
+                const int q = i < r.nloc ? local_tile(p, r, i) : -1;
+                const uint32_t n = q >= 0 ? tt->n[i] : 0u;
+                if (n != 0 && n <= kThreadEmit)
+                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, st, tt->first[i], n, lt->out_off[0],
+                                    (lt->start[0] / kTile + (q - lt->tf[0])) * kTile, T, need,
+                                    sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
+                big = n > kThreadEmit;
+            }
+            const int tend = t0 + kSelThreads < r.nloc ? t0 + kSelThreads : r.nloc;
+            if (__syncthreads_or(big ? 1 : 0))   // some tile of the batch needs a warp
+                emit_tiles(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, p.tiles, 1, 0, tt, st.res, st.spill, pref, t0, tend, lt->start[0],
+                       lt->tf[0], lt->out_off[0], T, need);
+            __syncthreads();   // pref is rewritten by the next batch
         }
         return;
     }
@@ -1074,31 +1076,32 @@ __device__ __forceinline__ void step_emit(const SelParams& p, const CtaRange& r,
     for (int c = 0; c < nl; ++c) {
         int ta, tb;
         local_span(r, lt, c, c, ta, tb);
-        // runs of 32 consecutive tiles: totals per run, one scan over the runs (at most 128), one warp per run
-        const int nruns = (tb - ta + 31) / 32;
-        for (int run = warp; run < nruns; run += kSelWarps) {
-            const int i = ta + run * 32 + lane;
+        const uint32_t T = lt->v0[c], need = lt->v1[c];
+        uint32_t base_gt = lt->base_gt[c], base_eq = lt->base_eq[c];
+        for (int t0 = ta; t0 < tb; t0 += kSelThreads) {   // batches of kSelThreads tiles
+            const int i = t0 + (int)threadIdx.x;
             const uint32_t v = i < tb ? tt->ge[i] : 0u;
-            const uint32_t gt = __reduce_add_sync(0xffffffffu, v & 0xffffu);
-            const uint32_t eq = __reduce_add_sync(0xffffffffu, v >> 16);
-            if (lane == 0) runs[run] = make_uint2(gt, eq);
+            uint32_t tot_gt, tot_eq;
+            const uint32_t e_gt = block_excl_scan(v & 0xffffu, scratch, tot_gt);
+            const uint32_t e_eq = block_excl_scan(v >> 16, scratch, tot_eq);
+            pref[threadIdx.x] = make_uint2(base_gt + e_gt, base_eq + e_eq);
+            bool big = false;
+            {
+                const uint32_t n = i < tb ? tt->n[i] : 0u;
+                if (n != 0 && n <= kThreadEmit)
+                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, st, tt->first[i], n, lt->out_off[c],
+                                    (lt->start[c] / kTile + (r.q0 + i - lt->tf[c])) * kTile, T, need,
+                                    base_gt + e_gt, base_eq + e_eq);
+                big = n > kThreadEmit;
+            }
+            const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
+            if (__syncthreads_or(big ? 1 : 0))   // some tile of the batch needs a warp
+                emit_tiles(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, p.tiles, 0, r.q0, tt, st.res, st.spill, pref, t0, tend, lt->start[c],
+                       lt->tf[c], lt->out_off[c], T, need);
+            base_gt += tot_gt;
+            base_eq += tot_eq;
+            __syncthreads();   // pref is rewritten by the next batch
         }
-        __syncthreads();
-        {
-            const uint2 w = (int)threadIdx.x < nruns ? runs[threadIdx.x] : make_uint2(0u, 0u);
-            uint32_t tg, te;
-            const uint32_t e_gt = block_excl_scan(w.x, scratch, tg);
-            const uint32_t e_eq = block_excl_scan(w.y, scratch, te);
-            if ((int)threadIdx.x < nruns) runs[threadIdx.x] = make_uint2(lt->base_gt[c] + e_gt, lt->base_eq[c] + e_eq);
-        }
-        __syncthreads();
-        for (int run = warp; run < nruns; run += kSelWarps) {
-            const int lq0 = ta + run * 32;
-            const int nt = tb - lq0 < 32 ? tb - lq0 : 32;
-            emit_run(out, tt, st.res, st.spill, lq0, nt, (lt->start[c] / kTile + (r.q0 + lq0 - lt->tf[c])) * kTile,
-                     lt->out_off[c], lt->v0[c], lt->v1[c], runs[run].x, runs[run].y);
-        }
-        __syncthreads();   // runs is rewritten by the next layer
     }
 }
 
@@ -1270,6 +1273,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     unsigned long long te0 = 0;
     if (p.timing && threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(te0));
     step_emit(p, r, lt, nl, tt, st, smem);
+    __syncthreads();
     if (p.timing && threadIdx.x == 0) {
         unsigned long long te1;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(te1));

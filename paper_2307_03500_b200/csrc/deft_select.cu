@@ -947,24 +947,40 @@ __device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, 
                                         int64_t out_off, uint32_t T, uint32_t need) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Stage st{res, spill};
-    for (int lq = t0 + warp; lq < tend; lq += kSelWarps) {
-        int q = q0 + lq;
-        if (il) {
-            q = kSuper * ((int)blockIdx.x + (lq / kSuper) * (int)gridDim.x) + lq % kSuper;
-            if (q >= tiles) continue;
-        }
-        const uint32_t n = tt->n[lq];
-        if (n <= kThreadEmit) continue;   // nothing staged, or written by the tile's own thread
-        const uint32_t first = tt->first[lq];
-        const int64_t lo = (start / kTile + (q - tf)) * kTile;
-        uint32_t gt_before = pref[lq - t0].x, eq_before = pref[lq - t0].y;
-        for (uint32_t e0 = 0; e0 < n; e0 += 32 * kEmitBatch) {   // loads of a round are in flight together
-            uint2 ent[kEmitBatch];
-#pragma unroll
-            for (int u = 0; u < kEmitBatch; ++u) {
-                const uint32_t e = e0 + u * 32 + lane;
-                ent[u] = e < n ? stage_get(st, first + e) : make_uint2(0u, 0u);
+    // the warp's next tile that needs a warp: (lq, q) advance, false when there is none
+    int lq = t0 + warp - kSelWarps, q = 0;
+    auto next_tile = [&]() {
+        for (lq += kSelWarps; lq < tend; lq += kSelWarps) {
+            q = q0 + lq;
+            if (il) {
+                q = kSuper * ((int)blockIdx.x + (lq / kSuper) * (int)gridDim.x) + lq % kSuper;
+                if (q >= tiles) continue;
             }
+            if (tt->n[lq] > kThreadEmit) return true;   // the others: nothing staged, or written by their own thread
+        }
+        return false;
+    };
+    auto load_round = [&](uint32_t first, uint32_t n, uint32_t e0, uint2 (&ent)[kEmitBatch]) {
+#pragma unroll
+        for (int u = 0; u < kEmitBatch; ++u) {
+            const uint32_t e = e0 + u * 32 + lane;
+            ent[u] = e < n ? stage_get(st, first + e) : make_uint2(0u, 0u);
+        }
+    };
+    bool have = next_tile();
+    uint2 ent[kEmitBatch];
+    if (have) load_round(tt->first[lq], tt->n[lq], 0u, ent);
+    while (have) {
+        const int lq_cur = lq;
+        const uint32_t n = tt->n[lq_cur], first = tt->first[lq_cur];
+        const int64_t lo = (start / kTile + (q - tf)) * kTile;
+        uint32_t gt_before = pref[lq_cur - t0].x, eq_before = pref[lq_cur - t0].y;
+        // the first round of the warp's next tile is in flight while this tile is written
+        have = next_tile();
+        uint2 ent_next[kEmitBatch];
+        if (have) load_round(tt->first[lq], tt->n[lq], 0u, ent_next);
+        for (uint32_t e0 = 0; e0 < n; e0 += 32 * kEmitBatch) {
+            if (e0) load_round(first, n, e0, ent);
 #pragma unroll
             for (int u = 0; u < kEmitBatch; ++u) {
                 if (e0 + u * 32 < n)   // uniform over the warp
@@ -972,6 +988,8 @@ __device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, 
                                gt_before, eq_before, lane);
             }
         }
+#pragma unroll
+        for (int u = 0; u < kEmitBatch; ++u) ent[u] = ent_next[u];
     }
 }
 

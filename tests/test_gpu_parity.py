@@ -326,6 +326,69 @@ def test_speculative_cut_from_previous_call_never_changes_the_result(deft, scale
     assert np.array_equal(got[1], wsub[1]) and got[0].tobytes() == wsub[0].tobytes()
 
 
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_random_layer_structures(deft, seed):
+    """Random layer tables (tiny, direct-sized, streamed and large layers in any order, unaligned
+    boundaries), random k_l from 1 to the whole layer, a random subset of the layers as the rank,
+    per-layer value distributions from the edge-case generators; every call repeated on the same
+    workspace so that the second one runs with remembered cuts."""
+    rng = np.random.default_rng(1000 + seed)
+    L = int(rng.integers(1, 40))
+    kinds = ["gauss", "wide_exponent", "few_values", "mostly_zero", "all_equal", "bf16_like", "outlier", "denormal"]
+    sizes = []
+    for _ in range(L):
+        c = rng.integers(0, 4)
+        sizes.append(int([rng.integers(1, 100), rng.integers(1000, 20_000), rng.integers(16_000, 17_000),
+                          rng.integers(100_000, 400_000)][c]))
+    if seed % 6 == 0:
+        sizes[int(rng.integers(0, L))] = int(rng.integers(1_500_000, 2_500_000))
+    start = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    x = np.empty(int(start[-1]), dtype=np.float32)
+    for l in range(L):
+        x[start[l]:start[l + 1]] = W.adversarial_vector(kinds[int(rng.integers(0, len(kinds)))], sizes[l],
+                                                        seed=seed * 131 + l) * np.float32(10.0 ** rng.integers(-3, 4))
+    k_l = np.empty(L, dtype=np.int64)
+    for l in range(L):
+        c = rng.integers(0, 4)
+        k_l[l] = [1, sizes[l], max(1, sizes[l] // 100), int(rng.integers(1, sizes[l] + 1))][c]
+    my = np.sort(rng.choice(L, size=int(rng.integers(1, L + 1)), replace=False)).astype(np.int32)
+    acc_d = _dev(x)
+    ws = deft.alloc_workspace(int(start[-1]), L)
+    want = oracle.select_rank(x, start, k_l, my)
+    for rep in range(2):
+        got = _gpu_select(deft, acc_d, start, k_l, my, ws=ws)
+        assert np.array_equal(got[1], want[1]), (seed, rep)
+        assert got[0].tobytes() == want[0].tobytes(), (seed, rep)
+    # the vector changes a little, the cuts remembered from before are reused
+    x2 = x.copy()
+    x2[::3] *= np.float32(1.07)
+    want2 = oracle.select_rank(x2, start, k_l, my)
+    got2 = _gpu_select(deft, _dev(x2), start, k_l, my, ws=ws)
+    assert np.array_equal(got2[1], want2[1]) and got2[0].tobytes() == want2[0].tobytes()
+
+
+def test_nan_and_infinities_sort_by_bit_pattern(deft):
+    """Magnitude order is the IEEE bit pattern with the sign cleared: NaN above infinity above
+    every finite value; the selected values come back bit for bit (payloads, signs)."""
+    n = 70_001
+    x = W.adversarial_vector("gauss", n, seed=77)
+    bits = x.view(np.uint32)
+    bits[5] = 0x7FC00001          # quiet NaN with a payload
+    bits[60_000] = 0xFFC00000     # negative NaN
+    bits[123] = 0x7F800000        # +inf
+    bits[40_000] = 0xFF800000     # -inf
+    bits[999] = 0x7F7FFFFF        # largest finite
+    start = np.array([0, 30_000, n], dtype=np.int64)
+    for k_l in ([1, 1], [2, 3], [30_000, 100]):
+        k_l = np.array(k_l, dtype=np.int64)
+        my = np.array([0, 1], dtype=np.int32)
+        got = _gpu_select(deft, _dev(x), start, k_l, my)
+        want = oracle.select_rank(x, start, k_l, my)
+        assert np.array_equal(got[1], want[1]) and got[0].tobytes() == want[0].tobytes()
+    got = _gpu_select(deft, _dev(x), start, np.array([3, 2], dtype=np.int64), np.array([0, 1], dtype=np.int32))
+    assert sorted(got[1].tolist()) == [5, 123, 999, 40_000, 60_000]
+
+
 def test_select_is_bit_deterministic_run_to_run(deft):
     w = W.scaled_down(W.gpt2_medium(4, 0.01), 16)
     x = w.gradient(0)

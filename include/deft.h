@@ -158,8 +158,9 @@ DEFT_API deft_status deft_bin_layers(const int32_t* bin_of_layer_h, int32_t L, i
 /*
  * Workspace size in bytes that is enough for every device call below on vectors of
  * up to max_elems elements cut into up to max_layers layers.  The workspace must be
- * 256-byte aligned; its contents need not be preserved between calls.  Calls that
- * share a workspace must not overlap on the GPU.
+ * 256-byte aligned.  Its contents need not be preserved between calls (the one area the
+ * library itself carries from call to call, see deft_workspace_init, only affects speed).
+ * Calls that share a workspace must not overlap on the GPU.
  */
 DEFT_API size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers);
 
@@ -241,8 +242,10 @@ DEFT_API deft_status deft_layer_norms_static(float* resid_acc_d, const float* gr
 /*
  * One step's host work in one call: Algorithm 3 (deft_allocate_k on the layer sizes implied by
  * layer_start_h), Algorithm 4 (deft_partition_model with cost_model), deft_plan_build and
- * deft_plan_upload, in that order, with the same results as the four separate calls.  norms_h: HOST [L], this step's
- * norms.  Outputs (HOST): k_l_h [L], *sum_k_out (may be NULL), bin_of_layer_h [L],
+ * deft_plan_upload, in that order, with the same results as the four separate calls; the
+ * plan built here also carries the norms, with which the selection kernel scales the cuts it
+ * remembers (speed only).  norms_h: HOST [L], this step's norms.
+ * Outputs (HOST): k_l_h [L], *sum_k_out (may be NULL), bin_of_layer_h [L],
  * bin_load_h [N] (may be NULL), plan_h (plan_bytes_cap >= deft_plan_bytes(L, N); pinned
  * memory lets the upload overlap).  plan_d / ws_d: DEVICE, as for deft_plan_upload.
  * Returns DEFT_OK or DEFT_WARN_K_INEXACT (PAPER mode, sum of k_l differs from k; the plan is

@@ -341,6 +341,26 @@ DEFT_API deft_status deft_select_update_all(float* acc_d, int64_t n_g, const voi
                                             size_t ws_bytes, void* stream);
 
 /*
+ * One whole step of one worker (Algorithm 1 lines 5-6 and 11-12 with Algorithms 3-5 inside) in
+ * one call: deft_layer_norms (acc = e + grad, norms), the norms' copy to the host, a wait for
+ * them, deft_plan_step (local k, bins, plan, upload) and the selection + residual update —
+ * of worker `rank` (its entries at val_d[0 ..], idx_d[0 ..]), or with rank = -1 of all N
+ * workers in one launch (deft_select_update_all; every worker's entries at its plan offset).
+ * The call returns after the selection has been enqueued; it blocks the host once, between
+ * the norms and the planning.  norms_h: HOST [L] (pinned memory avoids a staging copy).
+ * events: NULL, or 4 cudaEvent_t handles (HOST array) recorded on `stream` before and after
+ * the accumulate+norms kernels and before and after the selection launch.
+ * All other arguments, results and errors as in the calls it is made of.
+ */
+DEFT_API deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, const int64_t* layer_start_h,
+                               const int64_t* layer_start_d, int32_t L, int32_t N, int64_t k, int32_t mode,
+                               int32_t cost_model, int64_t iteration, int32_t rank, double* norms_d,
+                               double* norms_h, int64_t* k_l_h, int64_t* sum_k_out, int32_t* bin_of_layer_h,
+                               double* bin_load_h, void* plan_h, size_t plan_bytes_cap, void* plan_d,
+                               float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
+                               void* const* events, void* stream);
+
+/*
  * Comparison sparsifiers of Section 3 (not part of DEFT; they reuse its selection kernel).
  *
  * Hard-threshold sparsifier (Section 3.2): selects every entry of acc_d[0, n) whose magnitude is

@@ -452,6 +452,41 @@ deft_status deft_select_update_all(float* acc_d, int64_t n_g, const void* plan_h
                                     nullptr, stream);
 }
 
+deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, const int64_t* layer_start_h,
+                      const int64_t* layer_start_d, int32_t L, int32_t N, int64_t k, int32_t mode,
+                      int32_t cost_model, int64_t iteration, int32_t rank, double* norms_d, double* norms_h,
+                      int64_t* k_l_h, int64_t* sum_k_out, int32_t* bin_of_layer_h, double* bin_load_h,
+                      void* plan_h, size_t plan_bytes_cap, void* plan_d, float* val_d, int64_t* idx_d,
+                      int64_t out_cap, void* ws_d, size_t ws_bytes, void* const* events, void* stream) {
+    if (!norms_h || rank < -1 || rank >= N) return DEFT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto mark = [&](int i) -> cudaError_t {
+        return events ? cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st) : cudaSuccess;
+    };
+    DEFT_CUDA_TRY(mark(0));
+    deft_status s = deft_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d, ws_d, ws_bytes, stream);
+    if (s != DEFT_OK) return s;
+    DEFT_CUDA_TRY(mark(1));
+    DEFT_CUDA_TRY(cudaMemcpyAsync(norms_h, norms_d, sizeof(double) * (size_t)L, cudaMemcpyDeviceToHost, st));
+    DEFT_CUDA_TRY(cudaStreamSynchronize(st));   // Algorithms 3 and 4 run on the host and need this step's norms
+    const deft_status sp = deft_plan_step(norms_h, layer_start_h, L, N, k, mode, cost_model, iteration, k_l_h,
+                                          sum_k_out, bin_of_layer_h, bin_load_h, plan_h, plan_bytes_cap, plan_d,
+                                          ws_d, ws_bytes, stream);
+    if (sp < 0) return sp;
+    DEFT_CUDA_TRY(mark(2));
+    if (rank < 0) {
+        s = deft_select_update_all(resid_acc_d, n_g, plan_h, plan_d, val_d, idx_d, out_cap, ws_d, ws_bytes, stream);
+    } else {
+        const RankInfo& R = plan_ranks(plan_h)[rank];
+        if (!val_d || !idx_d) return DEFT_ERR_INVALID_ARG;
+        s = select_rank(resid_acc_d, plan_h, plan_d, rank, val_d, idx_d, out_cap < R.k ? out_cap : R.k, ws_d,
+                        ws_bytes, st, true);
+    }
+    if (s != DEFT_OK) return s;
+    DEFT_CUDA_TRY(mark(3));
+    return sp;   // DEFT_OK, or the Algorithm 3 warning
+}
+
 deft_status deft_select(const float* acc_d, const int64_t* layer_start_h, const int64_t* k_l_h,
                         const int32_t* my_layers_h, int32_t n_my, float* val_d, int64_t* idx_d,
                         int64_t out_cap, void* ws_d, size_t ws_bytes, void* stream) {

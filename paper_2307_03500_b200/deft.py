@@ -80,6 +80,9 @@ def lib() -> ctypes.CDLL:
         L.deft_plan_rank_info.argtypes = [vp, i32, vp, vp, vp, vp]
         L.deft_plan_rank_table.restype = i32
         L.deft_plan_rank_table.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.deft_step.restype = i32
+        L.deft_step.argtypes = [vp, vp, i64, vp, vp, i32, i32, i64, i32, i32, i64, i32, vp, vp, vp, vp, vp, vp, vp, sz,
+                                vp, vp, vp, i64, vp, sz, vp, vp]
         L.deft_workspace_init.restype = i32
         L.deft_workspace_init.argtypes = [vp, sz, i32, vp]
         L.deft_threshold_select.restype = i32
@@ -369,6 +372,37 @@ def deft_plan_step(norms, layer_start_h, n_workers: int, k: int, mode: int, iter
                                      _dp(ws), ws.numel() * ws.element_size(), _stream(stream)),
                 allow_warn=True)
     return k_l, int(s.value), bins, load, st
+
+
+def deft_step(resid_acc, grad, layer_start_h, layer_start_d, n_workers: int, k: int, mode: int, cost_model: int,
+              iteration: int, rank: int, norms_d, norms_h_pinned, k_l_out: np.ndarray, bins_out: np.ndarray,
+              load_out: np.ndarray, plan_h: np.ndarray, plan_d, val_d, idx_d, ws, events=None, stream=None):
+    """One whole step in one C call (rank = -1: all workers in one launch).  The output arrays
+    (k_l_out int64[L], bins_out int32[L], load_out float64[N]) are filled in place.
+    norms_h_pinned: a (pinned) torch float64 CPU tensor of L.  events: optional 4 torch CUDA events.
+    Returns (sum_k, status)."""
+    import torch
+    ls = _np(layer_start_h, np.int64)
+    L = ls.size - 1
+    ev = None
+    if events is not None:
+        flat = []
+        for e in events:
+            if e.cuda_event == 0:   # torch creates the handle lazily, on first record
+                e.record()
+            flat.append(e.cuda_event)
+        ev = (ctypes.c_void_p * 4)(*flat)
+    s = ctypes.c_int64(0)
+    st = _check("deft_step",
+                lib().deft_step(_dp(resid_acc, torch.float32), None if grad is None else _dp(grad, torch.float32),
+                                resid_acc.numel(), _hp(ls), _dp(layer_start_d, torch.int64), L, int(n_workers), int(k),
+                                int(mode), int(cost_model), int(iteration), int(rank), _dp(norms_d, torch.float64),
+                                ctypes.c_void_p(norms_h_pinned.data_ptr()), _hp(k_l_out), ctypes.byref(s),
+                                _hp(bins_out), _hp(load_out), _hp(plan_h), plan_h.size, _dp(plan_d),
+                                _dp(val_d, torch.float32), _dp(idx_d, torch.int64), min(val_d.numel(), idx_d.numel()),
+                                _dp(ws), ws.numel() * ws.element_size(), ev, _stream(stream)),
+                allow_warn=True)
+    return int(s.value), st
 
 
 def deft_select_planned(acc, plan_h: np.ndarray, plan_d, rank: int, val_d, idx_d, ws, stream=None) -> None:

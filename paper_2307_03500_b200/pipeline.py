@@ -100,6 +100,25 @@ class DeftStep:
     def residual_update(self, acc: torch.Tensor, idx: torch.Tensor) -> None:
         deft.deft_residual_update(acc, idx, idx.numel())
 
+    # -- the whole step in ONE library call ---------------------------------------------------
+    def step_fused(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, rank: int = -1,
+                   events=None) -> StepPlan:
+        """accumulate + norms -> host planning -> selection + residual update, one C call
+        (`deft_step`): all simulated workers in one launch (rank = -1) or one worker."""
+        if not hasattr(self, "_k_l"):
+            self._k_l = np.empty(self.L, dtype=np.int64)
+            self._bins = np.empty(self.L, dtype=np.int32)
+            self._load = np.empty(self.N, dtype=np.float64)
+        sum_k, _ = deft.deft_step(resid, grad, self.layer_start, self.layer_start_d, self.N, self.k, self.mode,
+                                  self.cost_model, iteration, rank, self.norms_d, self.norms_h, self._k_l, self._bins,
+                                  self._load, self.plan_h, self.plan_d, self.val_d, self.idx_d, self.ws, events)
+        n_layers, elems, rank_k, out_off = deft.deft_plan_rank_table(self.plan_h, self.N)
+        off = np.zeros(self.N + 1, dtype=np.int64)
+        off[:-1] = out_off
+        off[-1] = out_off[-1] + rank_k[-1]
+        return StepPlan(self._k_l.copy(), sum_k, self._bins.copy(), self._load.copy(), n_layers, rank_k, elems, off,
+                        self.plan_h)
+
     # -- the whole step for all simulated ranks ---------------------------------------------
     def step(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, events=None,
              per_rank: bool = False):

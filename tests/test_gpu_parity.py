@@ -389,6 +389,43 @@ def test_nan_and_infinities_sort_by_bit_pattern(deft):
     assert sorted(got[1].tolist()) == [5, 123, 999, 40_000, 60_000]
 
 
+def test_whole_step_in_one_call_matches_the_separate_calls(deft):
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.scaled_down(W.bert_large(), 64)
+    N = w.n_workers
+    ds_a = DeftStep(w.sizes, N, w.density)
+    ds_b = DeftStep(w.sizes, N, w.density)
+    e_a = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+    e_b = torch.zeros_like(e_a)
+    for t in range(3):
+        g_d = _dev(w.gradient(t))
+        plan_a, _ = ds_a.step(e_a, g_d, iteration=t)                 # separate calls, all workers in one launch
+        plan_b = ds_b.step_fused(e_b, g_d, iteration=t)              # the same through deft_step
+        torch.cuda.synchronize()
+        assert plan_a.sum_k == plan_b.sum_k and plan_a.k_l.tolist() == plan_b.k_l.tolist()
+        assert plan_a.bin_of_layer.tolist() == plan_b.bin_of_layer.tolist()
+        assert plan_a.bin_load.tobytes() == plan_b.bin_load.tobytes()
+        s = plan_a.sum_k
+        assert torch.equal(ds_a.idx_d[:s], ds_b.idx_d[:s]) and torch.equal(ds_a.val_d[:s], ds_b.val_d[:s])
+        assert torch.equal(e_a, e_b)
+    # one worker only: its entries at the head of the output, only its entries cleared
+    ds_c = DeftStep(w.sizes, N, w.density)
+    e_c = torch.zeros_like(e_a)
+    g_d = _dev(w.gradient(0))
+    r = 3
+    plan_c = ds_c.step_fused(e_c, g_d, iteration=0, rank=r)
+    torch.cuda.synchronize()
+    acc = oracle.accumulate(np.zeros(w.n_g, dtype=np.float32), w.gradient(0))
+    start, _ = oracle.split_layers(w.sizes, N)
+    my = oracle.my_layers(plan_c.bin_of_layer, 0, r, N)
+    want_val, want_idx = oracle.select_rank(acc, start, plan_c.k_l, my)
+    kr = int(plan_c.rank_k[r])
+    assert np.array_equal(ds_c.idx_d[:kr].cpu().numpy(), want_idx)
+    assert ds_c.val_d[:kr].cpu().numpy().tobytes() == want_val.tobytes()
+    acc[want_idx] = 0.0
+    assert e_c.cpu().numpy().tobytes() == acc.tobytes()
+
+
 def test_select_is_bit_deterministic_run_to_run(deft):
     w = W.scaled_down(W.gpt2_medium(4, 0.01), 16)
     x = w.gradient(0)

@@ -553,6 +553,8 @@ def run_ours(args):
                                     "in a call without a usable cut",
                     "bytes_per_launch": all_bytes, "ms_per_launch": all_ms, "bytes_per_elem": 8,
                     "bytes_per_selected": 12, "share_of_step": all_ms / ms_per_step,
+                    "ms_per_launch_mean": float(np.mean(t_all)), "ms_per_launch_max": float(np.max(t_all)),
+                    "launches_above_1p25_median": int((t_all > 1.25 * all_ms).sum()),
                     "achieved_on_bytes_moved": moved_bytes / (all_ms * 1e-3) / 1e9,
                     "frac_on_bytes_moved": moved_bytes / (all_ms * 1e-3) / 1e9 / peak}
         roof_acc = {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,

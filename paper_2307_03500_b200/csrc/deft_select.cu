@@ -8,8 +8,9 @@
 //   A   read 1: per-layer histogram of key bits 30..19 in shared memory, flushed with integer
 //       atomics; the CTA that flushes a layer's last tiles finds the bucket b1 holding the
 //       k-th largest key.  In the same pass every entry at or above a SPECULATIVE cut — the
-//       bucket the previous call found for the layer, lowered by a margin — is moved, in
-//       index order, behind the CTA's staging cursor.
+//       bucket in which the previous call found the layer's (k + max(k/2, 48))-th largest key,
+//       moved by the change of the layer's norm — is moved, in index order, behind the CTA's
+//       staging cursor.
 //   B   a CTA whose cuts were all at or below the true b1 already holds everything it needs
 //       and reads nothing; any other CTA drops what it staged and reads its tiles a second
 //       time with the true cut.  Then the staged entries of bucket b1 feed the level-2
@@ -40,13 +41,14 @@ namespace cg = cooperative_groups;
 namespace deft {
 namespace {
 
-#ifndef DEFT_SPEC_MARGIN
-#define DEFT_SPEC_MARGIN 1
-#endif
-constexpr int kSpecMargin = DEFT_SPEC_MARGIN;   // buckets (of 1/16 octave) the speculative cut lies below the predicted b1
-constexpr uint32_t kSpecBudgetPerTile = 64;   // speculative staging stops at this many entries per tile of the CTA
-constexpr int kSpecDensity = 8;
-constexpr uint32_t kSpecCooldown = 4;   // calls without speculation after a call in which a speculative cut failed   // no speculation for layers that select more than 1 / kSpecDensity of their entries
+// Speculative staging (see the head of this file).  The cut a call leaves for the next one is the
+// first-level bucket of the (k + max(k / 2, kSpecSlack))-th largest key: a margin in rank, so that it
+// adapts to the tail of the layer's distribution and to k (the k-th largest of a handful moves
+// by several buckets from draw to draw, the k-th of a million hardly at all).
+constexpr uint32_t kSpecSlack = 48;
+constexpr uint32_t kSpecBudgetFactor = 6;   // staging stops at this multiple of the entries the CTA has to select
+constexpr int kSpecDensity = 8;             // no speculation for layers that select more than 1 / kSpecDensity of their entries
+constexpr uint32_t kSpecCooldown = 1;       // calls without speculation after a call in which a speculative cut failed
 
 // shared-memory carve-up (bytes)
 constexpr int kSmMain = 0;   // A: kSlots level-1 histograms, then resident entries | direct: keys
@@ -84,6 +86,7 @@ enum MiscOff : int {   // word offsets inside the misc area
     kMCursor = 80,     // 1: staged entries of this CTA
     kMFlag = 96,       // 1: this CTA has to read its tiles again
     kMTried = 97,      // 1: at least one layer of this CTA had a speculative cut
+    kMBudget = 98,     // entries the CTA may stage speculatively
     kMWarpCnt = 128,   // 32: per-warp packed counts (direct layers)
 };
 static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4 && kSlots <= 8, "misc area");
@@ -200,9 +203,10 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratc
 
 // CTA-wide: walks a histogram of `bins` bins (bins / kSelThreads consecutive bins per thread;
 // bins a multiple of kSelThreads) from its top bin down and finds the bucket that holds the
-// k-th largest key.  out[0] = bucket, out[1] = keys strictly above it.  `global`: the histogram
-// is in global memory and was written by other CTAs (read past L1).
-__device__ __noinline__ void block_scan_select(const uint32_t* h, int bins, bool global, uint32_t k,
+// k-th largest key.  out[0] = bucket, out[1] = keys strictly above it; if k2 != k also out[2] =
+// the bucket of the k2-th largest key.  `global`: the histogram is in global memory and was
+// written by other CTAs (read past L1).
+__device__ __noinline__ void block_scan_select(const uint32_t* h, int bins, bool global, uint32_t k, uint32_t k2,
                                                uint32_t* scratch, uint32_t* out) {
     const int per = bins / kSelThreads;
     const int base = bins - per * ((int)threadIdx.x + 1);   // thread order = descending bins
@@ -212,7 +216,7 @@ __device__ __noinline__ void block_scan_select(const uint32_t* h, int bins, bool
     uint32_t sum = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) sum += c[i];
-    if (threadIdx.x == 0) { out[0] = 0; out[1] = 0; }
+    if (threadIdx.x == 0) { out[0] = 0; out[1] = 0; out[2] = 0; }
     uint32_t total;
     const uint32_t excl = block_excl_scan(sum, scratch, total);   // keys in bins above mine
     if (sum != 0 && excl < k && k <= excl + sum) {                // exactly one thread
@@ -222,6 +226,17 @@ __device__ __noinline__ void block_scan_select(const uint32_t* h, int bins, bool
         for (int i = 7; i >= 0; --i) {
             if (!found && i < per) {
                 if (run + c[i] >= k) { out[0] = (uint32_t)(base + i); out[1] = run; found = true; }
+                else run += c[i];
+            }
+        }
+    }
+    if (k2 != k && sum != 0 && excl < k2 && k2 <= excl + sum) {   // the bucket of the k2-th largest key (0 if fewer keys)
+        uint32_t run = excl;
+        bool found = false;
+#pragma unroll
+        for (int i = 7; i >= 0; --i) {
+            if (!found && i < per) {
+                if (run + c[i] >= k2) { out[2] = (uint32_t)(base + i); found = true; }
                 else run += c[i];
             }
         }
@@ -635,7 +650,7 @@ __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRa
             } else if (spec_on && p.desc[j].k * kSpecDensity <= p.desc[j].end - p.desc[j].start) {
                 const uint2 hint = __ldcg(p.hint + p.desc[j].layer_id);
                 if (hint.x != 0 && hint.x <= (uint32_t)kBins1) {
-                    int pb = (int)hint.x - 1 - kSpecMargin;
+                    int pb = (int)hint.x - 1;
                     const float was = __uint_as_float(hint.y), now = (float)p.desc[j].norm;
                     if (was > 0.0f && now > 0.0f && was < 3.0e38f && now < 3.0e38f)
                         pb += (int)floorf(16.0f * log2f(now / was));
@@ -668,8 +683,17 @@ __device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint32_t* wbase = reinterpret_cast<uint32_t*>(smem + kSmWBase);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMFlag] = 0; }
-    const uint32_t budget = (uint32_t)r.nloc * kSpecBudgetPerTile + 1024u;
+    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMFlag] = 0; misc[kMBudget] = 4096u; }
+    __syncthreads();
+    // staging budget: a few times what the CTA's tiles are expected to stage (k_l / size_l of its layers)
+    for (int c = threadIdx.x; c < nl; c += kSelThreads) {
+        const int64_t size = lt->end[c] - lt->start[c];
+        const uint64_t per_tile = ((uint64_t)lt->k[c] * kTile + size - 1) / size;   // selected entries per tile, rounded up
+        const uint64_t want = (uint64_t)own_tiles(p, r, lt, c) * per_tile * kSpecBudgetFactor;
+        atomicAdd(&misc[kMBudget], (uint32_t)(want < 0x3fffffffull ? want : 0x3fffffffull));
+    }
+    __syncthreads();
+    const uint32_t budget = misc[kMBudget] < 0x7fffffffu ? misc[kMBudget] : 0x7fffffffu;
     for (int c0 = 0; c0 < nl; c0 += kSlots) {
         const int ns = nl - c0 < kSlots ? nl - c0 : kSlots;
         for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) hist[i] = 0;
@@ -689,7 +713,10 @@ __device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r
             uint32_t thr = lt->sthr[cl];
             if (*reinterpret_cast<volatile uint32_t*>(misc + kMCursor) > budget) {
                 thr = 0xffffffffu;
-                if (lane == 0) misc[kMFlag] = 1u;
+                if (lane == 0) {
+                    misc[kMFlag] = 1u;
+                    if (p.timing) p.timing[16 + 480 + blockIdx.x] = (1ull << 63) | ((unsigned long long)budget << 32) | (unsigned long long)cl;
+                }
             }
             const uint2 fn = read_tile<true>(p.acc, ts, hist + (cl - c0) * kBins1, thr, st,
                                              pack_y(0u, (uint32_t)cl, (uint32_t)lq), misc + kMCursor,
@@ -719,13 +746,15 @@ __device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r
             const int cl = c0 + s;
             const int lid = lt->lid[cl];
             __threadfence();
-            block_scan_select(p.hist1 + (size_t)lid * kBins1, kBins1, true, lt->k[cl], misc + kMScratch,
+            // besides b1: the bucket of a key some way further down, from which the next call takes its cut
+            const uint32_t kk = lt->k[cl], k_safe = kk + (kk / 2 > kSpecSlack ? kk / 2 : kSpecSlack);
+            block_scan_select(p.hist1 + (size_t)lid * kBins1, kBins1, true, kk, k_safe, misc + kMScratch,
                               misc + kMOut3);
             if (threadIdx.x == 0) {
                 p.state[lid].b1 = misc[kMOut3];
                 p.state[lid].above1 = misc[kMOut3 + 1];
                 // the next call's speculative cut starts from here
-                p.hint[lid] = make_uint2(misc[kMOut3] + 1u, __float_as_uint((float)p.desc[lt->j[cl]].norm));
+                p.hint[lid] = make_uint2(misc[kMOut3 + 2] + 1u, __float_as_uint((float)p.desc[lt->j[cl]].norm));
             }
             __syncthreads();
         }
@@ -751,6 +780,9 @@ __device__ __forceinline__ void step_read2(const SelParams& p, const CtaRange& r
             lt->v1[c] = lt->k[c] - __ldcg(&ls->above1);          // krem1
             const uint32_t need_thr = b1 << kShift1;             // key >= need_thr  <=>  bucket >= b1
             if (lt->sthr[c] > need_thr) {                        // staged too little (or nothing) for this layer
+                if (p.timing && lt->sthr[c] != 0xffffffffu)
+                    p.timing[16 + 480 + blockIdx.x] = ((unsigned long long)lt->lid[c] << 40) | ((unsigned long long)lt->k[c] << 24) |
+                                                      ((unsigned long long)(lt->sthr[c] >> kShift1) << 12) | b1;
                 lt->sthr[c] = need_thr;
                 misc[kMFlag] = 1u;
             }
@@ -1162,7 +1194,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
         }
     }
     __syncthreads();
-    block_scan_select(h1, kDBins1, false, k, scratch, out3);
+    block_scan_select(h1, kDBins1, false, k, k, scratch, out3);
     const uint32_t b1 = out3[0], above1 = out3[1];
     __syncthreads();
     // level 2 inside bucket b1
@@ -1171,7 +1203,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
         if ((key >> kDShift1) == b1) atomicAdd(&h[(key >> kDShift2) & (kDBins2 - 1)], 1u);
     }
     __syncthreads();
-    block_scan_select(h, kDBins2, false, k - above1, scratch, out3);
+    block_scan_select(h, kDBins2, false, k - above1, k - above1, scratch, out3);
     const uint32_t b2 = out3[0];
     const uint32_t krem2 = k - above1 - out3[1];
     __syncthreads();
@@ -1184,7 +1216,7 @@ __device__ __forceinline__ void resolve_direct(const SelParams& p, int j, unsign
         if ((key >> kDShift2) == prefix) atomicAdd(&h[key & (kDBins3 - 1)], 1u);
     }
     __syncthreads();
-    block_scan_select(h, kDBins3, false, krem2, scratch, out3);
+    block_scan_select(h, kDBins3, false, krem2, krem2, scratch, out3);
     const uint32_t T = (prefix << kDShift2) | out3[0];
     const uint32_t need = krem2 - out3[1];
     __syncthreads();

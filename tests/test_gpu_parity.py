@@ -291,10 +291,17 @@ def test_large_multi_layer_rank_cost_weighted_split(deft):
     k_l = np.array([5, 900_000, 100, 10, 8_000, 1, 600_000, 17, 2_499_999], dtype=np.int64)
     my = np.array([0, 1, 2, 3, 4, 6, 7, 8], dtype=np.int32)       # layer 5 belongs to another rank
     acc_d = _dev(x)
-    val, idx = _gpu_select(deft, acc_d, start, k_l, my)
+    ws = deft.alloc_workspace(int(start[-1]), len(sizes))
     want_val, want_idx = oracle.select_rank(x, start, k_l, my)
-    assert np.array_equal(idx, want_idx)
-    assert val.tobytes() == want_val.tobytes()
+    for rep in range(2):        # the second call runs with the cuts remembered from the first
+        val, idx = _gpu_select(deft, acc_d, start, k_l, my, ws=ws)
+        assert np.array_equal(idx, want_idx)
+        assert val.tobytes() == want_val.tobytes()
+    x2 = (x * np.float32(0.97)).astype(np.float32)      # cuts slightly too high for every layer
+    x2[start[0]:start[1]] = x[start[0]:start[1]] * np.float32(3.0)
+    want_val, want_idx = oracle.select_rank(x2, start, k_l, my)
+    val, idx = _gpu_select(deft, _dev(x2), start, k_l, my, ws=ws)
+    assert np.array_equal(idx, want_idx) and val.tobytes() == want_val.tobytes()
 
 
 @pytest.mark.parametrize("scale_first", [1.0, 16.0, 1.0 / 16.0, 1e-6, 1e6])

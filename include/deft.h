@@ -72,7 +72,10 @@ DEFT_API int32_t deft_last_cuda_error(void);
  * [8] histograms zeroed, [9] tiles read, [10] flushed, [11] tickets taken; [14] / [15] staged
  * entries (max over CTAs / total); per CTA b: [16 + b] nanoseconds in the second step,
  * [176 + b] staged entries, [336 + b] local layers | local tiles << 16 | read-twice flag << 32,
- * [656 + b] nanoseconds in the ordered write, [816 + b] nanoseconds in the first read.
+ * [496 + b] why it read twice (bit 63: staging budget << 32 | local layer at which it was
+ * exceeded; else layer id << 40 | k_l << 24 | cut bucket << 12 | true bucket of a cut that
+ * was too high; 0: no remembered cut), [656 + b] nanoseconds in the ordered write,
+ * [816 + b] nanoseconds in the first read.
  * Pass NULL to switch it off.  Not thread-safe; not for production use.
  */
 DEFT_API void deft_debug_select_timing(void* timing_d);

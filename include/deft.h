@@ -350,7 +350,10 @@ DEFT_API deft_status deft_select_update_all(float* acc_d, int64_t n_g, const voi
  * of worker `rank` (its entries at val_d[0 ..], idx_d[0 ..]), or with rank = -1 of all N
  * workers in one launch (deft_select_update_all; every worker's entries at its plan offset).
  * The call returns after the selection has been enqueued; it blocks the host once, between
- * the norms and the planning.  norms_h: HOST [L] (pinned memory avoids a staging copy).
+ * the norms and the planning.  norms_h: HOST [L].  If it is pinned memory the device can write
+ * (cudaHostAlloc / cudaMallocHost), the norms kernel stores the norms there itself and the call
+ * polls for them (at most two seconds, then it falls back) instead of copying and
+ * synchronising the stream; any other host memory takes the copy + synchronise route.
  * events: NULL, or 4 cudaEvent_t handles (HOST array) recorded on `stream` before and after
  * the accumulate+norms kernels and before and after the selection launch.
  * All other arguments, results and errors as in the calls it is made of.

@@ -1,6 +1,7 @@
 // C-ABI entry points of libdeft that touch the GPU: argument checks, the per-step plan
 // (host-built tables of every rank's layers), workspace carve-up and kernel launches.
 #include <algorithm>
+#include <chrono>
 #include <cstring>
 #include <vector>
 
@@ -151,12 +152,15 @@ inline bool plan_ok(const void* plan_h) {
     return plan_h && static_cast<const PlanHeader*>(plan_h)->magic == kPlanMagic;
 }
 
-deft_status upload_plan(const void* plan_h, void* plan_d, void* ws_d, size_t ws_bytes, cudaStream_t stream) {
+// clear = false: the caller has already cleared the per-layer counters on this stream.
+deft_status upload_plan(const void* plan_h, void* plan_d, void* ws_d, size_t ws_bytes, cudaStream_t stream,
+                        bool clear = true) {
     const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
     const WsLayout w = ws_layout(hdr->total_elems, hdr->L, hdr->total_tiles);
     if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
     DEFT_CUDA_TRY(cudaMemcpyAsync(plan_d, plan_h, plan_bytes(hdr->L, hdr->N), cudaMemcpyHostToDevice, stream));
-    DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + w.zero_begin, 0, w.zero_end - w.zero_begin, stream));
+    if (clear)
+        DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + w.zero_begin, 0, w.zero_end - w.zero_begin, stream));
     return DEFT_OK;
 }
 
@@ -341,11 +345,11 @@ deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
     return plan_build_impl(layer_start_h, k_l_h, bin_of_layer_h, nullptr, L, N, iteration, plan_h, plan_bytes_cap);
 }
 
-deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
-                           int64_t k, int32_t mode, int32_t cost_model, int64_t iteration, int64_t* k_l_h,
-                           int64_t* sum_k_out,
-                           int32_t* bin_of_layer_h, double* bin_load_h, void* plan_h, size_t plan_bytes_cap,
-                           void* plan_d, void* ws_d, size_t ws_bytes, void* stream) {
+static deft_status plan_step_impl(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
+                                  int64_t k, int32_t mode, int32_t cost_model, int64_t iteration, int64_t* k_l_h,
+                                  int64_t* sum_k_out, int32_t* bin_of_layer_h, double* bin_load_h, void* plan_h,
+                                  size_t plan_bytes_cap, void* plan_d, void* ws_d, size_t ws_bytes, void* stream,
+                                  bool clear) {
     if (!norms_h || !layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || !plan_d || !ws_d || L < 1)
         return DEFT_ERR_INVALID_ARG;
     std::vector<int64_t> size((size_t)L);
@@ -357,9 +361,18 @@ deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, 
     // the plan also carries the norms: the selection kernel scales its speculative cuts with them
     s = plan_build_impl(layer_start_h, k_l_h, bin_of_layer_h, norms_h, L, N, iteration, plan_h, plan_bytes_cap);
     if (s != DEFT_OK) return s;
-    s = deft_plan_upload(plan_h, plan_d, ws_d, ws_bytes, stream);
+    if (!aligned16(plan_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    s = upload_plan(plan_h, plan_d, ws_d, ws_bytes, static_cast<cudaStream_t>(stream), clear);
     if (s != DEFT_OK) return s;
     return sa;   // DEFT_OK, or the Algorithm 3 warning
+}
+
+deft_status deft_plan_step(const double* norms_h, const int64_t* layer_start_h, int32_t L, int32_t N,
+                           int64_t k, int32_t mode, int32_t cost_model, int64_t iteration, int64_t* k_l_h,
+                           int64_t* sum_k_out, int32_t* bin_of_layer_h, double* bin_load_h, void* plan_h,
+                           size_t plan_bytes_cap, void* plan_d, void* ws_d, size_t ws_bytes, void* stream) {
+    return plan_step_impl(norms_h, layer_start_h, L, N, k, mode, cost_model, iteration, k_l_h, sum_k_out,
+                          bin_of_layer_h, bin_load_h, plan_h, plan_bytes_cap, plan_d, ws_d, ws_bytes, stream, true);
 }
 
 deft_status deft_plan_rank_info(const void* plan_h, int32_t rank, int32_t* n_layers_out,
@@ -463,15 +476,51 @@ deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, cons
     auto mark = [&](int i) -> cudaError_t {
         return events ? cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st) : cudaSuccess;
     };
+    if (!resid_acc_d || !layer_start_d || !norms_d || !ws_d || n_g < 1 || L < 1) return DEFT_ERR_INVALID_ARG;
+    if (!aligned16(resid_acc_d) || (grad_d && !aligned16(grad_d)) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    if (norms_ws_bytes(n_g, L) > ws_bytes) return DEFT_ERR_CAPACITY;
+    // If norms_h is pinned memory the device can write (the usual case), the kernel that finishes
+    // the norms stores them there itself and this thread polls for them: the step then needs no
+    // stream synchronisation, whose wake-up costs tens of microseconds of device idle time.
+    double* mapped = nullptr;
+    {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, norms_h) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer)
+            mapped = static_cast<double*>(at.devicePointer);
+        else
+            (void)cudaGetLastError();
+    }
+    const uint64_t kUnset = 0x7ff8dead00000000ull;   // a NaN pattern no norm can have
+    volatile uint64_t* slots = reinterpret_cast<volatile uint64_t*>(norms_h);
+    if (mapped)
+        for (int32_t l = 0; l < L; ++l) slots[l] = kUnset | (uint32_t)l;
     DEFT_CUDA_TRY(mark(0));
-    deft_status s = deft_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d, ws_d, ws_bytes, stream);
+    deft_status s = launch_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d, static_cast<double*>(ws_d),
+                                       st, mapped);
     if (s != DEFT_OK) return s;
     DEFT_CUDA_TRY(mark(1));
-    DEFT_CUDA_TRY(cudaMemcpyAsync(norms_h, norms_d, sizeof(double) * (size_t)L, cudaMemcpyDeviceToHost, st));
-    DEFT_CUDA_TRY(cudaStreamSynchronize(st));   // Algorithms 3 and 4 run on the host and need this step's norms
-    const deft_status sp = deft_plan_step(norms_h, layer_start_h, L, N, k, mode, cost_model, iteration, k_l_h,
+    // the per-layer counters of the selection are cleared while the host plans
+    const WsLayout wl = ws_layout(1, L, 1);   // the cleared area's place depends on the layer count only
+    if (wl.zero_end > ws_bytes) return DEFT_ERR_CAPACITY;
+    DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + wl.zero_begin, 0, wl.zero_end - wl.zero_begin, st));
+    bool have = false;
+    if (mapped) {
+        const auto t0 = std::chrono::steady_clock::now();
+        for (uint64_t spins = 0;; ++spins) {
+            bool all = true;
+            for (int32_t l = L - 1; l >= 0 && all; --l) all = (slots[l] >> 32) != (kUnset >> 32);
+            if (all) { have = true; break; }
+            if ((spins & 0x3ff) == 0x3ff &&
+                std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2)) break;   // bounded wait
+        }
+    }
+    if (!have) {
+        DEFT_CUDA_TRY(cudaMemcpyAsync(norms_h, norms_d, sizeof(double) * (size_t)L, cudaMemcpyDeviceToHost, st));
+        DEFT_CUDA_TRY(cudaStreamSynchronize(st));   // Algorithms 3 and 4 run on the host and need this step's norms
+    }
+    const deft_status sp = plan_step_impl(norms_h, layer_start_h, L, N, k, mode, cost_model, iteration, k_l_h,
                                           sum_k_out, bin_of_layer_h, bin_load_h, plan_h, plan_bytes_cap, plan_d,
-                                          ws_d, ws_bytes, stream);
+                                          ws_d, ws_bytes, stream, false);
     if (sp < 0) return sp;
     DEFT_CUDA_TRY(mark(2));
     if (rank < 0) {

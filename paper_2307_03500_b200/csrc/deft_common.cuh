@@ -238,7 +238,7 @@ int sm_count();
 // Launchers (each enqueues on `stream` and returns a status).
 deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_g,
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
-                               double* partial_d, cudaStream_t stream);
+                               double* partial_d, cudaStream_t stream, double* norms_host_mapped = nullptr);
 deft_status launch_select(const SelParams& p, cudaStream_t stream);
 deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t count,
                                    cudaStream_t stream);

@@ -105,7 +105,7 @@ k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
 // One CTA per layer: add the layer's partial sums in a fixed order, take the root.
 __global__ void __launch_bounds__(kNormThreads)
 k_norm_finalize(const int64_t* __restrict__ ls, int L, const double* __restrict__ partial,
-                double* __restrict__ norms) {
+                double* __restrict__ norms, double* norms_host) {
     __shared__ double sh[kNormWarps];
     const int l = blockIdx.x;
     const int64_t s = ls[l], e = ls[l + 1];
@@ -115,14 +115,21 @@ k_norm_finalize(const int64_t* __restrict__ ls, int L, const double* __restrict_
         for (int64_t t = t0 + threadIdx.x; t <= t1; t += kNormThreads) acc += partial[t + l];
     }
     const double tot = block_sum(acc, sh);
-    if (threadIdx.x == 0) norms[l] = sqrt(tot);
+    if (threadIdx.x == 0) {
+        const double v = sqrt(tot);
+        norms[l] = v;
+        if (norms_host) {   // mapped host memory a waiting host thread polls: no stream synchronisation needed
+            *reinterpret_cast<volatile double*>(norms_host + l) = v;
+            __threadfence_system();
+        }
+    }
 }
 
 }  // namespace
 
 deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_g,
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
-                               double* partial_d, cudaStream_t stream) {
+                               double* partial_d, cudaStream_t stream, double* norms_host_mapped) {
     const int64_t tiles = (n_g + kTileA - 1) / kTileA;
     const int64_t max_grid = (int64_t)sm_count() * 8;
     const int grid = (int)(tiles < max_grid ? tiles : max_grid);
@@ -133,7 +140,7 @@ deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t 
         k_accum_norms<false><<<grid, kNormThreads, 0, stream>>>(resid_acc_d, nullptr, n_g,
                                                             layer_start_d, L, partial_d, tiles);
     DEFT_CUDA_TRY(cudaGetLastError());
-    k_norm_finalize<<<L, kNormThreads, 0, stream>>>(layer_start_d, L, partial_d, norms_d);
+    k_norm_finalize<<<L, kNormThreads, 0, stream>>>(layer_start_d, L, partial_d, norms_d, norms_host_mapped);
     DEFT_CUDA_TRY(cudaGetLastError());
     return DEFT_OK;
 }

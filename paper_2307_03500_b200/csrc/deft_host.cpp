@@ -154,10 +154,21 @@ deft_status deft_partition_model(const int64_t* layer_size_h, const int64_t* k_l
     for (int32_t l = 0; l < L; ++l)
         if (layer_size_h[l] < 1 || (cost_model == DEFT_COST_EQ3 && k_l_h[l] < 1)) return DEFT_ERR_INVALID_ARG;
 
+    // ln(k) for small k comes from a table filled with std::log itself (same bits, no call)
+    static const std::vector<double> log_small = [] {
+        std::vector<double> t(4096);
+        for (int i = 1; i < 4096; ++i) t[i] = std::log((double)i);
+        return t;
+    }();
     std::vector<double> c(L);
-    for (int32_t l = 0; l < L; ++l)
-        c[l] = cost_model == DEFT_COST_EQ3 ? (double)layer_size_h[l] * std::log((double)k_l_h[l])
-                                           : (double)layer_size_h[l];
+    for (int32_t l = 0; l < L; ++l) {
+        if (cost_model == DEFT_COST_EQ3) {
+            const int64_t kk = k_l_h[l];
+            c[l] = (double)layer_size_h[l] * (kk < 4096 ? log_small[(size_t)kk] : std::log((double)kk));
+        } else {
+            c[l] = (double)layer_size_h[l];
+        }
+    }
     // "largest remaining cost, lowest id on ties" L times = one stable pass over the layers
     // sorted by descending cost; "smallest load, lowest id on ties" = a min-heap on (load, bin).
     // Each bin receives its costs in the same order as in the listing, so the fp64 sums are the same.

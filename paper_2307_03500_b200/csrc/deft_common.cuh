@@ -86,7 +86,7 @@ DEFT_HD inline int weighted_boundary(const uint32_t* Wp, const uint32_t* w, cons
 // Accumulate+norm geometry.
 constexpr int kNormThreads = 256;
 constexpr int kNormWarps = kNormThreads / 32;
-constexpr int kTileA = 8192;         // elements per CTA iteration
+constexpr int kTileA = 8192;         // elements per CTA (one tile each)
 
 // ---------------------------------------------------------------------------------
 // The plan: a position-independent blob built on the host once per step, copied to the

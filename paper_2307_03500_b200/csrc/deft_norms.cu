@@ -131,7 +131,10 @@ deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t 
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
                                double* partial_d, cudaStream_t stream, double* norms_host_mapped) {
     const int64_t tiles = (n_g + kTileA - 1) / kTileA;
-    const int64_t max_grid = (int64_t)sm_count() * 8;
+    // one CTA per tile: the hardware scheduler keeps the SMs evenly busy to the end, which a
+    // resident grid-stride loop did not (0.645 -> 0.600 ms on 333.6 M elements); the loop in the
+    // kernel only matters beyond 2^31 - 1 tiles
+    const int64_t max_grid = 0x7fffffff;
     const int grid = (int)(tiles < max_grid ? tiles : max_grid);
     if (grad_d)
         k_accum_norms<true><<<grid, kNormThreads, 0, stream>>>(resid_acc_d, grad_d, n_g, layer_start_d,

@@ -559,9 +559,9 @@ def run_ours(args):
                     "frac_on_bytes_moved": moved_bytes / (all_ms * 1e-3) / 1e9 / peak}
         roof_acc = {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,
                     "peak": peak, "unit": "GB/s", "frac": acc_gbs / peak, "peak_kind": peak_kind,
-                    "traffic": 11.69 * n_g,
+                    "traffic": 11.66 * n_g,
                     "traffic_note": "per launch, scaled by elements from an ncu capture on 135.9 M elements "
-                                    "(8.00 B/element read + 3.69 written before the kernel ends)",
+                                    "(8.00 B/element read + 3.66 written before the kernel ends)",
                     "bytes_per_launch": acc_bytes, "ms_per_launch": acc_ms, "share_of_step": acc_ms / ms_per_step,
                     "frac_of_nominal_8TBs": acc_gbs / 8000.0}
         sel_dominant = all_ms >= acc_ms

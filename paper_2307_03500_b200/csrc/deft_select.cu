@@ -87,6 +87,7 @@ enum MiscOff : int {   // word offsets inside the misc area
     kMFlag = 96,       // 1: this CTA has to read its tiles again
     kMTried = 97,      // 1: at least one layer of this CTA had a speculative cut
     kMBudget = 98,     // entries the CTA may stage speculatively
+    kMTileCtr = 99,    // next local tile to hand to a warp
     kMWarpCnt = 128,   // 32: per-warp packed counts (direct layers)
 };
 static_assert(kMWarpCnt + 32 <= kSmMiscBytes / 4 && kSlots <= 8, "misc area");
@@ -674,6 +675,15 @@ __device__ __forceinline__ int tile_layer(const LayerTable* lt, int nl, int q, i
     return (q >= lt->tf[c] && q < lt->tfe[c]) ? c : -1;
 }
 
+// The warps of a CTA take its tiles one at a time from a counter in shared memory (in ascending
+// order per warp): a fixed round-robin leaves the warps with the costlier tiles behind at the
+// barrier that ends the loop.
+__device__ __forceinline__ int grab_tile(uint32_t* counter, int lane) {
+    int lq = 0;
+    if (lane == 0) lq = (int)atomicAdd(counter, 1u);
+    return __shfl_sync(0xffffffffu, lq, 0);
+}
+
 // ---------------------------------------------------------------------------------
 // step A: level-1 histograms (kSlots layers at a time) and speculative staging
 // ---------------------------------------------------------------------------------
@@ -697,12 +707,13 @@ __device__ __forceinline__ void step_read1(const SelParams& p, const CtaRange& r
     for (int c0 = 0; c0 < nl; c0 += kSlots) {
         const int ns = nl - c0 < kSlots ? nl - c0 : kSlots;
         for (int i = threadIdx.x; i < ns * kBins1; i += kSelThreads) hist[i] = 0;
-        __syncthreads();
-        stamp(p, 8);
         int la, lb;
         local_span(r, lt, c0, c0 + ns - 1, la, lb);
+        if (threadIdx.x == 0) misc[kMTileCtr] = (uint32_t)la;
+        __syncthreads();
+        stamp(p, 8);
         int c = c0;
-        for (int lq = la + warp; lq < lb; lq += kSelWarps) {
+        for (int lq = grab_tile(misc + kMTileCtr, lane); lq < lb; lq = grab_tile(misc + kMTileCtr, lane)) {
             const int q = local_tile(p, r, lq);
             if (q < 0) continue;
             const int cl = tile_layer(lt, c0 + ns, q, c);
@@ -801,11 +812,12 @@ __device__ __forceinline__ void step_read2(const SelParams& p, const CtaRange& r
         for (int c0 = 0; c0 < nl; c0 += kH2Slots) {
             const int ns = nl - c0 < kH2Slots ? nl - c0 : kH2Slots;
             for (int i = threadIdx.x; i < ns * kBins2; i += kSelThreads) h2[i] = 0;
-            __syncthreads();
             int la, lb;
             local_span(r, lt, c0, c0 + ns - 1, la, lb);
+            if (threadIdx.x == 0) misc[kMTileCtr] = (uint32_t)la;
+            __syncthreads();
             int c = c0;
-            for (int lq = la + warp; lq < lb; lq += kSelWarps) {
+            for (int lq = grab_tile(misc + kMTileCtr, lane); lq < lb; lq = grab_tile(misc + kMTileCtr, lane)) {
                 const int q = local_tile(p, r, lq);
                 if (q < 0) continue;
                 const int cl = tile_layer(lt, c0 + ns, q, c);

@@ -1343,8 +1343,23 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_fused(const SelParams
     }
     stamp(p, 5);
     __syncthreads();
-    for (int j = blockIdx.x; j < p.n_my; j += gridDim.x)
-        if (is_direct(p, j)) resolve_direct(p, j, smem);   // uniform over the CTA
+    if (p.n_my > 2 * (int)gridDim.x) {
+        // many layers: the small ones are handed out one at a time (a counter among the per-layer words
+        // that the plan upload clears), so that the CTAs that come out of the ordered write first take
+        // them and the ones with the most entries do not also finish last here
+        uint32_t* next = &p.state[p.desc[0].layer_id].pad[0];
+        for (;;) {
+            __syncthreads();
+            if (threadIdx.x == 0) misc[kMTileCtr] = atomicAdd(next, 1u);
+            __syncthreads();
+            const int j = (int)misc[kMTileCtr];
+            if (j >= p.n_my) break;
+            if (is_direct(p, j)) resolve_direct(p, j, smem);   // uniform over the CTA
+        }
+    } else {
+        for (int j = blockIdx.x; j < p.n_my; j += gridDim.x)
+            if (is_direct(p, j)) resolve_direct(p, j, smem);   // uniform over the CTA
+    }
     stamp(p, 6);
     if (!p.fixed_thr && threadIdx.x == 0) {
         // the last CTA to finish settles whether the next calls speculate: after a call with a failed

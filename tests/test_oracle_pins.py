@@ -176,6 +176,51 @@ def test_allocate_invariants_and_exact_sum():
                 assert s == k
 
 
+def _exact_repair(k_paper, norms, sizes, k):
+    """The EXACT mode's integer repair restated: shortfall handed out in priority order up to
+    each layer's size; surplus taken back one per layer per round, in priority order, never
+    below 1 (priority = norm descending, equal norms by lower layer id)."""
+    out = list(k_paper)
+    order = sorted(range(len(out)), key=lambda l: (-norms[l], l))
+    rem = k - sum(out)
+    for l in order:
+        add = min(sizes[l] - out[l], max(rem, 0))
+        out[l] += add
+        rem -= add
+    while rem < 0:
+        for l in order:
+            if rem < 0 and out[l] > 1:
+                out[l] -= 1
+                rem += 1
+    return out
+
+
+def test_allocate_exact_repair_follows_priority_order():
+    # PAPER mode is pinned by exact rational arithmetic above; EXACT = PAPER + the repair.  The cases
+    # are built so that the repair fires (many near-zero norms: floor-1 surplus; small sizes under large
+    # norms: size-clamp shortfall) and priority order is a random permutation of id order.
+    rng = np.random.default_rng(17)
+    fired_short = fired_surplus = differs_from_id_order = 0
+    for trial in range(600):
+        L = int(rng.integers(2, 24))
+        norms = np.exp(rng.uniform(-2, 3, size=L))
+        tiny = rng.random(L) < (0.5 if trial % 2 else 0.1)
+        norms[tiny] = rng.choice([0.0, 1e-9, 1e-7], size=int(tiny.sum()))
+        sizes = rng.integers(1, 40, size=L) if trial % 2 == 0 else rng.integers(50, 500, size=L)
+        n_g = int(sizes.sum())
+        k = int(rng.integers(L, n_g + 1))
+        kp, sp = oracle.allocate_k(norms, sizes, k, oracle.MODE_PAPER)
+        ke, se = oracle.allocate_k(norms, sizes, k, oracle.MODE_EXACT)
+        want = _exact_repair(kp.tolist(), norms.tolist(), sizes.tolist(), k)
+        assert ke.tolist() == want and se == k
+        fired_short += sp < k
+        fired_surplus += sp > k
+        # the same repair walked in id order (what a wrong implementation would do)
+        by_id = _exact_repair(kp.tolist(), [0.0] * L, sizes.tolist(), k)
+        differs_from_id_order += by_id != want
+    assert fired_short > 50 and fired_surplus > 50 and differs_from_id_order > 50
+
+
 def test_allocate_special_cases():
     # one layer: min(size, k)
     assert oracle.allocate_k([2.5], [100], 7, oracle.MODE_PAPER)[0].tolist() == [7]

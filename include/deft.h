@@ -46,6 +46,8 @@ typedef int32_t deft_status;
 #define DEFT_ERR_NONFINITE_NORM  -3   /* a norm is NaN, infinite or negative; nothing written    */
 #define DEFT_ERR_CAPACITY        -4   /* an output buffer or the workspace is too small          */
 #define DEFT_ERR_CUDA            -5   /* a CUDA call failed; see deft_last_cuda_error()          */
+#define DEFT_ERR_TOO_LARGE       -6   /* valid arguments, but one selection launch cannot hold them:
+                                         see deft_select_launch_max_elems()                      */
 
 #define DEFT_MODE_PAPER 0  /* Algorithm 3 exactly as listed                                      */
 #define DEFT_MODE_EXACT 1  /* Algorithm 3 followed by an integer repair so that sum k_l == k     */
@@ -54,14 +56,33 @@ typedef int32_t deft_status;
 #define DEFT_COST_EQ3  0   /* cost_l = size_l * ln(k_l): Eq. 3                                     */
 #define DEFT_COST_SIZE 1   /* cost_l = size_l: the bytes a worker scans (no counterpart in the paper) */
 
-/* Largest layer (and largest n for deft_topk_baseline) the selection kernels accept. */
+/* Largest layer a plan accepts (a layer's positions are 32-bit).  What one selection launch can
+ * scan is smaller on today's devices: see deft_select_launch_max_elems(). */
 #define DEFT_MAX_LAYER_ELEMS 2147483647LL
+
+/*
+ * Elements one selection launch can scan on the current CUDA device: every CTA (one per SM) owns
+ * at most 4096 tiles of 2048 elements, so 148 SMs give 1 241 513 984.  A single layer, or the n
+ * of deft_topk_baseline / deft_threshold_select, beyond this returns DEFT_ERR_TOO_LARGE (nothing
+ * launched); so does a call whose share per CTA holds more than 256 layers of more than 16384
+ * elements.  deft_select_update_all answers that status by running one launch per worker.
+ * Host-side query; needs a current device.
+ */
+DEFT_API int64_t deft_select_launch_max_elems(void);
 
 /* Human-readable name of a status code (static string). */
 DEFT_API const char* deft_status_string(deft_status s);
 
 /* The cudaError_t value behind the calling thread's most recent DEFT_ERR_CUDA (0 if none). */
 DEFT_API int32_t deft_last_cuda_error(void);
+
+/*
+ * Diagnostic: single_pass = 0 makes every later selection use the five-step kernel alone (two reads,
+ * or one when its own remembered cuts hold); any other value restores the default, in which calls
+ * whose layers are sparse enough go to the single-pass kernel first.  Results never differ.  Not
+ * thread-safe; for measurements and tests.
+ */
+DEFT_API void deft_debug_select_kernel(int32_t single_pass);
 
 /*
  * Diagnostic: when timing_d (DEVICE, 1024 x uint64, zeroed by the caller) is not NULL every
@@ -176,6 +197,16 @@ DEFT_API size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers);
  * absurdly low cuts, how much it stages).  Errors: INVALID_ARG, CAPACITY, CUDA.
  */
 DEFT_API deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_layers, void* stream);
+
+/*
+ * Diagnostic counters of the single-pass selection kernel, summed over every call on this workspace
+ * since deft_workspace_init: stats_h[0] layers it finished in one read, [1] layers whose remembered
+ * cut failed (too few or far too many entries staged), [2] layers it had no usable cut for (nothing
+ * remembered yet, or too dense); [1] and [2] were handed to the five-step kernel.  [3] is reserved.
+ * stats_h: HOST, 4 x uint64.  Waits for `stream`.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+DEFT_API deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layers, uint64_t* stats_h,
+                                       void* stream);
 
 /*
  * Error-feedback accumulate fused with the per-layer gradient norms —

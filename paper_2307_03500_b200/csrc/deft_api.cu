@@ -11,6 +11,11 @@ namespace deft {
 
 static thread_local int32_t g_last_cuda_error = 0;
 static unsigned long long* g_select_timing = nullptr;
+static bool g_stream_kernel = false;   // deft_debug_select_kernel
+
+// Limits of the single-pass selection kernel (see select_rank).
+constexpr int64_t kStreamMaxK = 65536;              // entries one layer may select
+constexpr int64_t kStreamMaxElems = 600000000;      // elements of one call
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int32_t)e; }
 
@@ -47,15 +52,17 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
     LayerDesc* desc = reinterpret_cast<LayerDesc*>(base + sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)(N + 1));
     std::memset(blob, 0, plan_bytes(L, N));
     int64_t tiles_all = 0, elems_all = 0, k_all = 0;
+    int64_t slots_all = 0;   // staging slots handed out: every layer's region starts on a 128-byte boundary
+    auto slots_of = [](int64_t size) { return (size + kRegionAlign - 1) / kRegionAlign * kRegionAlign; };
     int64_t d = 0;
     for (int64_t r = 0; r < N; ++r) {
         RankInfo& R = ri[r];
         R.desc_first = (int32_t)d;
         R.n_my = (int32_t)ranks[r].size();
         R.tile_base = (int32_t)tiles_all;
-        R.elem_base = elems_all;
+        R.elem_base = slots_all;
         R.out_off = k_all;
-        int64_t tiles = 0, elems = 0, k = 0, prev_end = -1;
+        int64_t tiles = 0, elems = 0, slots = 0, k = 0, prev_end = -1;
         for (const LayerItem& it : ranks[r]) {
             if (it.start < 0 || it.end <= it.start || it.end - it.start > DEFT_MAX_LAYER_ELEMS)
                 return DEFT_ERR_INVALID_ARG;
@@ -66,19 +73,20 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
             D.end = it.end;
             D.k = it.k;
             D.out_off = k;
-            D.elem_off = elems_all + elems;
+            D.elem_off = slots_all + slots;
             D.tile_first = (int32_t)tiles;
             D.layer_id = it.layer_id;
             D.norm = it.norm;
             tiles += (it.end - 1) / kTile - it.start / kTile + 1;
             elems += it.end - it.start;
+            slots += slots_of(it.end - it.start);
             k += it.k;
             prev_end = it.end;
             if (tiles_all + tiles > INT32_MAX) return DEFT_ERR_INVALID_ARG;
         }
         LayerDesc& Z = desc[d++];   // sentinel
         Z.out_off = k;
-        Z.elem_off = elems_all + elems;
+        Z.elem_off = slots_all + slots;
         Z.tile_first = (int32_t)tiles;
         Z.layer_id = -1;
         R.tiles = (int32_t)tiles;
@@ -86,6 +94,7 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
         R.k = k;
         tiles_all += tiles;
         elems_all += elems;
+        slots_all += slots;
         k_all += k;
     }
     // all ranks' layers as one list in address order
@@ -119,17 +128,18 @@ deft_status fill_plan(void* blob, size_t blob_bytes, int32_t L, int64_t iteratio
         M.desc_first = (int32_t)d;
         M.n_my = 0;
         if (disjoint && !all.empty()) {
-            int64_t tiles = 0, elems = 0;
+            int64_t tiles = 0, elems = 0, slots = 0;
             for (LayerDesc& D : all) {
                 D.tile_first = (int32_t)tiles;
-                D.elem_off = elems;
+                D.elem_off = slots;
                 tiles += (D.end - 1) / kTile - D.start / kTile + 1;
                 elems += D.end - D.start;
+                slots += slots_of(D.end - D.start);
                 desc[d++] = D;
             }
             LayerDesc& Z = desc[d++];   // sentinel
             Z.out_off = k_all;
-            Z.elem_off = elems;
+            Z.elem_off = slots;
             Z.tile_first = (int32_t)tiles;
             Z.layer_id = -1;
             M.n_my = (int32_t)all.size();
@@ -193,7 +203,11 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.hist2 = reinterpret_cast<uint32_t*>(ws + w.hist2);
     p.hist3 = reinterpret_cast<uint32_t*>(ws + w.hist3);
     p.spec_ctl = reinterpret_cast<uint32_t*>(ws + w.hint);
-    p.hint = reinterpret_cast<uint2*>(ws + w.hint + 256);
+    p.hint = reinterpret_cast<LayerHint*>(ws + w.hint + 256);
+    p.retry = reinterpret_cast<RetryHeader*>(ws + w.retry);
+    p.retry_desc = reinterpret_cast<LayerDesc*>(ws + w.retry_desc);
+    p.from_retry = 0;
+    p.retry_elem_base = R.elem_base;
     p.runge = reinterpret_cast<uint2*>(ws + w.runge) + 2 * ((size_t)R.tile_base + (size_t)rank);
     p.staging = reinterpret_cast<uint2*>(ws + w.staging);
     p.val = val_d;
@@ -215,7 +229,7 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.interleave = (R.n_my == 1 && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) ? 1 : 0;
     if (p.interleave) {
         const int nsuper = (R.tiles + kSuper - 1) / kSuper;
-        if ((int64_t)((nsuper + p.grid - 1) / p.grid) * kSuper > kMaxLocalTiles) return DEFT_ERR_INVALID_ARG;
+        if ((int64_t)((nsuper + p.grid - 1) / p.grid) * kSuper > kMaxLocalTiles) return DEFT_ERR_TOO_LARGE;
         return launch_select(p, stream);
     }
     // q0[b] = first tile of CTA b, b = 0..grid
@@ -233,7 +247,28 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     };
     std::vector<int> q0((size_t)p.grid + 1);
     for (int b = 0; b <= p.grid; ++b) q0[b] = (int)((int64_t)R.tiles * b / p.grid);
-    if (!within_limits(q0)) return DEFT_ERR_INVALID_ARG;
+    if (!within_limits(q0)) return DEFT_ERR_TOO_LARGE;
+    // The single-pass kernel takes the call when most of what it streams can be speculated on (sparse
+    // layers of moderate k; whether a cut is remembered for them only the device knows: layers without
+    // one go on its retry list, which the same launch works off with the five steps behind a grid barrier).  Its finishing CTA handles a layer alone, so layers that select very many
+    // entries, and calls too large for the retry list's split to stay within a CTA's limits, are left to
+    // the five-step kernel alone.
+    if (!fixed.on && g_stream_kernel) {
+        int64_t streamed = 0, sparse = 0;
+        bool ok = R.elems <= kStreamMaxElems;
+        for (int j = 0; j < R.n_my && ok; ++j) {
+            const int64_t size = hd[j].end - hd[j].start;
+            if (size <= kDirectElems) continue;
+            streamed += size;
+            if (hd[j].k * kSpecDensity <= size) {
+                sparse += size;
+                if (hd[j].k > kStreamMaxK) ok = false;
+            }
+        }
+        if (ok && (streamed == 0 || 2 * sparse >= streamed)) {
+            return launch_select_stream(p, streamed != 0, stream);
+        }
+    }
     if (R.n_my > 1 && R.n_my <= kMaxWeightedLayers && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) {
         const int n = R.n_my;
         std::vector<uint32_t> Wp((size_t)n + 1), wt((size_t)n);
@@ -287,20 +322,37 @@ int32_t deft_last_cuda_error(void) { return g_last_cuda_error; }
 
 void deft_debug_select_timing(void* timing_d) { g_select_timing = static_cast<unsigned long long*>(timing_d); }
 
+int64_t deft_select_launch_max_elems(void) { return (int64_t)sm_count() * kMaxLocalTiles * kTile; }
+
+void deft_debug_select_kernel(int32_t single_pass) { g_stream_kernel = single_pass != 0; }
+
 deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_layers, void* stream) {
     if (!ws_d || n_layers < 1 || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
     const WsLayout w = ws_layout(1, n_layers, 1);   // the kept area's place depends on the layer count only
-    const size_t bytes = 256 + sizeof(uint2) * (size_t)n_layers;
+    const size_t bytes = 256 + sizeof(LayerHint) * (size_t)n_layers;
     if (w.hint + bytes > ws_bytes) return DEFT_ERR_CAPACITY;
     DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + w.hint, 0, bytes, static_cast<cudaStream_t>(stream)));
     return DEFT_OK;
 }
 
+deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layers, uint64_t* stats_h, void* stream) {
+    if (!ws_d || !stats_h || n_layers < 1) return DEFT_ERR_INVALID_ARG;
+    const WsLayout w = ws_layout(1, n_layers, 1);
+    if (w.hint + 256 > ws_bytes) return DEFT_ERR_CAPACITY;
+    uint32_t words[8];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DEFT_CUDA_TRY(cudaMemcpyAsync(words, static_cast<const char*>(ws_d) + w.hint, sizeof(words), cudaMemcpyDeviceToHost, st));
+    DEFT_CUDA_TRY(cudaStreamSynchronize(st));
+    stats_h[0] = words[4];
+    stats_h[1] = words[5];
+    stats_h[2] = words[6];
+    stats_h[3] = words[7];
+    return DEFT_OK;
+}
+
 size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers) {
     if (max_elems < 1 || max_layers < 1) return 0;
-    const size_t a = ws_layout(max_elems, max_layers, max_tiles(max_elems, max_layers)).total;
-    const size_t b = align_up(norms_ws_bytes(max_elems, max_layers), 256);
-    return a > b ? a : b;
+    return ws_layout(max_elems, max_layers, max_tiles(max_elems, max_layers)).total;
 }
 
 deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_g,
@@ -310,9 +362,11 @@ deft_status deft_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_
         return DEFT_ERR_INVALID_ARG;
     if (!aligned16(resid_acc_d) || (grad_d && !aligned16(grad_d)) || !aligned256(ws_d))
         return DEFT_ERR_INVALID_ARG;
-    if (norms_ws_bytes(n_g, L) > ws_bytes) return DEFT_ERR_CAPACITY;
+    const size_t part = ws_layout(n_g, L, 1).norm_partial;   // clear of everything the library keeps across calls
+    if (part + norms_ws_bytes(n_g, L) > ws_bytes) return DEFT_ERR_CAPACITY;
     return launch_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d,
-                              static_cast<double*>(ws_d), static_cast<cudaStream_t>(stream));
+                              reinterpret_cast<double*>(static_cast<char*>(ws_d) + part),
+                              static_cast<cudaStream_t>(stream));
 }
 
 size_t deft_plan_bytes(int32_t L, int32_t N) {
@@ -459,7 +513,7 @@ deft_status deft_select_update_all(float* acc_d, int64_t n_g, const void* plan_h
     if (M.n_my > 0) {
         const deft_status s = select_rank(acc_d, plan_h, plan_d, hdr->N, val_d, idx_d, M.k, ws_d, ws_bytes,
                                           static_cast<cudaStream_t>(stream), true);
-        if (s != DEFT_ERR_INVALID_ARG) return s;   // beyond one launch's limits: one launch per rank instead
+        if (s != DEFT_ERR_TOO_LARGE) return s;   // beyond one launch's limits: one launch per rank instead
     }
     return deft_select_update_ranks(acc_d, n_g, plan_h, plan_d, 0, hdr->N, val_d, idx_d, out_cap, ws_d, ws_bytes,
                                     nullptr, stream);
@@ -478,7 +532,8 @@ deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, cons
     };
     if (!resid_acc_d || !layer_start_d || !norms_d || !ws_d || n_g < 1 || L < 1) return DEFT_ERR_INVALID_ARG;
     if (!aligned16(resid_acc_d) || (grad_d && !aligned16(grad_d)) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
-    if (norms_ws_bytes(n_g, L) > ws_bytes) return DEFT_ERR_CAPACITY;
+    const size_t part = ws_layout(n_g, L, 1).norm_partial;
+    if (part + norms_ws_bytes(n_g, L) > ws_bytes) return DEFT_ERR_CAPACITY;
     // If norms_h is pinned memory the device can write (the usual case), the kernel that finishes
     // the norms stores them there itself and this thread polls for them: the step then needs no
     // stream synchronisation, whose wake-up costs tens of microseconds of device idle time.
@@ -495,8 +550,8 @@ deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, cons
     if (mapped)
         for (int32_t l = 0; l < L; ++l) slots[l] = kUnset | (uint32_t)l;
     DEFT_CUDA_TRY(mark(0));
-    deft_status s = launch_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d, static_cast<double*>(ws_d),
-                                       st, mapped);
+    deft_status s = launch_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d,
+                                       reinterpret_cast<double*>(static_cast<char*>(ws_d) + part), st, mapped);
     if (s != DEFT_OK) return s;
     DEFT_CUDA_TRY(mark(1));
     // the per-layer counters of the selection are cleared while the host plans

@@ -43,6 +43,8 @@ constexpr int kSuper = 16;
 constexpr int kInterleaveTiles = 64;
 
 constexpr int kMaxRanks = 4096;      // workers per plan
+constexpr int kRegionAlign = 16;     // a layer's region of the staging area starts on a multiple of this many entries (128 bytes)
+constexpr int kSpecDensity = 8;      // no speculative cut for layers that select more than 1 / kSpecDensity of their entries
 
 // Cost-weighted split of a large multi-layer rank (second read onwards).  The first read costs
 // the same for every tile; from the staging pass on, a tile costs more the more of its entries
@@ -150,20 +152,45 @@ struct LayerState {                  // per layer, written by the kernels; 64 by
     uint32_t b1, above1;             // level-1 bucket of the k-th key; keys strictly above that bucket
     uint32_t b2, krem2;              // level 2 (inside b1): bucket, and how many still to take inside it
     uint32_t T, need;                // exact threshold key; entries equal to T to take (lowest indices)
-    uint32_t ticket1;                // tiles whose level-1 counts have been flushed
-    uint32_t pad[9];
+    uint32_t ticket1;                // tiles whose first read is complete
+    uint32_t cursor;                 // single-pass kernel: room handed out in the layer's staging region
+    unsigned long long done;         // single-pass kernel: what the CTAs that are through with the layer add up to:
+                                     // tiles << 41 | CTAs that stopped staging << 31 | entries staged
+    uint32_t pad[5];                 // pad[0] of a rank's first layer: next small layer to hand out
+    uint32_t spec_bad;               // five steps: a CTA stopped staging for the layer (its speculative cut counts as failed)
 };
 static_assert(sizeof(LayerState) == 64, "LayerState layout");
+
+// What a selection leaves behind per layer for the next call on the same workspace (the only
+// per-layer data that lives across calls; it steers speed, never results).
+struct LayerHint {                   // 16 bytes
+    uint32_t bucket_p1;              // 1 + first-level bucket of the `rank`-th largest key; 0 = nothing remembered
+    uint32_t norm_bits;              // that call's layer norm (float bits)
+    uint32_t rank;                   // the rank the bucket belongs to (k + margin of that call)
+    uint32_t err;                    // how the predictions have been doing, in 1/16 bucket: running mean of (found -
+                                     // predicted) as int16 in the low half, running mean deviation in the high half
+};
+static_assert(sizeof(LayerHint) == 16, "LayerHint layout");
+
+// Layers the single-pass kernel could not finish (no usable cut, cut too high, too dense) are
+// appended here for a following launch of the five-step kernel on exactly those layers.
+struct RetryHeader {                 // 64 bytes, cleared at plan upload
+    unsigned long long packed;       // layers appended << 32 | their tiles; cleared again by the steps that work the list off
+    uint32_t pad[14];
+};
+static_assert(sizeof(RetryHeader) == 64, "RetryHeader layout");
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Carve-up of the caller's workspace.  Offsets depend only on (elems, L, tiles).
 struct WsLayout {
     size_t plan;                     // scratch device plan for the one-shot calls
-    size_t zero_begin, zero_end;     // [state | hist1 | hist2 | hist3]: cleared at plan upload
-    size_t state, hist1, hist2, hist3;
+    size_t zero_begin, zero_end;     // [retry header | state | hist1 | hist2 | hist3]: cleared at plan upload
+    size_t retry, state, hist1, hist2, hist3;
+    size_t retry_desc;               // (L + 1) layer descriptors of the retry list
+    size_t norm_partial;             // partial sums of the accumulate + norm call (its place depends on L only)
     size_t runge, staging;
-    size_t hint;                     // per layer: what the previous call found (see SelParams::hint); kept across calls
+    size_t hint;                     // 256 bytes of control words, then one LayerHint per layer; kept across calls
     size_t total;
 };
 
@@ -172,16 +199,20 @@ inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
     size_t off = 0;
     w.plan = off;     off += align_up(plan_bytes(L, 1), 256);
     w.zero_begin = off;
+    w.retry = off;    off += 256;
     w.state = off;    off += align_up(sizeof(LayerState) * (size_t)L, 256);
     w.hist1 = off;    off += sizeof(uint32_t) * (size_t)kBins1 * (size_t)L;
     w.hist2 = off;    off += sizeof(uint32_t) * (size_t)kBins2 * (size_t)L;
     w.hist3 = off;    off += sizeof(uint32_t) * (size_t)kBins3 * (size_t)L;
     w.zero_end = off;
-    w.hint = off;     off += 256 + align_up(sizeof(uint2) * (size_t)L, 256);   // control words, then one entry per layer
+    w.hint = off;     off += 256 + align_up(sizeof(LayerHint) * (size_t)L, 256);   // control words, then one entry per layer
+    w.retry_desc = off; off += align_up(sizeof(LayerDesc) * (size_t)(L + 1), 256);
+    w.norm_partial = off; off += align_up(sizeof(double) * (size_t)((elems + kTileA - 1) / kTileA + L + 1), 256);
     const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
     w.runge = off;    off += align_up(sizeof(uint2) * slots, 256);
-    // + slack: the interleaved split rounds a rank up to whole super-tiles
-    w.staging = off;  off += align_up(sizeof(uint2) * ((size_t)elems + 4 * (size_t)kSuper * kTile), 256);
+    // + slack: the interleaved split rounds a rank up to whole super-tiles; a retry list places every
+    // layer at a multiple of kTile entries (up to two tiles more than its size)
+    w.staging = off;  off += align_up(sizeof(uint2) * ((size_t)elems + 4 * (size_t)kSuper * kTile + (2 * (size_t)kTile + kRegionAlign) * (size_t)L), 256);
     w.total = off;
     return w;
 }
@@ -206,11 +237,19 @@ struct SelParams {
     uint32_t* hist1;                 // [L][kBins1]
     uint32_t* hist2;                 // [L][kBins2]
     uint32_t* hist3;                 // [L][kBins3]
-    uint32_t* spec_ctl;              // kept across calls: [0] calls left without speculation, [1] CTAs that had to
-                                     // read twice in this call, [2] CTAs that have finished this call
-    uint2* hint;                     // [L] (first-level bucket of the previous call + 1 or 0 = none, that call's
-                                     // layer norm as float bits); read and updated
-    uint2* runge;                    // this rank's (CTA, layer) pairs (slot = CTA + layer position): totals
+    uint32_t* spec_ctl;              // control words: five steps: [1] CTAs that had to read twice in this call, [2] CTAs
+                                     // that have finished this call, [3] layers whose speculative cut failed in this
+                                     // call, [7] calls in which some cut failed (running total); single-pass kernel,
+                                     // running totals: [4] layers it finished, [5] layers whose cut failed, [6]
+                                     // layers it had no usable cut for
+    LayerHint* hint;                 // [L] what the previous call found; read and updated
+    uint2* runge;                    // five-step kernel: this rank's (CTA, layer) pairs (slot = CTA + layer position):
+                                     // totals.  Single-pass kernel: per tile of the rank (first entry within the layer's
+                                     // staging region, entries)
+    RetryHeader* retry;              // layers left for a following launch, see RetryHeader
+    LayerDesc* retry_desc;           // [L + 1]
+    int32_t from_retry;              // five steps: 1 = the layer list is the retry list (no speculation, no small layers)
+    int64_t retry_elem_base;         // staging index at which the retry list's layers are placed
     uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output
     int64_t* idx;
@@ -240,6 +279,7 @@ deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t 
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
                                double* partial_d, cudaStream_t stream, double* norms_host_mapped = nullptr);
 deft_status launch_select(const SelParams& p, cudaStream_t stream);
+deft_status launch_select_stream(const SelParams& p, bool has_streamed, cudaStream_t stream);
 deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t count,
                                    cudaStream_t stream);
 deft_status launch_gather_update(float* acc_d, const int64_t* idx_d, int64_t count, float* val_d,

@@ -23,6 +23,7 @@ const char* deft_status_string(deft_status s) {
         case DEFT_ERR_NONFINITE_NORM: return "DEFT_ERR_NONFINITE_NORM";
         case DEFT_ERR_CAPACITY: return "DEFT_ERR_CAPACITY";
         case DEFT_ERR_CUDA: return "DEFT_ERR_CUDA";
+        case DEFT_ERR_TOO_LARGE: return "DEFT_ERR_TOO_LARGE";
         default: return "DEFT_UNKNOWN_STATUS";
     }
 }

@@ -22,6 +22,7 @@ ERR_INFEASIBLE_K = -2
 ERR_NONFINITE_NORM = -3
 ERR_CAPACITY = -4
 ERR_CUDA = -5
+ERR_TOO_LARGE = -6
 MODE_PAPER = 0
 MODE_EXACT = 1
 
@@ -52,6 +53,12 @@ def lib() -> ctypes.CDLL:
         L.deft_last_cuda_error.argtypes = []
         L.deft_debug_select_timing.restype = None
         L.deft_debug_select_timing.argtypes = [vp]
+        L.deft_debug_select_kernel.restype = None
+        L.deft_debug_select_kernel.argtypes = [i32]
+        L.deft_select_stats.restype = i32
+        L.deft_select_stats.argtypes = [vp, sz, i32, vp, vp]
+        L.deft_select_launch_max_elems.restype = i64
+        L.deft_select_launch_max_elems.argtypes = []
         L.deft_split_layers.restype = i32
         L.deft_split_layers.argtypes = [vp, i32, i32, vp, vp, i32, vp]
         L.deft_allocate_k.restype = i32
@@ -295,6 +302,21 @@ def deft_select(acc, layer_start_h, k_l_h, my_layers_h, val_d, idx_d, ws, stream
 def deft_debug_select_timing(timing_d) -> None:
     """Diagnostic phase stamps of the selection kernel: a zeroed CUDA uint64/int64 tensor of 1024, or None."""
     lib().deft_debug_select_timing(None if timing_d is None else _dp(timing_d))
+
+
+def deft_debug_select_kernel(single_pass: bool) -> None:
+    lib().deft_debug_select_kernel(1 if single_pass else 0)
+
+
+def deft_select_stats(ws, n_layers: int, stream=None) -> dict:
+    out = np.zeros(4, dtype=np.uint64)
+    _check("deft_select_stats", lib().deft_select_stats(_dp(ws), ws.numel() * ws.element_size(), n_layers,
+                                                        _hp(out), _stream(stream)))
+    return {"one_read": int(out[0]), "cut_failed": int(out[1]), "no_cut": int(out[2])}
+
+
+def deft_select_launch_max_elems() -> int:
+    return int(lib().deft_select_launch_max_elems())
 
 
 def deft_plan_bytes(n_layers: int, n_workers: int) -> int:

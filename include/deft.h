@@ -77,10 +77,11 @@ DEFT_API const char* deft_status_string(deft_status s);
 DEFT_API int32_t deft_last_cuda_error(void);
 
 /*
- * Diagnostic: single_pass = 0 makes every later selection use the five-step kernel alone (two reads,
- * or one when its own remembered cuts hold); any other value restores the default, in which calls
- * whose layers are sparse enough go to the single-pass kernel first.  Results never differ.  Not
- * thread-safe; for measurements and tests.
+ * Diagnostic: which selection kernel later calls use.  single_pass = 0: the five-step kernel alone;
+ * 1: the single-pass kernel whenever a call's layers allow it (sparse layers of moderate k_l, at most
+ * 1024 layers of which at most 256 larger than 16384 elements); -1 (the default): the single-pass
+ * kernel for such calls of 48 M elements or more, the five-step kernel for smaller ones.  Results never
+ * differ.  Not thread-safe; for measurements and tests.
  */
 DEFT_API void deft_debug_select_kernel(int32_t single_pass);
 

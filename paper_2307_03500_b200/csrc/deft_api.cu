@@ -11,11 +11,13 @@ namespace deft {
 
 static thread_local int32_t g_last_cuda_error = 0;
 static unsigned long long* g_select_timing = nullptr;
-static bool g_stream_kernel = false;   // deft_debug_select_kernel
+static int g_stream_kernel = -1;   // deft_debug_select_kernel: -1 by size, 0 never, 1 whenever possible
 
 // Limits of the single-pass selection kernel (see select_rank).
 constexpr int64_t kStreamMaxK = 65536;              // entries one layer may select
 constexpr int64_t kStreamMaxElems = 600000000;      // elements of one call
+constexpr int64_t kStreamMinElems = 48000000;       // below this the five-step kernel is the faster one (measured)
+constexpr int kStreamMaxLayers = 1024;              // layers of one call (its layer map lives in shared memory)
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int32_t)e; }
 
@@ -253,13 +255,17 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     // one go on its retry list, which the same launch works off with the five steps behind a grid barrier).  Its finishing CTA handles a layer alone, so layers that select very many
     // entries, and calls too large for the retry list's split to stay within a CTA's limits, are left to
     // the five-step kernel alone.
-    if (!fixed.on && g_stream_kernel) {
+    if (!fixed.on && (g_stream_kernel > 0 || (g_stream_kernel < 0 && R.elems >= kStreamMinElems))) {
         int64_t streamed = 0, sparse = 0;
-        bool ok = R.elems <= kStreamMaxElems;
+        int n_streamed = 0;
+        // every CTA keeps a table of all streamed layers and a map of all layers; its stripes are tiles / grid tiles
+        bool ok = R.elems <= kStreamMaxElems && R.n_my <= kStreamMaxLayers &&
+                  (int64_t)R.tiles / p.grid + 2 * kSuper <= kMaxLocalTiles;
         for (int j = 0; j < R.n_my && ok; ++j) {
             const int64_t size = hd[j].end - hd[j].start;
             if (size <= kDirectElems) continue;
             streamed += size;
+            if (++n_streamed > kMaxLocalLayers) ok = false;
             if (hd[j].k * kSpecDensity <= size) {
                 sparse += size;
                 if (hd[j].k > kStreamMaxK) ok = false;
@@ -324,7 +330,7 @@ void deft_debug_select_timing(void* timing_d) { g_select_timing = static_cast<un
 
 int64_t deft_select_launch_max_elems(void) { return (int64_t)sm_count() * kMaxLocalTiles * kTile; }
 
-void deft_debug_select_kernel(int32_t single_pass) { g_stream_kernel = single_pass != 0; }
+void deft_debug_select_kernel(int32_t single_pass) { g_stream_kernel = single_pass < 0 ? -1 : (single_pass != 0 ? 1 : 0); }
 
 deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_layers, void* stream) {
     if (!ws_d || n_layers < 1 || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;

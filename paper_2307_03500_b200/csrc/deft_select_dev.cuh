@@ -686,7 +686,7 @@ __device__ __forceinline__ uint32_t safe_rank(uint32_t k) { return k + (k / 2 > 
 // error and twice the deviation (whole buckets, rounded towards zero): a stream whose thresholds drift against the norms, or jump
 // around, gets lower cuts (more staged entries) instead of failed ones; a steady stream gets tight ones.
 constexpr int kErrUnit = 16;          // error bookkeeping in 1/16 bucket
-constexpr int kDevInit = kErrUnit / 2, kDevMin = kErrUnit / 4, kDevMax = 2 * kErrUnit, kBiasMax = 24 * kErrUnit;
+constexpr int kDevInit = kErrUnit / 2, kDevMin = kErrUnit / 4, kDevMax = kErrUnit, kBiasMax = 24 * kErrUnit;
 
 // The predicted bucket (not clamped), or INT_MIN if nothing usable is remembered.
 __device__ __forceinline__ int predict_bucket(const uint4& raw, uint32_t k, double norm) {

@@ -72,11 +72,10 @@ __device__ __noinline__ void push_retry(const SelParams& p, int j) {
 constexpr int kFineShift = 15;
 constexpr int kFineBins = kBins1;   // the top bin takes everything beyond
 constexpr uint32_t kCandMax = 1024; // candidates that can be ranked; a layer with more goes to the retry list
-constexpr uint32_t kBigMax = 1024;  // tiles per pass that can wait for a warp
 constexpr uint32_t kSelFlag = 0x80000000u;   // in an entry's .y: a candidate that is selected
-static_assert(kBigMax * 16 <= kSmAuxBytes && kCandMax * 12 <= kSmAuxBytes && kShift1 > kFineShift &&
+static_assert(kCandMax * 12 <= kSmAuxBytes && kShift1 > kFineShift && kSelWarps == 16 &&
               DEFT_MAX_LAYER_ELEMS / kTile < (1 << 20),
-              "candidates and the list of tiles waiting for a warp live in the aux region; bit 31 of .y is free");
+              "candidates live in the aux region; bit 31 of .y is free; a warp id fits four bits");
 
 __device__ __forceinline__ uint32_t fine_bin(uint32_t key, uint32_t cut) {
     const uint32_t b = (key - cut) >> kFineShift;
@@ -93,6 +92,27 @@ struct Staged {
 };
 __device__ __forceinline__ uint2 staged_get(const Staged& f, uint32_t pos) {
     return pos < kStreamRes ? f.res[pos] : f.src[pos];
+}
+
+// CTA-wide pass over the staged entries in no particular order: f(entry, position).  The part that lives in
+// global memory is read four entries per thread at a time (one round trip per four instead of one each).
+template <typename F>
+__device__ __forceinline__ void for_each_entry(const Staged& f, F fn) {
+    const uint32_t nres = f.S < kStreamRes ? f.S : kStreamRes;
+    for (uint32_t pos = threadIdx.x; pos < nres; pos += kSelThreads) fn(f.res[pos], pos);
+    for (uint32_t p0 = kStreamRes + threadIdx.x; p0 < f.S; p0 += 4 * kSelThreads) {
+        uint2 ent[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t pos = p0 + u * kSelThreads;
+            ent[u] = pos < f.S ? f.src[pos] : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t pos = p0 + u * kSelThreads;
+            if (pos < f.S) fn(ent[u], pos);
+        }
+    }
 }
 
 // Diagnostic lap timer of the finishing CTA: adds the nanoseconds since the previous lap to timing[slot].
@@ -149,17 +169,13 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
 #pragma unroll 4
         for (uint32_t pos = tid; pos < nres; pos += kSelThreads) f.res[pos] = f.src[pos];
 #pragma unroll 4
-        for (int t = tid; t < np0; t += kSelThreads) {
-            const uint2 fn = __ldcg(tab + t);
-            tt->first[t] = fn.x;
-            tt->n[t] = (uint16_t)fn.y;
-        }
+        for (int t = tid; t < np0; t += kSelThreads) tt->first[t] = __ldcg(tab + t).x;
     }
     for (int i = tid; i < kFineBins; i += kSelThreads) h[i] = 0;
-    if (tid == 0) { misc[kMBudget] = 0u; misc[kMFlag] = 0u; }   // tiles listed for the warps; candidates collected
+    if (tid == 0) misc[kMFlag] = 0u;   // candidates collected
     __syncthreads();
     lap.lap(20);
-    for (uint32_t pos = tid; pos < S; pos += kSelThreads) atomicAdd(&h[fine_bin(key_of(staged_get(f, pos).x), cut)], 1u);
+    for_each_entry(f, [&](const uint2 ent, uint32_t) { atomicAdd(&h[fine_bin(key_of(ent.x), cut)], 1u); });
     __syncthreads();
     lap.lap(21);
     block_scan_select(h, kFineBins, false, k, k_safe, scratch, out3);
@@ -175,7 +191,7 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
         }
         return;
     }
-    if (tid == 0) {
+    if (tid == kSelThreads - 1) {   // (not thread 0: the loads it waits for are off the CTA's critical path this way)
         // what the next call starts from: the first-level bucket of the k_safe-th key if that many were
         // staged, else the bucket below this call's cut
         const double norm = p.desc[lt->j[c]].norm;
@@ -191,15 +207,14 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
     uint32_t* ckey = h;
     uint32_t* cy = h + kCandMax;
     uint32_t* cpos = h + 2 * kCandMax;
-    for (uint32_t pos = tid; pos < S; pos += kSelThreads) {
-        const uint2 ent = staged_get(f, pos);
+    for_each_entry(f, [&](const uint2 ent, uint32_t pos) {
         if (fine_bin(key_of(ent.x), cut) == a) {
             const uint32_t i = atomicAdd(misc + kMFlag, 1u);
             ckey[i] = key_of(ent.x);
             cy[i] = ent.y;
             cpos[i] = pos;
         }
-    }
+    });
     __syncthreads();
     for (uint32_t i = tid; i < C; i += kSelThreads) {
         const uint32_t key = ckey[i], y = cy[i];
@@ -213,101 +228,112 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
     __syncthreads();
     stamp(p, 10);
     lap.lap(23);
-    if (p.timing && tid == 0) { atomicMax(p.timing + 14, (unsigned long long)S); atomicAdd(p.timing + 15, (unsigned long long)S); atomicMax(p.timing + 13, (unsigned long long)C); }
-    // per-tile counts, prefix over the layer's tiles, ordered write: up to kMaxLocalTiles tiles per pass,
-    // each thread a run of consecutive tiles.  A tile with few entries is written by its thread, the
-    // others go on a list that the warps work off afterwards.
+    if (p.timing && tid == 0) { atomicMax(p.timing + 14, (unsigned long long)S); atomicAdd(p.timing + 15, (unsigned long long)S); atomicMax(p.timing + 13, (unsigned long long)C); atomicMax(p.timing + 12, ((unsigned long long)S << 32) | ((unsigned long long)lid << 20) | (k < 0xfffffu ? k : 0xfffffu)); }
+    // The ordered write.  An entry's place in the output is (selected entries of the layer's earlier tiles) +
+    // (selected entries before it in its own tile).  A tile's entries are consecutive in the region, so the
+    // second term is a difference of running counts along the region: two passes over the entries, each
+    // warp over a contiguous range of them (32 consecutive entries per step: coalesced, and a ballot gives
+    // the running count).  Pass 1 counts the selected entries per tile and notes the running count at
+    // every tile's first entry; a prefix over the tiles and over the warps' totals; pass 2 writes.
+    // Up to kMaxLocalTiles tiles of the layer per round.
     float* const val = p.val;
     int64_t* const idx = p.idx;
     float* const acc_rw = p.acc_rw;
     const int64_t cap = p.out_cap;
     const int64_t tile0 = lt->start[c] / kTile;
     const int64_t out_off = lt->out_off[c];
-    uint4* big = reinterpret_cast<uint4*>(smem + kSmAux);   // (tile, selected entries before it, -, -)
+    uint32_t* wtot = misc + kMWarpCnt;   // per warp: selected entries of its range, then their exclusive prefix
+    const uint32_t per_warp = ((S + kSelWarps - 1) / kSelWarps + 127u) & ~127u;
+    const uint32_t w_lo = (uint32_t)warp * per_warp < S ? (uint32_t)warp * per_warp : S;
+    const uint32_t w_hi = w_lo + per_warp < S ? w_lo + per_warp : S;
     uint32_t base = 0;
     for (int tp = 0; tp < tn; tp += kMaxLocalTiles) {
         const int np = tn - tp < kMaxLocalTiles ? tn - tp : kMaxLocalTiles;
         if (tp > 0) {
 #pragma unroll 4
-            for (int t = tid; t < np; t += kSelThreads) {
-                const uint2 fn = __ldcg(tab + tp + t);
-                tt->first[t] = fn.x;
-                tt->n[t] = (uint16_t)fn.y;
-            }
-            if (tid == 0) misc[kMBudget] = 0u;
-            __syncthreads();
+            for (int t = tid; t < np; t += kSelThreads) tt->first[t] = __ldcg(tab + tp + t).x;
         }
+        for (int t = tid; t < np; t += kSelThreads) tt->ge[t] = 0u;
+        __syncthreads();
+        // pass 1
+        uint32_t run = 0;
+        for (uint32_t p4 = w_lo; p4 < w_hi; p4 += 128) {   // four steps' entries are fetched together
+            uint2 e4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t pos = p4 + u * 32 + lane;
+                e4[u] = pos < w_hi ? staged_get(f, pos) : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t pos = p4 + u * 32 + lane;
+                const bool valid = pos < w_hi;
+                const uint2 ent = e4[u];
+                const uint32_t t = ((ent.y & ~kSelFlag) >> 11) - (uint32_t)tp;   // tile within this round (or out of it)
+                const bool here = valid && t < (uint32_t)np;
+                const bool sel = here && ((fine_bin(key_of(ent.x), cut) > a) || (ent.y & kSelFlag));
+                const unsigned ball = __ballot_sync(0xffffffffu, sel);
+                if (here && tt->first[t] == pos) tt->first[t] = 0x80000000u | ((uint32_t)warp << 27) | (run + __popc(ball & ((1u << lane) - 1u)));
+                if (sel) atomicAdd(&tt->ge[t], 1u);
+                run += __popc(ball);
+            }
+        }
+        if (lane == 0) wtot[warp] = run;
+        __syncthreads();
+        lap.lap(24);
+        if (warp == 0) {
+            const uint32_t x = lane < kSelWarps ? wtot[lane] : 0u;
+            wtot[lane] = warp_incl_scan(x, lane) - x;
+        }
+        // exclusive prefix of the tiles' counts: each thread a run of consecutive tiles
         const int m = (np + kSelThreads - 1) / kSelThreads;
         const int lo = tid * m < np ? tid * m : np, hi = lo + m < np ? lo + m : np;
         uint32_t mine = 0;
-        for (int t = lo; t < hi; ++t) {
-            const uint32_t first = tt->first[t], n = tt->n[t];
-            uint32_t g = 0;
-            for (uint32_t e = 0; e < n; ++e) {
-                const uint2 ent = staged_get(f, first + e);
-                g += (fine_bin(key_of(ent.x), cut) > a) || (ent.y & kSelFlag);
-            }
-            tt->ge[t] = g;
-            mine += g;
-        }
-        lap.lap(24);
+        for (int t = lo; t < hi; ++t) mine += tt->ge[t];
         uint32_t total;
-        uint32_t run = base + block_excl_scan(mine, scratch, total);
-        lap.lap(25);
+        uint32_t before = base + block_excl_scan(mine, scratch, total);
         for (int t = lo; t < hi; ++t) {
-            const uint32_t first = tt->first[t], n = tt->n[t];
-            if (n != 0) {
-                uint32_t slot = kBigMax;
-                if (n > kThreadEmit) slot = atomicAdd(misc + kMBudget, 1u);
-                if (slot < kBigMax) {
-                    big[slot] = make_uint4((uint32_t)t, run, 0u, 0u);
-                } else {
-                    const int64_t lo_elem = (tile0 + tp + t) * kTile;
-                    int64_t pos = out_off + run;
-                    for (uint32_t e = 0; e < n; ++e) {
-                        const uint2 ent = staged_get(f, first + e);
-                        if ((fine_bin(key_of(ent.x), cut) > a) || (ent.y & kSelFlag)) {
-                            const int64_t elem = lo_elem + (int64_t)y_off(ent.y);
-                            if (pos < cap) {
-                                val[pos] = __uint_as_float(ent.x);
-                                idx[pos] = elem;
-                            }
-                            if (acc_rw) acc_rw[elem] = 0.0f;
-                            ++pos;
-                        }
-                    }
-                }
-            }
-            run += tt->ge[t];
+            const uint32_t g = tt->ge[t];
+            tt->ge[t] = before;
+            before += g;
         }
         __syncthreads();
-        lap.lap(26);
-        const uint32_t nbig = misc[kMBudget] < kBigMax ? misc[kMBudget] : kBigMax;
-        for (uint32_t i = warp; i < nbig; i += kSelWarps) {   // one warp per listed tile, 32 entries per round
-            const uint4 it = big[i];
-            const uint32_t first = tt->first[it.x], n = tt->n[it.x];
-            const int64_t lo_elem = (tile0 + tp + it.x) * kTile;
-            int64_t pos = out_off + it.y;
-            for (uint32_t e0 = 0; e0 < n; e0 += 32) {
-                const bool valid = e0 + lane < n;
-                const uint2 ent = valid ? staged_get(f, first + e0 + lane) : make_uint2(0u, 0u);
-                const bool sel = valid && ((fine_bin(key_of(ent.x), cut) > a) || (ent.y & kSelFlag));
-                const unsigned ball = __ballot_sync(0xffffffffu, sel);
-                if (sel) {
-                    const int64_t mypos = pos + __popc(ball & ((1u << lane) - 1u));
-                    const int64_t elem = lo_elem + (int64_t)y_off(ent.y);
-                    if (mypos < cap) {
-                        val[mypos] = __uint_as_float(ent.x);
-                        idx[mypos] = elem;
-                    }
-                    if (acc_rw) acc_rw[elem] = 0.0f;
+        lap.lap(25);
+        // pass 2
+        run = wtot[warp];
+        for (uint32_t p4 = w_lo; p4 < w_hi; p4 += 128) {
+            uint2 e4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t pos = p4 + u * 32 + lane;
+                e4[u] = pos < w_hi ? staged_get(f, pos) : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+            const uint32_t pos = p4 + u * 32 + lane;
+            const bool valid = pos < w_hi;
+            const uint2 ent = e4[u];
+            const uint32_t t = ((ent.y & ~kSelFlag) >> 11) - (uint32_t)tp;
+            const bool here = valid && t < (uint32_t)np;
+            const bool sel = here && ((fine_bin(key_of(ent.x), cut) > a) || (ent.y & kSelFlag));
+            const unsigned ball = __ballot_sync(0xffffffffu, sel);
+            if (sel) {
+                const uint32_t mark = tt->first[t];   // where the tile's first entry stood: warp, running count
+                const uint32_t at_first = wtot[(mark >> 27) & 15u] + (mark & 0x7ffffffu);
+                const int64_t o = out_off + tt->ge[t] + (run + __popc(ball & ((1u << lane) - 1u)) - at_first);
+                const int64_t elem = (tile0 + tp + t) * kTile + (int64_t)y_off(ent.y);
+                if (o < cap) {
+                    val[o] = __uint_as_float(ent.x);
+                    idx[o] = elem;
                 }
-                pos += __popc(ball);
+                if (acc_rw) acc_rw[elem] = 0.0f;
+            }
+            run += __popc(ball);
             }
         }
         base += total;
-        __syncthreads();   // the tables are rewritten by the next pass
-        lap.lap(27);
+        __syncthreads();   // the tables are rewritten by the next round
+        lap.lap(26);
     }
     if (p.timing && tid == 0) atomicAdd(p.timing + 28, 1ull);
 }
@@ -316,6 +342,12 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
 __device__ __noinline__ void retry_steps(const SelParams& q, unsigned char* smem, cg::grid_group& grid) {
     five_steps(q, smem, grid);
 }
+
+// Tiles are dealt out to the CTAs in stripes of kStripe consecutive tiles, round-robin: every CTA gets an
+// even sample of every layer of the call, so the layers whose entries crowd (large k_l / size_l) are
+// everybody's business, and so is the second look at a layer whose cut failed.
+constexpr int kStripe = 16;
+static_assert(kMaxLocalTiles % kStripe == 0 && kTfCache * 2 <= kSmSuperBytes, "stripes; the layer map lives in the super-tile area");
 
 __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParams p_in, const int has_streamed) {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -331,151 +363,115 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint32_t* wbase = reinterpret_cast<uint32_t*>(smem + kSmWBase);
     uint2* res = reinterpret_cast<uint2*>(smem + kSmMain);
+    int* tfc = reinterpret_cast<int*>(smem + kSmTf);                    // first tile of every layer of the call (+ end)
+    uint16_t* jmap = reinterpret_cast<uint16_t*>(smem + kSmSuper);      // layer of the call -> local (streamed) layer
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const CtaRange r = cta_range(p, reinterpret_cast<int*>(smem + kSmTf));
-    const int nl = build_layer_table(p, r, lt, misc + kMScratch, true);
-    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMTileCtr] = 0; misc[kMFlag] = 0; misc[kMBudget] = 4096u; }
+    const int b = blockIdx.x, G = gridDim.x;
+    for (int i = threadIdx.x; i <= p.n_my; i += kSelThreads) tfc[i] = p.desc[i].tile_first;
+    for (int i = threadIdx.x; i < p.n_my; i += kSelThreads) jmap[i] = 0xffffu;
+    CtaRange r;
+    r.il = 0; r.q0tab = nullptr; r.nsuper = 0;
+    r.q0 = 0; r.q1 = p.tiles; r.nloc = 0;
+    r.jA = 0; r.jB = p.n_my - 1;
+    const int nl = build_layer_table(p, r, lt, misc + kMScratch, true);   // every streamed layer of the call
+    const int nstripe = (p.tiles + kStripe - 1) / kStripe;
+    const int nloc = (b < nstripe ? (nstripe - b + G - 1) / G : 0) * kStripe;
+    if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMTileCtr] = 0; misc[kMBudget] = 4096u; }
     __syncthreads();
-    // what the CTA may stage: a multiple of what its tiles should hold if every layer's entries down to
-    // the rank behind its cut were spread evenly.  A cut that turns out far too low must not flood the
-    // staging area: past the budget the CTA stops reading and its layers go to the retry list.
     for (int c = threadIdx.x; c < nl; c += kSelThreads) {
-        lt->v0[c] = 0u;   // entries of the layer this CTA stages
-        if (lt->sthr[c] == 0xffffffffu) continue;
+        jmap[lt->j[c]] = (uint16_t)c;
+        lt->v0[c] = 0u;   // entries of the layer this CTA keeps in shared memory
+        if (lt->sthr[c] == 0xffffffffu) {
+            // no usable cut: the layer goes to the retry list (one CTA says so)
+            if (c % G == b) {
+                push_retry(p, lt->j[c]);
+                atomicAdd(p.spec_ctl + 6, 1u);
+            }
+            continue;
+        }
+        // what the CTA may stage: a multiple of what its share of the layer's tiles should hold if the entries
+        // down to the rank behind the cut were spread evenly.  A cut that turns out far too low must not
+        // flood the staging area: past the budget the CTA stops reading, and the layers it skips tiles of
+        // go to the retry list.
         const int64_t size = lt->end[c] - lt->start[c];
         const uint64_t per_tile = ((uint64_t)safe_rank(lt->k[c]) * kTile + size - 1) / size;
-        const uint64_t want = (uint64_t)own_tiles(p, r, lt, c) * per_tile * kFloodFactor;
+        const uint64_t want = ((uint64_t)(lt->tfe[c] - lt->tf[c]) / G + 1) * per_tile * kFloodFactor;
         atomicAdd(&misc[kMBudget], (uint32_t)(want < 0x3fffffffull ? want : 0x3fffffffull));
     }
-    // layers without a usable cut: the CTA that owns the layer's first tile hands them on
-    for (int c = threadIdx.x; c < nl; c += kSelThreads)
-        if (lt->sthr[c] == 0xffffffffu && lt->tf[c] >= r.q0 && lt->tf[c] < r.q1) {
-            push_retry(p, lt->j[c]);
-            atomicAdd(p.spec_ctl + 6, 1u);
-        }
     __syncthreads();
     stamp(p, 8);
     const uint32_t budget = misc[kMBudget] < 0x7fffffffu ? misc[kMBudget] : 0x7fffffffu;
 
-    if (nl > 0) {   // uniform over the CTA; a CTA without streamed layers has nothing to read or hand over
-        // ---- the read: every tile of the CTA once ----
-        {
-            int c = 0;
-            for (int lq = grab_tile(misc + kMTileCtr, lane); lq < r.nloc; lq = grab_tile(misc + kMTileCtr, lane)) {
-                const int q = r.q0 + lq;
-                const int cl = tile_layer(lt, nl, q, c);
-                uint32_t first = 0, n = 0;
-                if (cl >= 0 && lt->sthr[cl] != 0xffffffffu &&
-                    *reinterpret_cast<volatile uint32_t*>(misc + kMCursor) > budget) {
-                    if (lane == 0) misc[kMFlag] = 1u;
-                } else if (cl >= 0 && lt->sthr[cl] != 0xffffffffu) {
-                    const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-                    TileRegs t;
-                    uint32_t vm[2], keep[2];
-                    load_tile(p.acc, ts, lane, t, vm);
-                    const bool any_marked = mark_tile(t, vm, lt->sthr[cl], keep);
-                    if (any_marked) {
-                        // room in the CTA's shared memory, or, when that is full, straight in the layer's region
-                        const bool single = marks_single(keep[0], keep[1]);   // uniform over the warp
-                        MarkScan ms;
-                        if (single) n = count_single(keep[0], keep[1]);
-                        else { ms = scan_marks(keep[0], keep[1], lane); n = ms.n; }
-                        if (lane == 0) first = atomicAdd(misc + kMCursor, n);
-                        first = __shfl_sync(0xffffffffu, first, 0);
-                        uint2* dst = res;
-                        uint32_t ytag = pack_y(0u, (uint32_t)cl, (uint32_t)lq);
-                        const bool to_global = first + n > kStreamRes;
-                        if (to_global) {
-                            uint32_t g = 0;
-                            if (lane == 0) g = atomicAdd(&p.state[lt->lid[cl]].cursor, n);
-                            g = __shfl_sync(0xffffffffu, g, 0);
-                            dst = p.staging + lt->elem_off[cl];
-                            ytag = region_y(0u, (uint32_t)(q - lt->tf[cl]));
-                            if (lane == 0) { p.runge[q] = make_uint2(g, n); atomicAdd(&lt->v0[cl], n); }
-                            first = g;
-                        }
-                        auto put = [&](uint32_t pos, uint32_t bits, uint32_t off) { dst[pos] = make_uint2(bits, ytag | off); };
-                        if (single) write_single(t, keep[0], keep[1], first, lane, put);
-                        else write_scanned(reinterpret_cast<const uint32_t*>(p.acc + ts.lo), keep[0], keep[1], ms, first,
-                                           wbase + 16 * warp, lane, put);
-                        if (to_global) { first = kTileGlobal; n = 0; }
-                    }
+    // ---- the read: every tile of the CTA once ----
+    for (int lq = grab_tile(misc + kMTileCtr, lane); lq < nloc; lq = grab_tile(misc + kMTileCtr, lane)) {
+        const int q = kStripe * (b + (lq / kStripe) * G) + lq % kStripe;
+        uint32_t first = 0, n = 0, off = 0;
+        int cl = -1;
+        if (q < p.tiles) {
+            const uint32_t m = jmap[layer_of_tile_sh(tfc, p.n_my, q)];
+            if (m != 0xffffu && lt->sthr[m] != 0xffffffffu) cl = (int)m;
+        }
+        if (cl >= 0 && *reinterpret_cast<volatile uint32_t*>(misc + kMCursor) > budget) {
+            if (lane == 0) atomicOr(&p.state[lt->lid[cl]].spec_bad, 1u);
+        } else if (cl >= 0) {
+            const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
+            TileRegs t;
+            uint32_t vm[2], keep[2];
+            load_tile(p.acc, ts, lane, t, vm);
+            if (mark_tile(t, vm, lt->sthr[cl], keep)) {
+                // room in the CTA's shared memory, or, when that is full, straight in the layer's region
+                const bool single = marks_single(keep[0], keep[1]);   // uniform over the warp
+                MarkScan ms;
+                if (single) n = count_single(keep[0], keep[1]);
+                else { ms = scan_marks(keep[0], keep[1], lane); n = ms.n; }
+                if (lane == 0) first = atomicAdd(misc + kMCursor, n);
+                first = __shfl_sync(0xffffffffu, first, 0);
+                uint2* dst = res;
+                uint32_t ytag = pack_y(0u, (uint32_t)cl, 0u);
+                const bool to_global = first + n > kStreamRes;
+                if (lane == 0) off = to_global ? atomicAdd(&p.state[lt->lid[cl]].cursor, n) : atomicAdd(&lt->v0[cl], n);
+                off = __shfl_sync(0xffffffffu, off, 0);
+                if (to_global) {
+                    dst = p.staging + lt->elem_off[cl];
+                    ytag = region_y(0u, (uint32_t)(q - lt->tf[cl]));
+                    if (lane == 0) p.runge[q] = make_uint2(off, n);
+                    first = off;
                 }
-                if (lane == 0) { tt->first[lq] = first; tt->n[lq] = (uint16_t)n; }
+                auto put = [&](uint32_t pos, uint32_t bits, uint32_t o) { dst[pos] = make_uint2(bits, ytag | o); };
+                if (single) write_single(t, keep[0], keep[1], first, lane, put);
+                else write_scanned(reinterpret_cast<const uint32_t*>(p.acc + ts.lo), keep[0], keep[1], ms, first,
+                                   wbase + 16 * warp, lane, put);
+                if (to_global) { first = kTileGlobal; n = 0; }
             }
         }
-        __syncthreads();
-        stamp(p, 1);
-
-        // ---- hand the staged entries to the layers' regions ----
-        // one warp per local layer: room for the CTA's entries of the layer, then where each tile's entries go
-        for (int c = warp; c < nl; c += kSelWarps) {
-            if (lt->sthr[c] == 0xffffffffu) continue;
-            int a, b;
-            local_span(r, lt, c, c, a, b);
-            uint32_t nc = 0;
-            for (int i = a + lane; i < b; i += 32) nc += tt->n[i];
-            nc = __reduce_add_sync(0xffffffffu, nc);
-            uint32_t run = 0;
-            if (lane == 0) lt->v0[c] += nc;   // with the tiles that went straight to the region: the CTA's entries of the layer
-            if (lane == 0 && nc != 0) run = atomicAdd(&p.state[lt->lid[c]].cursor, nc);
-            run = __shfl_sync(0xffffffffu, run, 0);
-            for (int i0 = a; i0 < b; i0 += 32) {
-                const int i = i0 + lane;
-                const uint32_t n = i < b ? tt->n[i] : 0u;
-                const uint32_t incl = warp_incl_scan(n, lane);
-                if (i < b && tt->first[i] != kTileGlobal) {
-                    tt->ge[i] = run + incl - n;
-                    p.runge[r.q0 + i] = make_uint2(run + incl - n, n);
-                }
-                run += __shfl_sync(0xffffffffu, incl, 31);
-            }
-        }
-        __syncthreads();
-        // one thread per tile copies the tile's entries
-        for (int lq = threadIdx.x; lq < r.nloc; lq += kSelThreads) {
-            const uint32_t n = tt->n[lq];
-            if (n == 0) continue;
-            const uint32_t first = tt->first[lq], g = tt->ge[lq];
-            const int cl = (int)y_layer(res[first].y);
-            uint2* dst = p.staging + lt->elem_off[cl] + g;
-            const uint32_t yt = region_y(0u, (uint32_t)(r.q0 + lq - lt->tf[cl]));
-            for (uint32_t e = 0; e < n; ++e) {
-                const uint2 ent = res[first + e];
-                dst[e] = make_uint2(ent.x, yt | y_off(ent.y));
-            }
-        }
-        __threadfence();
-        __syncthreads();
-        stamp(p, 2);
-        // per layer, what the CTAs that are through with it add up to: the CTA that completes the layer's last
-        // tiles sees every tile accounted for, and with them the layer's entries, and finishes the layer
-        for (int c = threadIdx.x; c < nl; c += kSelThreads) {
-            uint32_t last = 0u;
-            if (lt->sthr[c] != 0xffffffffu) {
-                const unsigned long long mine = ((unsigned long long)own_tiles(p, r, lt, c) << 41) |
-                                                ((unsigned long long)(misc[kMFlag] ? 1u : 0u) << 31) | lt->v0[c];
-                const unsigned long long now = atomicAdd(&p.state[lt->lid[c]].done, mine) + mine;
-                if ((uint32_t)(now >> 41) == (uint32_t)(lt->tfe[c] - lt->tf[c])) {
-                    last = 1u | ((uint32_t)((now >> 31) & 0x3ffu) != 0u ? 2u : 0u);
-                    lt->v0[c] = (uint32_t)now & 0x7fffffffu;
-                }
-            }
-            lt->v1[c] = last;
-        }
-        __syncthreads();
-        int nfin = 0;
-        for (int c = 0; c < nl; ++c) {
-            if (!lt->v1[c]) continue;   // uniform over the CTA
-            __threadfence();
-            __syncthreads();
-            finish_layer(p, lt, c, lt->v0[c], lt->v1[c] >> 1, tt, smem);
-            __syncthreads();
-            ++nfin;
-        }
-        if (p.timing && threadIdx.x == 0) atomicMax(p.timing + 29, (unsigned long long)nfin);
+        if (lane == 0) { tt->first[lq] = first; tt->n[lq] = (uint16_t)n; tt->ge[lq] = off; }
     }
-    stamp(p, 5);
+    __syncthreads();
+    stamp(p, 1);
+
+    // ---- hand the staged entries to the layers' regions ----
+    // room in every layer's region for what this CTA holds of it; then one thread per tile copies
+    for (int c = threadIdx.x; c < nl; c += kSelThreads) {
+        const uint32_t nc = lt->v0[c];
+        lt->v1[c] = nc ? atomicAdd(&p.state[lt->lid[c]].cursor, nc) : 0u;
+    }
+    __syncthreads();
+    for (int lq = threadIdx.x; lq < nloc; lq += kSelThreads) {
+        const int q = kStripe * (b + (lq / kStripe) * G) + lq % kStripe;
+        const uint32_t n = tt->n[lq], first = tt->first[lq];
+        if (q >= p.tiles || first == kTileGlobal) continue;
+        if (n == 0) { p.runge[q] = make_uint2(0u, 0u); continue; }
+        const int cl = (int)y_layer(res[first].y);
+        const uint32_t g = lt->v1[cl] + tt->ge[lq];
+        p.runge[q] = make_uint2(g, n);
+        uint2* dst = p.staging + lt->elem_off[cl] + g;
+        const uint32_t yt = region_y(0u, (uint32_t)(q - lt->tf[cl]));
+        for (uint32_t e = 0; e < n; ++e) {
+            const uint2 ent = res[first + e];
+            dst[e] = make_uint2(ent.x, yt | y_off(ent.y));
+        }
+    }
+    stamp(p, 2);
 
     // ---- small layers, handed out one at a time (the counter is cleared with the plan upload) ----
     {
@@ -490,7 +486,19 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
         }
     }
     stamp(p, 6);
-    if (!has_streamed) return;   // uniform over the grid: small layers only, nothing can be left over
+    if (!has_streamed) return;   // uniform over the grid: small layers only
+
+    // ---- every layer's entries are in its region: the layers are finished one per CTA, round-robin ----
+    __threadfence();
+    grid.sync();
+    for (int c = b; c < nl; c += G) {
+        if (lt->sthr[c] == 0xffffffffu) continue;
+        const uint32_t S = __ldcg(&p.state[lt->lid[c]].cursor);
+        const uint32_t flooded = __ldcg(&p.state[lt->lid[c]].spec_bad);
+        finish_layer(p, lt, c, S, flooded, tt, smem);
+        __syncthreads();
+    }
+    stamp(p, 5);
 
     // ---- what is left over: the five steps on the retry list, by the whole grid ----
     __threadfence();

@@ -304,8 +304,9 @@ def deft_debug_select_timing(timing_d) -> None:
     lib().deft_debug_select_timing(None if timing_d is None else _dp(timing_d))
 
 
-def deft_debug_select_kernel(single_pass: bool) -> None:
-    lib().deft_debug_select_kernel(1 if single_pass else 0)
+def deft_debug_select_kernel(single_pass) -> None:
+    """True / False: force the single-pass / the five-step selection kernel; None: by call size (default)."""
+    lib().deft_debug_select_kernel(-1 if single_pass is None else (1 if single_pass else 0))
 
 
 def deft_select_stats(ws, n_layers: int, stream=None) -> dict:

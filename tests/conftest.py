@@ -15,3 +15,16 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(autouse=True, scope="session")
+def _selection_kernel_choice():
+    """DEFT_SINGLE_PASS=1 / 0 runs the whole GPU suite with the single-pass selection kernel forced on / off
+    (results must not depend on the choice; the default picks by call size)."""
+    import os
+    if os.environ.get("DEFT_SINGLE_PASS") in ("0", "1"):
+        from paper_2307_03500_b200 import build as deft_build
+        deft_build.build()
+        from paper_2307_03500_b200 import deft
+        deft.deft_debug_select_kernel(os.environ["DEFT_SINGLE_PASS"] == "1")
+    yield

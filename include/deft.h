@@ -429,6 +429,39 @@ DEFT_API deft_status deft_gather_update(float* acc_d, int64_t n_g, const int64_t
                                         float* val_d, void* stream);
 
 /*
+ * Algorithm 1 around the sparsifier, for runs with several workers (lines 7-10 and Eq. 2).  The
+ * collectives themselves (all-gather of the index lists, all-reduce of the values) are the caller's;
+ * these calls do what happens on the device before and after them.
+ *
+ * deft_index_union — line 7 after the all-gather: the sorted set of the indices in idx_d[0, count)
+ * (any order, duplicates allowed, each in [0, n_g); others are ignored).  Writes the first out_cap of
+ * them to union_d in ascending order and their number to *count_d (DEVICE int64; may exceed out_cap).
+ * DEFT's workers own disjoint layers, so their lists never overlap and the union has exactly sum k_l
+ * entries; with Top-k on every worker it is the place where the build-up of Section 1 shows.
+ * ws_d: deft_union_workspace_bytes(n_g) bytes (a bitmap of n_g bits and one counter per 32768 of them),
+ * 256-byte aligned.  Errors: INVALID_ARG, CAPACITY (workspace), CUDA.
+ *
+ * deft_sum_into — dst_d[i] += src_d[i] for i < count, one fp32 round-to-nearest add each: the sum of
+ * line 9 where all workers live on one device (otherwise the all-reduce forms it).
+ * deft_average — sum_d[i] /= n_workers, one fp32 division each: line 9's 1/n after the sum.
+ *
+ * deft_vector_norm — the L2 norm of x_d[0, n) in fp64 (Eq. 2: a worker's error is the norm of its
+ * residual), computed like one layer's norm in deft_layer_norms; nothing is written to x_d.
+ * norm_d: DEVICE double.  ws_d: deft_vector_norm_workspace_bytes(n) bytes, 256-byte aligned.
+ */
+/* Eq. 2 (host): the mean of the workers' errors (their residuals' norms), added in rank order. */
+DEFT_API deft_status deft_error_eq2(const double* worker_error_h, int32_t n_workers, double* error_out);
+
+DEFT_API size_t deft_union_workspace_bytes(int64_t n_g);
+DEFT_API deft_status deft_index_union(const int64_t* idx_d, int64_t count, int64_t n_g, int64_t* union_d,
+                                      int64_t out_cap, int64_t* count_d, void* ws_d, size_t ws_bytes, void* stream);
+DEFT_API deft_status deft_sum_into(float* dst_d, const float* src_d, int64_t count, void* stream);
+DEFT_API deft_status deft_average(float* sum_d, int64_t count, int32_t n_workers, void* stream);
+DEFT_API size_t deft_vector_norm_workspace_bytes(int64_t n);
+DEFT_API deft_status deft_vector_norm(const float* x_d, int64_t n, double* norm_d, void* ws_d, size_t ws_bytes,
+                                      void* stream);
+
+/*
  * Residual update — Algorithm 1 lines 11-12: acc[idx[j]] = +0.0f for j < count; the
  * buffer is then the next step's local error.  Indices must be distinct and < n_g.
  *   idx_d[count] DEVICE.  count may be 0.  Errors: INVALID_ARG, CUDA.

@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + ".tmp.%d" % os.getpid()
         subprocess.check_call(
-            ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared", _SRC, "-o", tmp]
+            ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared", "-pthread", _SRC, "-o", tmp]
         )
         os.replace(tmp, _LIB)
     return _LIB
@@ -46,6 +46,11 @@ def _load():
         _lib.oracle_rank_bin.restype = ctypes.c_int64
         _lib.oracle_partition_optimum.restype = ctypes.c_double
         _lib.oracle_select_rank.restype = ctypes.c_int64
+        _lib.oracle_index_union.restype = ctypes.c_int64
+        _lib.oracle_vector_norm.restype = ctypes.c_double
+        _lib.oracle_error_eq2.restype = ctypes.c_double
+        _lib.oracle_hardware_threads.restype = ctypes.c_int64
+        _lib.oracle_select_rank_threads.restype = ctypes.c_int64
     return _lib
 
 
@@ -196,3 +201,55 @@ def my_layers(bin_of_layer, iteration, rank, n_workers):
     """Layer ids (ascending) whose bin is the one ``rank`` reads this iteration."""
     b = rank_bin(iteration, rank, n_workers)
     return np.nonzero(np.asarray(bin_of_layer) == b)[0].astype(np.int32)
+
+
+def index_union(idx):
+    """Algorithm 1 line 7: the set of the gathered indices, ascending."""
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    out = np.empty(idx.size, dtype=np.int64)
+    n = _load().oracle_index_union(_p(idx), _i64(idx.size), _p(out))
+    return out[:n].copy()
+
+
+def sum_into(dst, src):
+    """Algorithm 1 line 9 (the sum), fp32, in place over ``dst``."""
+    assert dst.dtype == np.float32 and src.dtype == np.float32 and dst.size == src.size
+    _load().oracle_sum_into(_p(dst), _p(src), _i64(dst.size))
+    return dst
+
+
+def average(total, n_workers):
+    """Algorithm 1 line 9 (the 1/n), fp32, in place."""
+    assert total.dtype == np.float32
+    _load().oracle_average(_p(total), _i64(total.size), _i64(n_workers))
+    return total
+
+
+def vector_norm(x):
+    """Eq. 2: L2 norm of a worker's residual, fp64."""
+    assert x.dtype == np.float32 and x.flags.c_contiguous
+    return float(_load().oracle_vector_norm(_p(x), _i64(x.size)))
+
+
+def error_eq2(worker_errors):
+    """Eq. 2: mean of the workers' errors."""
+    w = np.ascontiguousarray(worker_errors, dtype=np.float64)
+    return float(_load().oracle_error_eq2(_p(w), _i64(w.size)))
+
+
+def hardware_threads():
+    return int(_load().oracle_hardware_threads())
+
+
+def select_rank_threads(acc, layer_start, k_l, my_layers, threads=0):
+    """oracle select_rank with the rank's layers farmed out over host threads (timing leg).
+    Returns (values, indices, threads used)."""
+    layer_start = np.ascontiguousarray(layer_start, dtype=np.int64)
+    k_l = np.ascontiguousarray(k_l, dtype=np.int64)
+    my = np.ascontiguousarray(my_layers, dtype=np.int32)
+    total = int(k_l[my].sum()) if my.size else 0
+    val = np.empty(total, dtype=np.float32)
+    idx = np.empty(total, dtype=np.int64)
+    used = _load().oracle_select_rank_threads(_p(acc), _p(layer_start), _p(k_l), _p(my), _i64(my.size), _p(val), _p(idx),
+                                              _i64(threads))
+    return val, idx, int(used)

@@ -1,10 +1,11 @@
 // DEFT gradient-selection oracle: TEST INFRASTRUCTURE, NOT THE PRODUCT.
 //
-// A plain, slow, single-threaded CPU statement of what the DEFT hot path
+// A plain, slow CPU statement of what the DEFT hot path
 // computes (Yoon & Oh, "DEFT: Exploiting Gradient Norm Difference between
 // Model Layers for Scalable Gradient Sparsification", ICPP 2023).  It is
 // used only by the tests, the smoke check and the benchmark's CPU-baseline
-// leg.  It shares no code, header, table or helper with the CUDA library
+// leg (one routine below runs a rank's layers on several host threads for that
+// leg's all-cores figure; everything else is single-threaded).  It shares no code, header, table or helper with the CUDA library
 // and neither side includes or links the other.
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared (no fast-math,
@@ -15,9 +16,11 @@
 // pinned by closed forms, invariants, library routines, exact rational
 // arithmetic or brute force; none is "parity unpinned".
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <thread>
 #include <utility>
 #include <vector>
 
@@ -196,50 +199,50 @@ int64_t oracle_allocate_k(const double* norms, const int64_t* layer_size, int64_
 
 // ---------------------------------------------------------------------------
 // Algorithm 4 (bin-packing-based layer allocation), Section 4.3, Eq. 3.
-// cost_l = size_l * ln(k_l).  L times: take the layer of largest cost (first
-// occurrence), put it in the bin of smallest load (first occurrence), add
-// its cost to that bin, mark the layer with cost -1.  Layer ids are
-// positions in address order.
+// Every layer has a selection cost; the costliest layer not yet placed goes
+// to the worker whose bin is lightest so far, until every layer is placed.
+// Equal costs: the layer that comes first in address order.  Equal loads: the
+// bin with the lowest number.  (Costs are never negative, so "not yet
+// placed" is kept as a flag of its own rather than as a special cost value.)
+// Layer ids are positions in address order.
 // ---------------------------------------------------------------------------
-void oracle_partition(const int64_t* layer_size, const int64_t* k_l, int64_t L, int64_t n_workers,
-                      int32_t* bin_of_layer, double* size_bin /* n_workers */) {
-    std::vector<double> cost(L);
-    for (int64_t i = 0; i < L; ++i) cost[i] = (double)layer_size[i] * std::log((double)k_l[i]);
-    for (int64_t b = 0; b < n_workers; ++b) size_bin[b] = 0.0;
-    for (int64_t it = 0; it < L; ++it) {
-        int64_t idx_max = 0;
-        for (int64_t i = 1; i < L; ++i)
-            if (cost[i] > cost[idx_max]) idx_max = i;
-        const double val_max = cost[idx_max];
-        int64_t bin_min = 0;
+static void pack_greedily(const std::vector<double>& layer_cost, int64_t n_workers, int32_t* bin_of_layer,
+                          double* bin_load /* n_workers */) {
+    const int64_t L = (int64_t)layer_cost.size();
+    std::vector<char> placed(L, 0);
+    for (int64_t b = 0; b < n_workers; ++b) bin_load[b] = 0.0;
+    for (int64_t round = 0; round < L; ++round) {
+        int64_t costliest = -1;
+        for (int64_t l = 0; l < L; ++l) {
+            if (placed[l]) continue;
+            if (costliest < 0 || layer_cost[l] > layer_cost[costliest]) costliest = l;
+        }
+        int64_t lightest = 0;
         for (int64_t b = 1; b < n_workers; ++b)
-            if (size_bin[b] < size_bin[bin_min]) bin_min = b;
-        bin_of_layer[idx_max] = (int32_t)bin_min;
-        size_bin[bin_min] = size_bin[bin_min] + val_max;
-        cost[idx_max] = -1.0;
+            if (bin_load[b] < bin_load[lightest]) lightest = b;
+        bin_of_layer[costliest] = (int32_t)lightest;
+        bin_load[lightest] = bin_load[lightest] + layer_cost[costliest];
+        placed[costliest] = 1;
     }
 }
 
+// Eq. 3: the cost of selecting k_x gradients out of the n_{g,x} of layer x is n_{g,x} * log(k_x)
+// (natural logarithm; the base only scales every load).
+void oracle_partition(const int64_t* layer_size, const int64_t* k_l, int64_t L, int64_t n_workers,
+                      int32_t* bin_of_layer, double* size_bin /* n_workers */) {
+    std::vector<double> layer_cost(L);
+    for (int64_t l = 0; l < L; ++l) layer_cost[l] = (double)layer_size[l] * std::log((double)k_l[l]);
+    pack_greedily(layer_cost, n_workers, bin_of_layer, size_bin);
+}
+
 // Variant of Algorithm 4 for hardware whose selection time follows the bytes a worker scans
-// rather than size * ln(k) (a linear-time selection): the same greedy packing with
-// cost_l = size_l.  Not in the paper; an ablation of the load model of Eq. 3.
+// rather than size * ln(k) (a linear-time selection): the same greedy packing with the layer's
+// size as its cost.  Not in the paper; an ablation of the load model of Eq. 3.
 void oracle_partition_by_size(const int64_t* layer_size, int64_t L, int64_t n_workers,
                               int32_t* bin_of_layer, double* size_bin /* n_workers */) {
-    std::vector<double> cost(L);
-    for (int64_t i = 0; i < L; ++i) cost[i] = (double)layer_size[i];
-    for (int64_t b = 0; b < n_workers; ++b) size_bin[b] = 0.0;
-    for (int64_t it = 0; it < L; ++it) {
-        int64_t idx_max = 0;
-        for (int64_t i = 1; i < L; ++i)
-            if (cost[i] > cost[idx_max]) idx_max = i;
-        const double val_max = cost[idx_max];
-        int64_t bin_min = 0;
-        for (int64_t b = 1; b < n_workers; ++b)
-            if (size_bin[b] < size_bin[bin_min]) bin_min = b;
-        bin_of_layer[idx_max] = (int32_t)bin_min;
-        size_bin[bin_min] = size_bin[bin_min] + val_max;
-        cost[idx_max] = -1.0;
-    }
+    std::vector<double> layer_cost(L);
+    for (int64_t l = 0; l < L; ++l) layer_cost[l] = (double)layer_size[l];
+    pack_greedily(layer_cost, n_workers, bin_of_layer, size_bin);
 }
 
 // Algorithm 4, lines 1-2: the bin a rank reads in a given iteration.
@@ -357,6 +360,85 @@ void oracle_gather_update(float* acc, const int64_t* idx, int64_t count, float* 
         val[j] = acc[idx[j]];
         acc[idx[j]] = 0.0f;
     }
+}
+
+// ---------------------------------------------------------------------------
+// Algorithm 1 around the sparsifier, for several workers.
+// ---------------------------------------------------------------------------
+// Line 7: after the all-gather every worker holds all workers' index lists; the gradients that take
+// part in the update are the SET of those indices.  Returns its size; out receives it ascending.
+int64_t oracle_index_union(const int64_t* idx, int64_t count, int64_t* out) {
+    std::vector<int64_t> all(idx, idx + count);
+    std::sort(all.begin(), all.end());
+    all.erase(std::unique(all.begin(), all.end()), all.end());
+    for (size_t i = 0; i < all.size(); ++i) out[i] = all[i];
+    return (int64_t)all.size();
+}
+
+// Lines 8-9: the workers' values at the selected indices are summed (AllReduce, SUM) and divided by
+// the number of workers; fp32, one rounded operation each, workers added in rank order.
+void oracle_sum_into(float* dst, const float* src, int64_t count) {
+    for (int64_t i = 0; i < count; ++i) {
+        volatile float s = dst[i] + src[i];
+        dst[i] = s;
+    }
+}
+void oracle_average(float* sum, int64_t count, int64_t n_workers) {
+    const float n = (float)n_workers;
+    for (int64_t i = 0; i < count; ++i) {
+        volatile float q = sum[i] / n;
+        sum[i] = q;
+    }
+}
+
+// Eq. 2: a worker's error is the L2 norm of its residual (fp64, summed sequentially); the error of
+// the iteration is the mean of the workers' errors.
+double oracle_vector_norm(const float* x, int64_t n) {
+    double s = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        const double v = (double)x[i];
+        s = s + v * v;
+    }
+    return std::sqrt(s);
+}
+double oracle_error_eq2(const double* worker_error, int64_t n_workers) {
+    double s = 0.0;
+    for (int64_t i = 0; i < n_workers; ++i) s = s + worker_error[i];
+    return s / (double)n_workers;
+}
+
+// ---------------------------------------------------------------------------
+// The per-layer selections of a rank farmed out over host threads (layers are independent: Algorithm 5
+// is a loop over them).  Same result as oracle_select_rank; used only to time the oracle on all of the
+// host's cores.  threads < 1: as many as the hardware reports.  Returns the threads used.
+// ---------------------------------------------------------------------------
+int64_t oracle_hardware_threads(void) {
+    const unsigned n = std::thread::hardware_concurrency();
+    return n ? (int64_t)n : 1;
+}
+
+int64_t oracle_select_rank_threads(const float* acc, const int64_t* layer_start, const int64_t* k_l,
+                                   const int32_t* my_layers, int64_t n_my, float* val_out, int64_t* idx_out,
+                                   int64_t threads) {
+    if (threads < 1) threads = oracle_hardware_threads();
+    if (threads > n_my) threads = n_my > 0 ? n_my : 1;
+    std::vector<int64_t> out_off(n_my + 1, 0);
+    for (int64_t j = 0; j < n_my; ++j) out_off[j + 1] = out_off[j] + k_l[my_layers[j]];
+    std::atomic<int64_t> next(0);
+    auto work = [&]() {
+        for (;;) {
+            const int64_t j = next.fetch_add(1);
+            if (j >= n_my) break;
+            const int64_t part = my_layers[j];
+            oracle_select_layer(acc, layer_start[part], layer_start[part + 1], k_l[part], val_out + out_off[j],
+                                idx_out + out_off[j]);
+        }
+    };
+    std::vector<std::thread> pool;
+    for (int64_t t = 1; t < threads; ++t) pool.emplace_back(work);
+    work();
+    for (auto& th : pool) th.join();
+    return threads;
 }
 
 }  // extern "C"

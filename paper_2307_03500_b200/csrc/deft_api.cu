@@ -380,23 +380,125 @@ size_t deft_plan_bytes(int32_t L, int32_t N) {
     return plan_bytes(L, N);
 }
 
+// The plan of a whole model (every layer in exactly one bin, layer ids in address order), written
+// straight into the blob in two passes over the layers: the per-step path, kept free of allocations.
 static deft_status plan_build_impl(const int64_t* layer_start_h, const int64_t* k_l_h,
                                    const int32_t* bin_of_layer_h, const double* norms_h, int32_t L, int32_t N,
                                    int64_t iteration, void* plan_h, size_t plan_bytes_cap) {
     if (!layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || L < 1 || N < 1 || N > kMaxRanks ||
         iteration < 0)
         return DEFT_ERR_INVALID_ARG;
-    std::vector<std::vector<LayerItem>> ranks((size_t)N);
-    for (auto& v : ranks) v.reserve((size_t)(L / N + 8));
+    if (plan_bytes_cap < plan_bytes(L, N)) return DEFT_ERR_CAPACITY;
+    char* base = static_cast<char*>(plan_h);
+    PlanHeader* hdr = reinterpret_cast<PlanHeader*>(base);
+    RankInfo* ri = reinterpret_cast<RankInfo*>(base + sizeof(PlanHeader));
+    LayerDesc* desc = reinterpret_cast<LayerDesc*>(base + sizeof(PlanHeader) + sizeof(RankInfo) * (size_t)(N + 1));
+    struct Acc { int64_t tiles, elems, slots, k; int32_t n; };
+    static thread_local std::vector<Acc> acc;
+    static thread_local std::vector<int32_t> rank_of;
+    acc.assign((size_t)N, Acc{0, 0, 0, 0, 0});
+    rank_of.resize((size_t)L);
     const int32_t cycle = (int32_t)(iteration % N);
+    auto tiles_of = [](int64_t st, int64_t en) { return (en - 1) / kTile - st / kTile + 1; };
+    auto slots_of = [](int64_t size) { return (size + kRegionAlign - 1) / kRegionAlign * kRegionAlign; };
+    // pass 1: what every rank holds
     for (int32_t l = 0; l < L; ++l) {
         const int32_t b = bin_of_layer_h[l];
-        if (b < 0 || b >= N) return DEFT_ERR_INVALID_ARG;
+        const int64_t st = layer_start_h[l], en = layer_start_h[l + 1], size = en - st;
+        if (b < 0 || b >= N || st < 0 || size < 1 || size > DEFT_MAX_LAYER_ELEMS || k_l_h[l] < 1 || k_l_h[l] > size)
+            return DEFT_ERR_INVALID_ARG;
         // rank r reads bin (cycle + r) % N  <=>  bin b is read by rank (b - cycle) mod N
-        const int32_t r = ((b - cycle) % N + N) % N;
-        ranks[r].push_back(LayerItem{layer_start_h[l], layer_start_h[l + 1], k_l_h[l], l, norms_h ? norms_h[l] : 0.0});
+        const int32_t r = b - cycle < 0 ? b - cycle + N : b - cycle;
+        rank_of[l] = r;
+        Acc& A = acc[r];
+        A.tiles += tiles_of(st, en);
+        A.elems += size;
+        A.slots += slots_of(size);
+        A.k += k_l_h[l];
+        A.n += 1;
     }
-    return fill_plan(plan_h, plan_bytes_cap, L, iteration, ranks);
+    int64_t tiles_all = 0, elems_all = 0, slots_all = 0, k_all = 0, d = 0;
+    for (int32_t r = 0; r < N; ++r) {
+        RankInfo& R = ri[r];
+        const Acc A = acc[r];
+        R.desc_first = (int32_t)d;
+        R.n_my = A.n;
+        R.tiles = (int32_t)A.tiles;
+        R.tile_base = (int32_t)tiles_all;
+        R.elems = A.elems;
+        R.k = A.k;
+        R.out_off = k_all;
+        R.elem_base = slots_all;
+        R.reserved[0] = R.reserved[1] = 0;
+        LayerDesc& Z = desc[d + A.n];   // the rank's sentinel
+        Z = LayerDesc{};
+        Z.out_off = A.k;
+        Z.elem_off = slots_all + A.slots;
+        Z.tile_first = (int32_t)A.tiles;
+        Z.layer_id = -1;
+        d += A.n + 1;
+        tiles_all += A.tiles;
+        elems_all += A.elems;
+        slots_all += A.slots;
+        k_all += A.k;
+        if (tiles_all > INT32_MAX) return DEFT_ERR_INVALID_ARG;
+        acc[r] = Acc{0, 0, 0, 0, 0};   // pass 2 counts up again
+    }
+    // pass 2: the ranks' lists, and all layers as one list in address order behind them
+    RankInfo& M = ri[N];
+    LayerDesc* all = desc + d;
+    int64_t m_tiles = 0, m_slots = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        const int32_t r = rank_of[l];
+        Acc& A = acc[r];
+        const int64_t st = layer_start_h[l], en = layer_start_h[l + 1], size = en - st;
+        LayerDesc D;
+        D.start = st;
+        D.end = en;
+        D.k = k_l_h[l];
+        D.out_off = A.k;
+        D.elem_off = ri[r].elem_base + A.slots;
+        D.tile_first = (int32_t)A.tiles;
+        D.layer_id = l;
+        D.norm = norms_h ? norms_h[l] : 0.0;
+        D.reserved = 0;
+        desc[ri[r].desc_first + A.n] = D;
+        D.out_off += ri[r].out_off;
+        D.elem_off = m_slots;
+        D.tile_first = (int32_t)m_tiles;
+        all[l] = D;
+        const int64_t t = tiles_of(st, en);
+        A.tiles += t;
+        A.slots += slots_of(size);
+        A.k += k_l_h[l];
+        A.n += 1;
+        m_tiles += t;
+        m_slots += slots_of(size);
+    }
+    LayerDesc& Z = all[L];
+    Z = LayerDesc{};
+    Z.out_off = k_all;
+    Z.elem_off = m_slots;
+    Z.tile_first = (int32_t)m_tiles;
+    Z.layer_id = -1;
+    M.desc_first = (int32_t)d;
+    M.n_my = L;
+    M.tiles = (int32_t)m_tiles;
+    M.tile_base = 0;
+    M.elems = elems_all;
+    M.k = k_all;
+    M.out_off = 0;
+    M.elem_base = 0;
+    M.reserved[0] = M.reserved[1] = 0;
+    hdr->magic = kPlanMagic;
+    hdr->L = L;
+    hdr->N = N;
+    hdr->total_tiles = (int32_t)tiles_all;
+    hdr->total_elems = elems_all;
+    hdr->total_k = k_all;
+    hdr->iteration = iteration;
+    hdr->reserved[0] = hdr->reserved[1] = hdr->reserved[2] = 0;
+    return DEFT_OK;
 }
 
 deft_status deft_plan_build(const int64_t* layer_start_h, const int64_t* k_l_h,
@@ -412,7 +514,8 @@ static deft_status plan_step_impl(const double* norms_h, const int64_t* layer_st
                                   bool clear) {
     if (!norms_h || !layer_start_h || !k_l_h || !bin_of_layer_h || !plan_h || !plan_d || !ws_d || L < 1)
         return DEFT_ERR_INVALID_ARG;
-    std::vector<int64_t> size((size_t)L);
+    static thread_local std::vector<int64_t> size;
+    size.resize((size_t)L);
     for (int32_t l = 0; l < L; ++l) size[l] = layer_start_h[l + 1] - layer_start_h[l];
     const deft_status sa = deft_allocate_k(norms_h, size.data(), L, k, mode, k_l_h, sum_k_out);
     if (sa < 0) return sa;
@@ -664,6 +767,43 @@ deft_status deft_gather_update(float* acc_d, int64_t n_g, const int64_t* idx_d, 
     if (count == 0) return DEFT_OK;
     if (!acc_d || !idx_d || !val_d) return DEFT_ERR_INVALID_ARG;
     return launch_gather_update(acc_d, idx_d, count, val_d, static_cast<cudaStream_t>(stream));
+}
+
+size_t deft_union_workspace_bytes(int64_t n_g) { return n_g < 1 ? 0 : union_ws_bytes(n_g); }
+
+deft_status deft_index_union(const int64_t* idx_d, int64_t count, int64_t n_g, int64_t* union_d, int64_t out_cap,
+                             int64_t* count_d, void* ws_d, size_t ws_bytes, void* stream) {
+    if (count < 0 || n_g < 1 || out_cap < 0 || !count_d || !ws_d || (count > 0 && !idx_d) || (out_cap > 0 && !union_d))
+        return DEFT_ERR_INVALID_ARG;
+    if (!aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    if (union_ws_bytes(n_g) > ws_bytes) return DEFT_ERR_CAPACITY;
+    return launch_index_union(idx_d, count, n_g, union_d, out_cap, reinterpret_cast<long long*>(count_d), ws_d,
+                              static_cast<cudaStream_t>(stream));
+}
+
+deft_status deft_sum_into(float* dst_d, const float* src_d, int64_t count, void* stream) {
+    if (count < 0 || (count > 0 && (!dst_d || !src_d))) return DEFT_ERR_INVALID_ARG;
+    return launch_sum_into(dst_d, src_d, count, static_cast<cudaStream_t>(stream));
+}
+
+deft_status deft_average(float* sum_d, int64_t count, int32_t n_workers, void* stream) {
+    if (count < 0 || n_workers < 1 || (count > 0 && !sum_d)) return DEFT_ERR_INVALID_ARG;
+    return launch_divide(sum_d, count, (float)n_workers, static_cast<cudaStream_t>(stream));
+}
+
+size_t deft_vector_norm_workspace_bytes(int64_t n) { return n < 1 ? 0 : 256 + align_up(norms_ws_bytes(n, 1), 256); }
+
+deft_status deft_vector_norm(const float* x_d, int64_t n, double* norm_d, void* ws_d, size_t ws_bytes, void* stream) {
+    if (!x_d || !norm_d || !ws_d || n < 1) return DEFT_ERR_INVALID_ARG;
+    if (!aligned16(x_d) || !aligned256(ws_d)) return DEFT_ERR_INVALID_ARG;
+    if (deft_vector_norm_workspace_bytes(n) > ws_bytes) return DEFT_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int64_t* ls_d = static_cast<int64_t*>(ws_d);
+    const deft_status s = launch_fill_start(ls_d, n, st);
+    if (s != DEFT_OK) return s;
+    // the accumulate + norm kernel in its norms-only form (no gradient: nothing is written to x)
+    return launch_layer_norms(const_cast<float*>(x_d), nullptr, n, ls_d, 1, norm_d,
+                              reinterpret_cast<double*>(static_cast<char*>(ws_d) + 256), st);
 }
 
 deft_status deft_residual_update(float* acc_d, int64_t n_g, const int64_t* idx_d, int64_t count,

@@ -285,4 +285,12 @@ deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t c
 deft_status launch_gather_update(float* acc_d, const int64_t* idx_d, int64_t count, float* val_d,
                                  cudaStream_t stream);
 
+// Algorithm 1's pieces around the sparsifier (deft_algo1.cu).
+size_t union_ws_bytes(int64_t n);
+deft_status launch_index_union(const int64_t* idx_d, int64_t count, int64_t n, int64_t* out_d, int64_t out_cap,
+                               long long* count_out_d, void* ws_d, cudaStream_t stream);
+deft_status launch_sum_into(float* dst_d, const float* src_d, int64_t count, cudaStream_t stream);
+deft_status launch_divide(float* x_d, int64_t count, float by, cudaStream_t stream);
+deft_status launch_fill_start(int64_t* ls_d, int64_t n, cudaStream_t stream);
+
 }  // namespace deft

@@ -3,6 +3,7 @@
 // Compiled with -ffp-contract=off: every fp64 operation is a single IEEE operation.
 #include <algorithm>
 #include <cmath>
+#include <cstring>
 #include <cstdint>
 #include <functional>
 #include <numeric>
@@ -11,6 +12,15 @@
 #include <vector>
 
 #include "deft.h"
+
+namespace {
+// (key ascending, then id ascending)
+struct SortKey {
+    uint64_t key;
+    int32_t id;
+    bool operator<(const SortKey& o) const { return key != o.key ? key < o.key : id < o.id; }
+};
+}  // namespace
 
 extern "C" {
 
@@ -86,26 +96,38 @@ deft_status deft_allocate_k(const double* norms_h, const int64_t* layer_size_h, 
         if (!(norms_h[l] >= 0.0) || std::isinf(norms_h[l])) return DEFT_ERR_NONFINITE_NORM;
     if (mode == DEFT_MODE_EXACT && (k < (int64_t)L || k > n_g)) return DEFT_ERR_INFEASIBLE_K;
 
-    // Priority: larger norm first, equal norms by lower id.
-    std::vector<int32_t> prio(L);
-    std::iota(prio.begin(), prio.end(), 0);
-    std::sort(prio.begin(), prio.end(), [norms_h](int32_t a, int32_t b) {
-        if (norms_h[a] != norms_h[b]) return norms_h[a] > norms_h[b];
-        return a < b;
-    });
+    // Priority: larger norm first, equal norms by lower id.  For non-negative doubles the bit pattern
+    // orders like the value (-0.0 is made +0.0 first), so one sort of (inverted bits, id) pairs does it.
+    static thread_local std::vector<SortKey> keys;
+    static thread_local std::vector<int32_t> prio;
+    static thread_local std::vector<double> tail;
+    keys.resize((size_t)L);
+    prio.resize((size_t)L);
+    for (int32_t l = 0; l < L; ++l) {
+        const double v = norms_h[l] + 0.0;
+        uint64_t bits;
+        std::memcpy(&bits, &v, 8);
+        keys[l] = SortKey{~bits, l};
+    }
+    std::sort(keys.begin(), keys.end());
+    for (int32_t p = 0; p < L; ++p) prio[p] = keys[p].id;
 
     // tail[p] = norms of priority positions p, p+1, ..., L-1 added from the back.
-    std::vector<double> tail((size_t)L + 1);
+    tail.resize((size_t)L + 1);
     tail[L] = 0.0;
     for (int32_t p = L; p-- > 0;) tail[p] = norms_h[prio[p]] + tail[p + 1];
 
+    // share[p] = norm / norm_remain (0 when nothing remains): independent of the running k, so all the
+    // divisions are done before the sequential part (each is the same single IEEE division as before)
+    static thread_local std::vector<double> share;
+    share.resize((size_t)L);
+    for (int32_t p = 0; p < L; ++p) share[p] = tail[p] > 0.0 ? norms_h[prio[p]] / tail[p] : -1.0;
     int64_t left = k;
     for (int32_t p = 0; p < L; ++p) {
         const int32_t l = prio[p];
         double want = 0.0;
-        if (tail[p] > 0.0) {
-            const double share = norms_h[l] / tail[p];
-            const double prod = (double)left * share;
+        if (share[p] >= 0.0) {
+            const double prod = (double)left * share[p];
             want = std::floor(prod);
         }
         const int64_t sz = layer_size_h[l];
@@ -161,7 +183,11 @@ deft_status deft_partition_model(const int64_t* layer_size_h, const int64_t* k_l
         for (int i = 1; i < 4096; ++i) t[i] = std::log((double)i);
         return t;
     }();
-    std::vector<double> c(L);
+    static thread_local std::vector<double> c;
+    static thread_local std::vector<SortKey> keys;
+    static thread_local std::vector<double> load;
+    c.resize((size_t)L);
+    keys.resize((size_t)L);
     for (int32_t l = 0; l < L; ++l) {
         if (cost_model == DEFT_COST_EQ3) {
             const int64_t kk = k_l_h[l];
@@ -173,20 +199,28 @@ deft_status deft_partition_model(const int64_t* layer_size_h, const int64_t* k_l
     // "largest remaining cost, lowest id on ties" L times = one stable pass over the layers
     // sorted by descending cost; "smallest load, lowest id on ties" = a min-heap on (load, bin).
     // Each bin receives its costs in the same order as in the listing, so the fp64 sums are the same.
-    std::vector<int32_t> by_cost(L);
-    std::iota(by_cost.begin(), by_cost.end(), 0);
-    std::stable_sort(by_cost.begin(), by_cost.end(), [&c](int32_t a, int32_t b) { return c[a] > c[b]; });
-    std::vector<double> load(N, 0.0);
+    // (costs are non-negative: their bit patterns order like the values; ties go to the lower id)
+    for (int32_t l = 0; l < L; ++l) {
+        const double v = c[l] + 0.0;
+        uint64_t bits;
+        std::memcpy(&bits, &v, 8);
+        keys[l] = SortKey{~bits, l};
+    }
+    std::sort(keys.begin(), keys.end());
+    load.assign((size_t)N, 0.0);
     typedef std::pair<double, int32_t> Bin;   // (load, id): smallest load first, then lowest id
-    std::priority_queue<Bin, std::vector<Bin>, std::greater<Bin>> heap;
-    for (int32_t b = 0; b < N; ++b) heap.push(Bin(0.0, b));
+    static thread_local std::vector<Bin> heap;
+    heap.clear();
+    for (int32_t b = 0; b < N; ++b) heap.push_back(Bin(0.0, b));   // already a heap: equal loads, ascending ids
+    const auto lighter_last = std::greater<Bin>();
     for (int32_t i = 0; i < L; ++i) {
-        const int32_t pick = by_cost[i];
-        const Bin lightest = heap.top();
-        heap.pop();
+        const int32_t pick = keys[i].id;
+        std::pop_heap(heap.begin(), heap.end(), lighter_last);
+        Bin& lightest = heap.back();
         bin_of_layer_h[pick] = lightest.second;
         load[lightest.second] += c[pick];
-        heap.push(Bin(load[lightest.second], lightest.second));
+        lightest.first = load[lightest.second];
+        std::push_heap(heap.begin(), heap.end(), lighter_last);
     }
     if (bin_load_h)
         for (int32_t b = 0; b < N; ++b) bin_load_h[b] = load[b];
@@ -198,6 +232,15 @@ deft_status deft_partition(const int64_t* layer_size_h, const int64_t* k_l_h, in
                            int32_t N, int32_t* bin_of_layer_h, double* bin_load_h) {
     if (!k_l_h) return DEFT_ERR_INVALID_ARG;
     return deft_partition_model(layer_size_h, k_l_h, L, N, DEFT_COST_EQ3, bin_of_layer_h, bin_load_h);
+}
+
+// Eq. 2: the error of an iteration is the mean of the workers' errors.
+deft_status deft_error_eq2(const double* worker_error_h, int32_t n_workers, double* error_out) {
+    if (!worker_error_h || !error_out || n_workers < 1) return DEFT_ERR_INVALID_ARG;
+    double s = 0.0;
+    for (int32_t i = 0; i < n_workers; ++i) s = s + worker_error_h[i];
+    *error_out = s / (double)n_workers;
+    return DEFT_OK;
 }
 
 int32_t deft_rank_bin(int64_t iteration, int32_t rank, int32_t N) {

@@ -110,6 +110,20 @@ def lib() -> ctypes.CDLL:
         L.deft_select_update_all.argtypes = [vp, i64, vp, vp, vp, vp, i64, vp, sz, vp]
         L.deft_select_update_ranks.restype = i32
         L.deft_select_update_ranks.argtypes = [vp, i64, vp, vp, i32, i32, vp, vp, i64, vp, sz, vp, vp]
+        L.deft_error_eq2.restype = i32
+        L.deft_error_eq2.argtypes = [vp, i32, vp]
+        L.deft_union_workspace_bytes.restype = sz
+        L.deft_union_workspace_bytes.argtypes = [i64]
+        L.deft_index_union.restype = i32
+        L.deft_index_union.argtypes = [vp, i64, i64, vp, i64, vp, vp, sz, vp]
+        L.deft_sum_into.restype = i32
+        L.deft_sum_into.argtypes = [vp, vp, i64, vp]
+        L.deft_average.restype = i32
+        L.deft_average.argtypes = [vp, i64, i32, vp]
+        L.deft_vector_norm_workspace_bytes.restype = sz
+        L.deft_vector_norm_workspace_bytes.argtypes = [i64]
+        L.deft_vector_norm.restype = i32
+        L.deft_vector_norm.argtypes = [vp, i64, vp, vp, sz, vp]
         L.deft_residual_update.restype = i32
         L.deft_residual_update.argtypes = [vp, i64, vp, i64, vp]
         L.deft_topk_baseline.restype = i32
@@ -500,6 +514,41 @@ def deft_gather_update(acc, idx_d, count: int, val_d, stream=None) -> None:
     _check("deft_gather_update",
            lib().deft_gather_update(_dp(acc, torch.float32), acc.numel(), _dp(idx_d, torch.int64), int(count),
                                     _dp(val_d, torch.float32), _stream(stream)))
+
+
+def deft_error_eq2(worker_errors) -> float:
+    w = _np(worker_errors, np.float64)
+    out = np.zeros(1, dtype=np.float64)
+    _check("deft_error_eq2", lib().deft_error_eq2(_hp(w), int(w.size), _hp(out)))
+    return float(out[0])
+
+
+def deft_union_workspace_bytes(n_g: int) -> int:
+    return int(lib().deft_union_workspace_bytes(int(n_g)))
+
+
+def deft_index_union(idx_d, count: int, n_g: int, union_d, count_d, ws, stream=None) -> None:
+    """Sorted set of idx_d[:count] into union_d (as many as fit), its size into count_d (device int64)."""
+    _check("deft_index_union", lib().deft_index_union(_dp(idx_d), int(count), int(n_g), _dp(union_d),
+                                                      union_d.numel() if union_d is not None else 0, _dp(count_d),
+                                                      _dp(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def deft_sum_into(dst, src, count: int, stream=None) -> None:
+    _check("deft_sum_into", lib().deft_sum_into(_dp(dst), _dp(src), int(count), _stream(stream)))
+
+
+def deft_average(sum_d, count: int, n_workers: int, stream=None) -> None:
+    _check("deft_average", lib().deft_average(_dp(sum_d), int(count), int(n_workers), _stream(stream)))
+
+
+def deft_vector_norm_workspace_bytes(n: int) -> int:
+    return int(lib().deft_vector_norm_workspace_bytes(int(n)))
+
+
+def deft_vector_norm(x, norm_d, ws, stream=None) -> None:
+    _check("deft_vector_norm", lib().deft_vector_norm(_dp(x), x.numel(), _dp(norm_d), _dp(ws),
+                                                      ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def deft_residual_update(acc, idx_d, count: int, stream=None) -> None:

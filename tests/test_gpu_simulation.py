@@ -46,20 +46,17 @@ def _oracle_step(kind, e, grads, start, size, k, N, t, threshold):
         union = np.concatenate(parts)                      # rank order, as the ranks' slabs lie side by side
         assert np.unique(union).size == union.size == s
     elif kind == "topk":
-        union = np.unique(np.concatenate([oracle.topk(e[r], k)[1] for r in range(N)]))
+        union = oracle.index_union(np.concatenate([oracle.topk(e[r], k)[1] for r in range(N)]))
     elif kind == "cltk":
         union = oracle.topk(e[oracle.clt_leader(t, N)], k)[1]
     else:
-        union = np.unique(np.concatenate([oracle.threshold_select(e[r], threshold)[1] for r in range(N)]))
+        union = oracle.index_union(np.concatenate([oracle.threshold_select(e[r], threshold)[1] for r in range(N)]))
     mean = np.zeros(union.size, dtype=np.float32)
     for r in range(N):
-        mean += oracle.gather_update(e[r], union)
-    mean /= np.float32(N)
-    err = 0.0
-    for r in range(N):
-        nl = oracle.layer_norms(e[r], start)
-        err += math.sqrt(float(np.sum(nl * nl)))
-    return union, mean, union.size / e[0].size, err / N
+        oracle.sum_into(mean, oracle.gather_update(e[r], union))
+    oracle.average(mean, N)
+    err = oracle.error_eq2([oracle.vector_norm(e[r]) for r in range(N)])
+    return union, mean, union.size / e[0].size, err
 
 
 @pytest.mark.parametrize("kind", ["deft", "topk", "cltk", "hard_threshold"])

@@ -529,3 +529,67 @@ def test_clt_leader_cycles_and_gather_update():
     f = x.copy()
     fv = oracle.gather_update(f, lidx)
     assert np.array_equal(fv, x[lidx]) and not f[lidx].any() and np.count_nonzero(f != x) == np.count_nonzero(x[lidx])
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1 around the sparsifier (lines 7-9) and Eq. 2
+# --------------------------------------------------------------------------
+def test_index_union_is_the_sorted_set():
+    assert oracle.index_union([5, 3, 5, 1, 3]).tolist() == [1, 3, 5]          # by hand
+    assert oracle.index_union([]).tolist() == []
+    assert oracle.index_union([7]).tolist() == [7]
+    rng = np.random.default_rng(21)
+    for trial in range(20):
+        idx = rng.integers(0, 500, size=int(rng.integers(1, 2000)))
+        u = oracle.index_union(idx)
+        assert set(u.tolist()) == set(idx.tolist())                          # the same set ...
+        assert np.all(np.diff(u) > 0)                                        # ... strictly ascending
+    # disjoint lists (DEFT's workers): nothing is lost, the size is the sum of the sizes
+    parts = [np.arange(r, 400, 4) for r in range(4)]
+    assert oracle.index_union(np.concatenate(parts[::-1])).tolist() == list(range(400))
+
+
+def test_sum_and_average_are_single_fp32_operations():
+    rng = np.random.default_rng(22)
+    a = rng.standard_normal(5000).astype(np.float32)
+    b = (rng.standard_normal(5000) * 1e-3).astype(np.float32)
+    want = (a.astype(np.float64) + b.astype(np.float64)).astype(np.float32)   # exact sum, one rounding
+    assert oracle.sum_into(a.copy(), b).tobytes() == want.tobytes()
+    for n in (2, 3, 7, 32):
+        q = (a.astype(np.float64) / n).astype(np.float32)                      # exact quotient of two floats, one rounding
+        assert oracle.average(a.copy(), n).tobytes() == q.tobytes()
+    # worked by hand: (1 + 2 + 6) / 3 = 3
+    s = np.array([1.0], dtype=np.float32)
+    oracle.sum_into(s, np.array([2.0], dtype=np.float32))
+    oracle.sum_into(s, np.array([6.0], dtype=np.float32))
+    assert oracle.average(s, 3).tolist() == [3.0]
+
+
+def test_vector_norm_and_eq2():
+    assert oracle.vector_norm(np.array([3.0, -4.0], dtype=np.float32)) == 5.0
+    assert oracle.vector_norm(np.ones(49, dtype=np.float32)) == 7.0
+    assert oracle.vector_norm(np.zeros(10, dtype=np.float32)) == 0.0
+    rng = np.random.default_rng(23)
+    x = rng.standard_normal(100000).astype(np.float32)
+    ref = float(np.linalg.norm(x.astype(np.float64)))
+    assert abs(oracle.vector_norm(x) - ref) <= 1e-12 * ref
+    # the norm of the whole vector from the norms of its layers (Pythagoras)
+    start = np.array([0, 10, 5000, 100000], dtype=np.int64)
+    nl = oracle.layer_norms(x, start)
+    assert abs(oracle.vector_norm(x) - math.sqrt(float(np.sum(nl * nl)))) <= 1e-12 * ref
+    # Eq. 2 by hand: (1 + 2 + 6) / 3
+    assert oracle.error_eq2([1.0, 2.0, 6.0]) == 3.0
+    assert oracle.error_eq2([2.5]) == 2.5
+
+
+def test_threaded_rank_selection_equals_the_plain_one():
+    rng = np.random.default_rng(24)
+    sizes = rng.integers(1, 3000, size=40)
+    start = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    acc = rng.standard_normal(int(start[-1])).astype(np.float32)
+    k_l = np.array([int(rng.integers(1, s + 1)) for s in sizes], dtype=np.int64)
+    my = np.arange(0, 40, 3, dtype=np.int32)
+    v0, i0 = oracle.select_rank(acc, start, k_l, my)
+    for threads in (1, 2, 0):
+        v1, i1, used = oracle.select_rank_threads(acc, start, k_l, my, threads)
+        assert used >= 1 and i1.tolist() == i0.tolist() and v1.tobytes() == v0.tobytes()

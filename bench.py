@@ -91,7 +91,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:  # noqa: BLE001
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.002)
 
     def start(self):
         if self._h is not None:
@@ -110,10 +110,12 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # the oracle on the host cores (CPU baseline and --impl reference)
 # ------------------------------------------------------------------------------------------
-def oracle_step_sample(w, g, budget_ranks: int = 4):
-    """One step of the oracle on a bounded sample: accumulate + norms over the whole vector,
-    both planners, then selection + zeroing for `budget_ranks` evenly spaced ranks; the rank
-    part is scaled to all N ranks by the elements scanned."""
+def oracle_step_sample(w, g, budget_ranks: int = 4, threads: int = 1, topk_slice: int = 0):
+    """One step of the oracle on a bounded sample, every part timed on its own: accumulate + norms over the
+    whole vector, both planners, then selection + zeroing for `budget_ranks` evenly spaced ranks (one host
+    thread; with threads != 1 the same ranks again with their layers farmed out over that many threads,
+    0 = all the hardware reports), and the conventional Top-k's sort on the first `topk_slice` elements.
+    The step time for all N ranks is an ESTIMATE: the rank part scaled by the elements scanned."""
     import oracle
     N = w.n_workers
     start, _ = oracle.split_layers(w.sizes, N)
@@ -129,25 +131,54 @@ def oracle_step_sample(w, g, budget_ranks: int = 4):
     t2 = time.perf_counter()
     ranks = sorted(set(int(round(i * N / budget_ranks)) % N for i in range(min(budget_ranks, N))))
     elems = 0
-    t_sel = 0.0
+    per_rank, per_rank_mt = [], []
+    used = 1
     for r in ranks:
         my = oracle.my_layers(bins, 0, r, N)
+        if threads != 1:   # before the single-thread pass zeroes the selected entries
+            ta = time.perf_counter()
+            _, _, used = oracle.select_rank_threads(e, start, k_l, my, threads)
+            per_rank_mt.append(time.perf_counter() - ta)
         ta = time.perf_counter()
         val, idx = oracle.select_rank(e, start, k_l, my)
         oracle.residual_update(e, idx)
-        t_sel += time.perf_counter() - ta
+        per_rank.append(time.perf_counter() - ta)
         elems += int(size[my].sum())
+    t_topk = None
+    if topk_slice:
+        n = min(int(topk_slice), w.n_g)
+        ta = time.perf_counter()
+        oracle.topk(e[:n], max(1, int(n * w.density)))
+        t_topk = time.perf_counter() - ta
     scale = w.n_g / max(1, elems)
+    t_sel = float(sum(per_rank))
     est = (t1 - t0) + (t2 - t1) + t_sel * scale
-    return {
-        "est_step_s": est, "t_acc_norms_s": t1 - t0, "t_planners_s": t2 - t1, "t_select_sampled_s": t_sel,
+    out = {
+        "est_step_s": est, "sampled_s": (t1 - t0) + (t2 - t1) + t_sel, "t_acc_norms_s": t1 - t0,
+        "t_planners_s": t2 - t1, "t_select_sampled_s": t_sel,
+        "t_select_rank_max_s": float(max(per_rank)), "t_select_rank_mean_s": float(np.mean(per_rank)),
         "ranks_sampled": ranks, "elems_sampled": elems, "scale": scale,
         "sample": "accumulate+norms over all %d elements, Algorithms 3+4, then selection+zeroing of ranks %s "
-                  "(%d elements) scaled by %.2f to all %d ranks" % (w.n_g, ranks, elems, scale, N),
+                  "(%d elements); the step for all %d ranks is estimated by scaling the rank part by %.2f" % (
+                      w.n_g, ranks, elems, N, scale),
     }
+    if per_rank_mt:
+        est_mt = (t1 - t0) + (t2 - t1) + float(sum(per_rank_mt)) * scale
+        out["all_cores"] = {"cores": used, "t_select_rank_max_s": float(max(per_rank_mt)),
+                            "t_select_rank_mean_s": float(np.mean(per_rank_mt)), "est_step_s": est_mt,
+                            "note": "layers of a rank farmed out over host threads (selection only; accumulate+norms "
+                                    "and the planners stay on one thread)"}
+    if t_topk is not None:
+        out["topk_sort"] = {"elements": min(int(topk_slice), w.n_g), "seconds": t_topk,
+                            "note": "full sort of (key, index) pairs on a prefix of the vector, one thread"}
+    return out
 
 
 def run_reference(args):
+    """The oracle, as it stands, on the host cores.  A step here is a bounded SAMPLE of the workload (the oracle
+    sorts; all 32 ranks of the 333 M-element vector take about half a minute per step): `ms_per_step` is the
+    wall time of the sampled step, `value` the throughput estimated from it for the whole step, and the
+    line says so ("estimated": true)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -159,17 +190,29 @@ def run_reference(args):
         oracle_step_sample(w, g, 1)
     res = [oracle_step_sample(w, g, args.cpu_ranks) for _ in range(steps)]
     est = float(np.mean([r["est_step_s"] for r in res]))
+    sampled = float(np.mean([r["sampled_s"] for r in res]))
     val = w.n_g / est / 1e9
     out = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": warm, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": warm, "ms_per_step": sampled * 1e3, "estimated": True, "est_full_step_ms": est * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "n_g": w.n_g, "n_workers": w.n_workers, "density": w.density, "k": w.k,
                    "seed": w.seed},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": res[-1]["sample"]},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": res[-1]["sample"],
+                         "estimated": True},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(out))
+
+
+def ncu_traffic():
+    """Per-element DRAM traffic of the kernels as measured by ncu (committed summaries under profiles/)."""
+    p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f)
+    return None
 
 
 # ------------------------------------------------------------------------------------------
@@ -294,6 +337,78 @@ def run_trace(args, dev):
                       "deft_at_topk_density": {"density": d_match, "rows": matched}}))
 
 
+def run_extra(dev):
+    """Short runs of the other configurations: the LSTM-shaped vector with the residual carried over 10 steps
+    (timed at step 10 and averaged over the 10), and six corners of the GPT-2-medium-shaped sweep
+    (density x workers): the whole step with all workers in one launch, the slowest worker's own launch, and
+    full-vector Top-k on the same vector.  A fresh device-side draw every step."""
+    import torch
+    from paper_2307_03500_b200 import deft
+    from paper_2307_03500_b200.pipeline import DeftStep
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def config(w, steps, warm):
+        N = w.n_workers
+        ds = DeftStep(w.sizes, N, w.density, device=dev)
+        e = torch.zeros(ds.n_g, dtype=torch.float32, device=dev)
+        g = torch.empty(ds.n_g, dtype=torch.float32, device=dev)
+        tk_val = torch.empty(ds.k, dtype=torch.float32, device=dev)
+        tk_idx = torch.empty(ds.k, dtype=torch.int64, device=dev)
+        tk_ws = deft.alloc_workspace(ds.n_g, 1, dev)
+        step_ms, sel_ms, topk_ms, rank_max = [], [], [], []
+        for it in range(warm + steps):
+            W.device_gradient(w, it, dev, out=g)
+            evs = [ev(), ev(), ev(), ev()]
+            a, b = ev(), ev()
+            a.record(stream)
+            ds.step_fused(e, g, it, -1, evs)
+            b.record(stream)
+            stream.synchronize()
+            if it >= warm:
+                step_ms.append(a.elapsed_time(b))
+                sel_ms.append(evs[2].elapsed_time(evs[3]))
+        for it in range(warm + steps, warm + steps + 3):   # per-worker launches and Top-k on the same vectors
+            W.device_gradient(w, it, dev, out=g)
+            deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)
+            ta, tb = ev(), ev()
+            ta.record(stream)
+            deft.deft_topk_baseline(e, ds.k, tk_val, tk_idx, tk_ws)
+            tb.record(stream)
+            ds.norms_h.copy_(ds.norms_d, non_blocking=True)
+            stream.synchronize()
+            plan = ds.plan(ds.norms_h.numpy(), it)
+            tri = [(ev(), ev(), ev()) for _ in range(N)]
+            for t3 in tri:
+                for x in t3:
+                    x.record(stream)
+            ds.select_and_update_all(e, plan, tri)
+            stream.synchronize()
+            topk_ms.append(ta.elapsed_time(tb))
+            rank_max.append(max(x.elapsed_time(y) for (x, y, z) in tri))
+        st = deft.deft_select_stats(ds.ws, ds.L)
+        row = {"workload": w.name, "n_g": ds.n_g, "n_workers": N, "density": w.density, "k": ds.k, "layers": ds.L,
+               "ms_per_step": float(np.mean(step_ms)), "ms_last_step": float(step_ms[-1]), "steps": steps,
+               "select_all_workers_one_launch_ms": float(np.median(sel_ms)),
+               "select_slowest_worker_ms": float(np.median(rank_max)), "topk_ms": float(np.median(topk_ms[1:])),
+               "speedup_vs_topk": float(np.median(topk_ms[1:]) / np.median(rank_max)), "layer_counters": st}
+        del ds, e, g, tk_val, tk_idx, tk_ws
+        torch.cuda.empty_cache()
+        return row
+
+    rows = []
+    lstm = W.WORKLOADS["lstm_lm"]()
+    r = config(lstm, 10, 0)   # residual carried over 10 steps from zero: no warm-up, the first call has no remembered cuts
+    r["note"] = "residual carried over 10 seeded steps; ms_per_step = mean over the 10, ms_last_step = step 10"
+    rows.append(r)
+    for d in (0.1, 0.001):
+        for N in (1, 8, 64):
+            rows.append(config(W.gpt2_medium(N, d), 3, 3))
+    return rows
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -411,6 +526,7 @@ def run_ours(args):
             elif args.mode == "norms":
                 deft.deft_layer_norms(e, g, ds.layer_start_d, ds.norms_d, ds.ws)
             else:
+                deft.deft_plan_upload(plan.plan_h, ds.plan_d, ds.ws)   # the per-layer counters are single-use
                 ds.select_rank(e, plan, r_big)
             b.record(stream)
             stream.synchronize()
@@ -425,6 +541,7 @@ def run_ours(args):
         one_step(it)
     barrier()
 
+    stats0 = deft.deft_select_stats(ds.ws, L)
     sampler = ClockSampler(local)
     sampler.start()
     recs = []
@@ -439,6 +556,29 @@ def run_ours(args):
     clocks = sampler.stop()
     total_ms = t_begin.elapsed_time(t_end)
     gpu_launches = launches["n"]
+    stats1 = deft.deft_select_stats(ds.ws, L)
+    layer_stats = {kk: stats1[kk] - stats0[kk] for kk in stats1}   # streamed layers over the timed steps
+
+    # a second, non-stationary stream: a pool of 4 draws cycled (the accumulated vector and with it every
+    # layer's threshold keep shifting against the norms), same step, same timing
+    ns_steps = max(8, min(args.steps, 40))
+    ns_pool = pool[:4] if len(pool) >= 4 else pool
+    ns_recs = []
+    s_a = deft.deft_select_stats(ds.ws, L)
+    tn0, tn1 = ev(), ev()
+    for it in range(4):
+        one_step(args.warmup + args.steps + it, None, ns_pool[it % len(ns_pool)])
+    barrier()
+    tn0.record(stream)
+    s_a = deft.deft_select_stats(ds.ws, L)
+    for it in range(ns_steps):
+        one_step(args.warmup + args.steps + 4 + it, ns_recs, ns_pool[it % len(ns_pool)])
+    tn1.record(stream)
+    barrier()
+    s_b = deft.deft_select_stats(ds.ws, L)
+    ns_ms = tn0.elapsed_time(tn1) / ns_steps
+    ns_sel = np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in ns_recs])
+    ns_stats = {kk: s_b[kk] - s_a[kk] for kk in s_b}
 
     # per-call statistics from the events recorded inside the timed region
     t_acc = np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in recs])
@@ -518,6 +658,14 @@ def run_ours(args):
     barrier()
     e2e_ms = te0.elapsed_time(te1) / e2e_steps
 
+    # the other configurations, a few steps each (rank 0 of a single-GPU run only)
+    extra = None
+    if world == 1 and not args.no_extra:
+        del g_stage
+        pool.clear()
+        torch.cuda.empty_cache()
+        extra = run_extra(dev)
+
     # max over ranks of the job
     ms_per_step = total_ms / args.steps
     if world > 1:
@@ -539,37 +687,60 @@ def run_ours(args):
         r_max = int(np.argmax(sel_med))
         cost_max = float(plan_w.bin_load.max())
         lnk = math.log(k)
-        # the all-ranks launch of the timed step
+        # the all-ranks launch of the timed step.  Bytes MOVED: a layer whose remembered cut held is read once;
+        # one whose cut failed, or that had none, is read again with the true cut after its histogram (twice
+        # more in the five-step kernel, twice in all on the single-pass kernel's retry list).  The layer
+        # counters of the library say how many layers went which way; layers are weighted equally here.
+        traffic = ncu_traffic() or {}
         all_ms = float(np.median(t_all))
         all_bytes = 8.0 * n_g + 12.0 * float(plan.sum_k)
         all_gbs = all_bytes / (all_ms * 1e-3) / 1e9
-        moved_bytes = 4.0 * n_g + 12.0 * float(plan.sum_k) + 4.0e6 * n_g / 135891278.0
-        roof_sel = {"bound": "hbm", "kernel": "k_select_fused (all %d workers' partitions in one launch)" % N,
-                    "achieved": all_gbs, "peak": peak, "unit": "GB/s", "frac": all_gbs / peak, "peak_kind": peak_kind,
-                    "traffic": 4.0 * n_g + 4.0e6 * n_g / 135891278.0,
-                    "traffic_note": "per launch, scaled by elements from an ncu capture on 135.9 M elements: 4.00 "
-                                    "B/element read + 4 MB written when the remembered cut holds (the vector is read "
-                                    "ONCE: half of the two-read algorithmic bytes are never moved); 8.00 B/element "
-                                    "in a call without a usable cut",
-                    "bytes_per_launch": all_bytes, "ms_per_launch": all_ms, "bytes_per_elem": 8,
-                    "bytes_per_selected": 12, "share_of_step": all_ms / ms_per_step,
+        n_layers_seen = max(1, sum(layer_stats.values()))
+        reread = (layer_stats["cut_failed"] + layer_stats["no_cut"]) / n_layers_seen
+        moved_bytes = 4.0 * n_g * (1.0 + 2.0 * reread) + 12.0 * float(plan.sum_k)
+        moved_gbs = moved_bytes / (all_ms * 1e-3) / 1e9
+        sel_traffic = traffic.get("selection_one_read")
+        roof_sel = {"bound": "hbm", "kernel": "selection of all %d workers' partitions in one launch "
+                                              "(k_select_stream for calls of 48 M elements or more, else k_select_fused)" % N,
+                    "achieved": moved_gbs, "peak": peak, "unit": "GB/s", "frac": moved_gbs / peak, "peak_kind": peak_kind,
+                    "achieved_note": "bytes moved per launch (4 B per element read once where the remembered cut held, "
+                                     "12 B per element where it did not, 12 B per selected entry) / event-timed duration",
+                    "traffic": (sel_traffic["dram_bytes_per_elem"] * n_g if sel_traffic else None),
+                    "traffic_note": ("per launch, scaled by elements from the ncu capture in %s" % sel_traffic["source"])
+                                    if sel_traffic else "no ncu summary found",
+                    "bytes_per_launch": moved_bytes, "ms_per_launch": all_ms, "share_of_step": all_ms / ms_per_step,
                     "ms_per_launch_mean": float(np.mean(t_all)), "ms_per_launch_max": float(np.max(t_all)),
-                    "launches_above_1p25_median": int((t_all > 1.25 * all_ms).sum()),
-                    "achieved_on_bytes_moved": moved_bytes / (all_ms * 1e-3) / 1e9,
-                    "frac_on_bytes_moved": moved_bytes / (all_ms * 1e-3) / 1e9 / peak}
+                    "layers_one_read": layer_stats["one_read"], "layers_cut_failed": layer_stats["cut_failed"],
+                    "layers_no_cut": layer_stats["no_cut"], "share_of_layers_read_again": reread,
+                    "frac_algorithmic": all_gbs / peak,
+                    "frac_algorithmic_note": "two-read definition: (8 B per element + 12 B per selected entry) / time / peak; "
+                                             "half of those bytes are never moved when the cut holds"}
+        acc_traffic = traffic.get("k_accum_norms")
         roof_acc = {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,
-                    "peak": peak, "unit": "GB/s", "frac": acc_gbs / peak, "peak_kind": peak_kind,
-                    "traffic": 11.66 * n_g,
-                    "traffic_note": "per launch, scaled by elements from an ncu capture on 135.9 M elements "
-                                    "(8.00 B/element read + 3.66 written before the kernel ends)",
+                    "peak": peak, "unit": "GB/s", "frac": min(1.0, acc_gbs / peak), "frac_uncapped": acc_gbs / peak,
+                    "frac_note": "the denominator is a measured copy (half reads, half writes); this kernel reads two "
+                                 "bytes for every byte it writes and runs a little above it: capped at 1",
+                    "peak_kind": peak_kind,
+                    "traffic": (acc_traffic["dram_bytes_per_elem"] * n_g if acc_traffic else None),
+                    "traffic_note": ("per launch, scaled by elements from the ncu capture in %s" % acc_traffic["source"])
+                                    if acc_traffic else "no ncu summary found",
                     "bytes_per_launch": acc_bytes, "ms_per_launch": acc_ms, "share_of_step": acc_ms / ms_per_step,
                     "frac_of_nominal_8TBs": acc_gbs / 8000.0}
         sel_dominant = all_ms >= acc_ms
         cpu = None
         if not args.no_cpu_baseline:
-            c = oracle_step_sample(w, g_host.numpy(), args.cpu_ranks)
+            c = oracle_step_sample(w, g_host.numpy(), args.cpu_ranks, threads=0, topk_slice=1 << 25)
             cpu = {"value": n_g / c["est_step_s"] / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                   "sample": c["sample"], "est_ms_per_step": c["est_step_s"] * 1e3}
+                   "estimated": True, "sample": c["sample"], "est_ms_per_step": c["est_step_s"] * 1e3,
+                   "measured_s": {"accumulate_norms": c["t_acc_norms_s"], "planners": c["t_planners_s"],
+                                  "select_rank_max": c["t_select_rank_max_s"], "select_rank_mean": c["t_select_rank_mean_s"],
+                                  "ranks_sampled": c["ranks_sampled"]},
+                   "topk_sort": c.get("topk_sort")}
+            if "all_cores" in c:
+                ac = c["all_cores"]
+                cpu["all_cores"] = {"cores": ac["cores"], "value": n_g / ac["est_step_s"] / 1e9, "unit": UNIT,
+                                    "select_rank_max_s": ac["t_select_rank_max_s"],
+                                    "select_rank_mean_s": ac["t_select_rank_mean_s"], "note": ac["note"]}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -589,15 +760,18 @@ def run_ours(args):
             "roofline": roof_sel if sel_dominant else roof_acc,
             "roofline_other": roof_acc if sel_dominant else roof_sel,
             "roofline_select_per_worker": {
-                "bound": "hbm", "call": "k_select_fused, one launch per worker (timed outside the step)",
-                "bytes_per_elem": 8, "bytes_per_selected": 12, "unit": "GB/s", "peak": peak,
-                "achieved_mean": float(sel_gbs[busy].mean()), "achieved_min": float(sel_gbs[busy].min()),
-                "achieved_max": float(sel_gbs[busy].max()), "frac_mean": float(sel_gbs[busy].mean() / peak),
-                "frac_slowest_rank": float(sel_gbs[r_max] / peak),
+                "bound": "hbm", "call": "one selection launch per worker (timed outside the step)",
+                "unit": "GB/s", "peak": peak,
+                "frac_mean": float((sel_gbs[busy] / 2.0).mean() / peak), "frac_slowest_rank": float(sel_gbs[r_max] / 2.0 / peak),
+                "frac_note": "bytes moved (4 B per element: the vector is read once when the remembered cut holds) / time / peak",
+                "frac_algorithmic_mean": float(sel_gbs[busy].mean() / peak),
+                "frac_algorithmic_slowest_rank": float(sel_gbs[r_max] / peak),
+                "frac_algorithmic_note": "two-read definition, 8 B per element + 12 B per selected entry; the target of "
+                                         ">= 0.6 per simulated rank refers to it and is NOT met",
+                "us_slowest_rank": float(sel_med.max() * 1e3), "us_mean": float(sel_med[busy].mean() * 1e3),
                 "floor_us_mean": float(sel_bytes[busy].mean() / peak / 1e3),
-                "traffic_per_elem_ncu": 4.02,
-                "note": "ranks of 8-16 M elements are latency-bound (floor 5-10 us, four grid barriers); "
-                        "the vector is read once when the remembered cut holds"},
+                "note": "ranks of 8-16 M elements are latency-bound: 33-60 MB take 13-15 us to stream even for a bare "
+                        "read kernel timed the same way; setup, four grid barriers and the steps between them add the rest"},
             "worker_view": {"ms_per_step_slowest_worker": worker_ms, "gelems": n_g / (worker_ms * 1e-3) / 1e9,
                             "t_acc_norms_ms": acc_ms, "t_host_ms": float(np.median(t_host)),
                             "t_host_note": "device-idle time between the norms and the selection launch: D2H copy of "
@@ -626,6 +800,18 @@ def run_ours(args):
                                    "frac": (4.0 * n_g + 12.0 * n_thr) / (t_thr * 1e-3) / 1e9 / peak},
                 "clt_k": {"leader_select_ms": t_topk, "follower_gather_ms": t_gather, "entries": k - 1}},
             "cpu_baseline": cpu,
+            "stream_nonstationary": {
+                "stream": "nonstationary", "what": "a pool of %d draws cycled while the residual accumulates" % len(ns_pool),
+                "steps": ns_steps, "ms_per_step": ns_ms, "select_ms_median": float(np.median(ns_sel)),
+                "select_ms_mean": float(np.mean(ns_sel)), "select_ms_max": float(np.max(ns_sel)),
+                "layers_one_read": ns_stats["one_read"], "layers_cut_failed": ns_stats["cut_failed"],
+                "layers_no_cut": ns_stats["no_cut"]},
+            "stream_stationary": {
+                "stream": "stationary", "what": "an independent draw every step", "steps": args.steps,
+                "ms_per_step": ms_per_step, "select_ms_median": all_ms, "select_ms_mean": float(np.mean(t_all)),
+                "select_ms_max": float(np.max(t_all)), "layers_one_read": layer_stats["one_read"],
+                "layers_cut_failed": layer_stats["cut_failed"], "layers_no_cut": layer_stats["no_cut"]},
+            "extra": extra,
         }
         print(json.dumps(out))
     if world > 1:
@@ -643,6 +829,7 @@ def main():
     ap.add_argument("--density", type=float, default=0.0)
     ap.add_argument("--cpu-ranks", type=int, default=4, help="ranks the oracle runs for the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--pool", type=int, default=105,
                     help="independent gradient draws kept on the device (one per step; cycled beyond that)")
     ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select", "sweep", "trace"],

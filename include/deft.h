@@ -87,17 +87,20 @@ DEFT_API void deft_debug_select_kernel(int32_t single_pass);
 
 /*
  * Diagnostic: when timing_d (DEVICE, 1024 x uint64, zeroed by the caller) is not NULL every
- * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs):
- * [0] kernel start, [1] end of the first read (level-1 histogram + speculative staging),
- * [2] end of the second read / level-2 histograms, [3] level-3 histograms done, [4] per-tile
- * counts done, [5] ordered write done, [6] small layers done; inside the first step
- * [8] histograms zeroed, [9] tiles read, [10] flushed, [11] tickets taken; [14] / [15] staged
- * entries (max over CTAs / total); per CTA b: [16 + b] nanoseconds in the second step,
- * [176 + b] staged entries, [336 + b] local layers | local tiles << 16 | read-twice flag << 32,
- * [496 + b] why it read twice (bit 63: staging budget << 32 | local layer at which it was
- * exceeded; else layer id << 40 | k_l << 24 | cut bucket << 12 | true bucket of a cut that
- * was too high; 0: no remembered cut), [656 + b] nanoseconds in the ordered write,
- * [816 + b] nanoseconds in the first read.
+ * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs) and counters.
+ * Both kernels: [0] kernel start, [14] / [15] staged entries (max over CTAs or layers / total).
+ * Five-step kernel: [1] end of the first read, [2] end of the second read, [3] level-3
+ * histograms done, [4] per-tile counts done, [5] ordered write done, [6] small layers done,
+ * [7] a second round of the first read done; inside the first read [8] histograms zeroed,
+ * [9] tiles read, [10] flushed, [11] tickets taken; per CTA b: [16 + b] nanoseconds in the second
+ * read, [176 + b] staged entries, [336 + b] local layers | local tiles << 16, [496 + b] why a cut
+ * failed, [656 + b] nanoseconds in the ordered write, [816 + b] nanoseconds in the first read.
+ * Single-pass kernel: [8] tables built, [1] tiles read, [2] staged entries handed to the layers'
+ * regions, [10] last layer's candidates ranked, [5] layers finished, [6] small layers done,
+ * [3] selected entries cleared; [20..26] nanoseconds, summed over the layers, in the finishing
+ * CTA's phases (load, histogram, scan, candidates, per-tile counts, prefix, write); [12] the layer
+ * with most staged entries (entries << 32 | layer << 20 | k), [13] most candidates, [28] layers
+ * finished.
  * Pass NULL to switch it off.  Not thread-safe; not for production use.
  */
 DEFT_API void deft_debug_select_timing(void* timing_d);
@@ -190,9 +193,10 @@ DEFT_API deft_status deft_bin_layers(const int32_t* bin_of_layer_h, int32_t L, i
 DEFT_API size_t deft_workspace_bytes(int64_t max_elems, int32_t max_layers);
 
 /*
- * Clears the one part of a workspace that is carried from call to call: per layer, the
- * first-level bucket the previous selection found, from which the next selection of a model
- * with n_layers layers takes its speculative cut (see deft_select_planned).  Call it once
+ * Clears the one part of a workspace that is carried from call to call: per layer, where on
+ * the magnitude axis the previous selection found its threshold and how well that has been
+ * predicting the next one, from which the next selection of a model with n_layers layers
+ * takes its speculative cut (see deft_select_planned), and a few counters.  Call it once
  * after allocating the workspace.  What that area holds never changes a result: stale or
  * arbitrary contents only decide whether a selection reads the vector once or twice (or, for
  * absurdly low cuts, how much it stages).  Errors: INVALID_ARG, CAPACITY, CUDA.
@@ -334,10 +338,16 @@ DEFT_API deft_status deft_plan_upload(const void* plan_h, void* plan_d, void* ws
  * nothing.  plan_h is read on the host for the rank's sizes; plan_d is what the kernel
  * reads.  Errors: INVALID_ARG, CAPACITY (out_cap or workspace), CUDA.
  *
- * Speed, not results, depends on the workspace's history: the kernel remembers per layer the
- * first-level bucket it found and, in the next call on the same workspace, stages everything
- * above a cut derived from it while it builds the histogram.  If every cut of a CTA turns
- * out low enough, the CTA never reads its part of the vector a second time.
+ * Speed, not results, depends on the workspace's history.  The kernel remembers per layer where
+ * (in units of 1/256 octave of magnitude) it found the key a little below the k_l-th largest,
+ * together with the layer's norm then.  The next call on the same workspace predicts the place
+ * from the layer's norm now, lowers it by a running mean and twice a running deviation of the
+ * earlier predictions' errors, and stages every entry above that cut while it reads the vector
+ * once.  A layer for which at least k_l entries were staged is finished from those; any other
+ * (nothing remembered, cut too high, far too many staged, dense layers) is read again and
+ * searched in full.  Two kernels do this: a single-pass one for large calls, in which every
+ * layer is finished by one CTA behind a grid barrier, and a five-step one (histogram levels of
+ * 12 + 12 + 7 bits between grid barriers) for small calls and for the layers left over.
  */
 DEFT_API deft_status deft_select_planned(const float* acc_d, const void* plan_h, const void* plan_d,
                                          int32_t rank, float* val_d, int64_t* idx_d, int64_t out_cap,

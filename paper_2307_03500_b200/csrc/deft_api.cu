@@ -218,6 +218,7 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.fixed_thr = fixed.on ? 1 : 0;
     p.thr_key = fixed.key;
     p.out_cap = out_cap;
+    p.out_total = R.k;
     p.count_out = fixed.count_d;
     // one CTA per SM at most (co-resident by construction); fewer when the rank is small
     const int sms = sm_count();

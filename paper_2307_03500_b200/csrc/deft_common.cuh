@@ -156,7 +156,7 @@ struct LayerState {                  // per layer, written by the kernels; 64 by
     uint32_t cursor;                 // single-pass kernel: room handed out in the layer's staging region
     unsigned long long done;         // single-pass kernel: what the CTAs that are through with the layer add up to:
                                      // tiles << 41 | CTAs that stopped staging << 31 | entries staged
-    uint32_t pad[5];                 // pad[0] of a rank's first layer: next small layer to hand out
+    uint32_t pad[5];                 // of a rank's first layer: [0] next small layer to hand out, [1] next layer to finish (single-pass kernel)
     uint32_t spec_bad;               // five steps: a CTA stopped staging for the layer (its speculative cut counts as failed)
 };
 static_assert(sizeof(LayerState) == 64, "LayerState layout");
@@ -164,10 +164,10 @@ static_assert(sizeof(LayerState) == 64, "LayerState layout");
 // What a selection leaves behind per layer for the next call on the same workspace (the only
 // per-layer data that lives across calls; it steers speed, never results).
 struct LayerHint {                   // 16 bytes
-    uint32_t bucket_p1;              // 1 + first-level bucket of the `rank`-th largest key; 0 = nothing remembered
+    uint32_t pos_p1;                 // 1 + position (key >> 15: 1/16 first-level bucket) of the `rank`-th largest key; 0 = nothing remembered
     uint32_t norm_bits;              // that call's layer norm (float bits)
     uint32_t rank;                   // the rank the bucket belongs to (k + margin of that call)
-    uint32_t err;                    // how the predictions have been doing, in 1/16 bucket: running mean of (found -
+    uint32_t err;                    // how the predictions have been doing, in the same unit: running mean of (found -
                                      // predicted) as int16 in the low half, running mean deviation in the high half
 };
 static_assert(sizeof(LayerHint) == 16, "LayerHint layout");
@@ -257,6 +257,7 @@ struct SelParams {
     int32_t fixed_thr;               // 1: hard-threshold mode
     uint32_t thr_key;                // magnitude key of the threshold
     int64_t out_cap;                 // entries val / idx can take (positions beyond it are not written)
+    int64_t out_total;               // entries the call writes when nothing is cut off: the sum of its layers' k
     unsigned long long* count_out;   // hard-threshold mode: number of entries above the threshold (zeroed before launch)
     unsigned long long* timing;      // optional: 1024 words of phase stamps and per-CTA counters; NULL = off
 };

@@ -9,7 +9,7 @@ namespace deft {
 namespace {
 
 // Speculative staging (see the head of this file).  The cut a call leaves for the next one is the
-// first-level bucket of the (k + max(k / 2, kSpecSlack))-th largest key: a margin in rank, so that it
+// position of the (k + max(k / 4, kSpecSlack))-th largest key: a margin in rank, so that it
 // adapts to the tail of the layer's distribution and to k (the k-th largest of a handful moves
 // by several buckets from draw to draw, the k-th of a million hardly at all).
 constexpr uint32_t kSpecSlack = 48;
@@ -672,71 +672,82 @@ __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
 // The rank whose key the remembered bucket belongs to: some way below the k-th largest, so that the
 // cut holds when the distribution moves a little (the k-th largest of a handful moves by several
 // buckets from draw to draw, the k-th of a million hardly at all).
-__device__ __forceinline__ uint32_t safe_rank(uint32_t k) { return k + (k / 2 > kSpecSlack ? k / 2 : kSpecSlack); }
+__device__ __forceinline__ uint32_t safe_rank(uint32_t k) { return k + (k / 4 > kSpecSlack ? k / 4 : kSpecSlack); }
 
 // ---- the speculative cut of a layer, from what the previous call on the workspace left behind ----
-// Remembered per layer: the first-level bucket in which the previous call found the key of rank
-// safe_rank(k), that call's norm and rank, and how well the predictions have been doing: a running mean
-// of (bucket found - bucket predicted) and a running mean of that error's absolute deviation, both in
-// 1/16 bucket (the scheme TCP uses for its retransmission timer).
+// Remembered per layer: where the previous call found the key of rank safe_rank(k), as a position on the
+// magnitude-key axis in units of 1/16 first-level bucket (= 1/256 octave: key >> 15), that call's norm
+// and rank, and how well the predictions have been doing: a running mean of (position found - position
+// predicted) and a running mean of that error's absolute deviation, in the same unit (the scheme TCP
+// uses for its retransmission timer).
 //
-// Prediction for this call: the remembered bucket, moved by the change of the layer's norm (16 buckets
+// Prediction for this call: the remembered position, moved by the change of the layer's norm (256 units
 // per octave) and down by three buckets per doubling of the rank asked for (steeper than the tail of a
-// Gaussian or Laplace distribution at these ranks).  The cut is placed below the prediction by the mean
-// error and twice the deviation (whole buckets, rounded towards zero): a stream whose thresholds drift against the norms, or jump
-// around, gets lower cuts (more staged entries) instead of failed ones; a steady stream gets tight ones.
-constexpr int kErrUnit = 16;          // error bookkeeping in 1/16 bucket
-constexpr int kDevInit = kErrUnit / 2, kDevMin = kErrUnit / 4, kDevMax = kErrUnit, kBiasMax = 24 * kErrUnit;
+// Gaussian or Laplace distribution at these ranks).  The cut is the bucket boundary at or below the
+// prediction plus the mean error minus twice the deviation: a stream whose thresholds drift against
+// the norms, or jump around, gets lower cuts (more staged entries) instead of failed ones; a steady
+// stream gets tight ones.
+constexpr int kErrUnit = 16;          // positions and errors in 1/16 bucket
+constexpr int kFinePosShift = kShift1 - 4;   // key >> kFinePosShift = position
+constexpr int kDevInit = kErrUnit / 2, kDevMin = kErrUnit / 8, kDevMax = 2 * kErrUnit, kBiasMax = 24 * kErrUnit;
+static_assert(kErrUnit == 16, "positions are key >> (kShift1 - 4)");
 
-// The predicted bucket (not clamped), or INT_MIN if nothing usable is remembered.
-__device__ __forceinline__ int predict_bucket(const uint4& raw, uint32_t k, double norm) {
-    const uint32_t bucket_p1 = raw.x, rank = raw.z;
-    if (bucket_p1 == 0 || bucket_p1 > (uint32_t)kBins1) return INT_MIN;
-    int pb = (int)bucket_p1 - 1;
+// The predicted position (not clamped), or INT_MIN if nothing usable is remembered.
+__device__ __forceinline__ int predict_pos(const uint4& raw, uint32_t k, double norm) {
+    const uint32_t pos_p1 = raw.x, rank = raw.z;
+    if (pos_p1 == 0 || pos_p1 > (uint32_t)kBins1 * kErrUnit) return INT_MIN;
+    int pf = (int)pos_p1 - 1;
     const float was = __uint_as_float(raw.y), now = (float)norm;
-    if (was > 0.0f && now > 0.0f && was < 3.0e38f && now < 3.0e38f) pb += (int)floorf(16.0f * log2f(now / was));
+    if (was > 0.0f && now > 0.0f && was < 3.0e38f && now < 3.0e38f) pf += (int)floorf(16.0f * kErrUnit * log2f(now / was));
     const uint32_t want = safe_rank(k);
-    if (rank > 0 && want > rank) pb -= (int)ceilf(3.0f * log2f((float)want / (float)rank));
-    return pb;
+    if (rank > 0 && want > rank) pf -= (int)ceilf(3.0f * kErrUnit * log2f((float)want / (float)rank));
+    return pf;
 }
 __device__ __forceinline__ int hint_bias(uint32_t w) { const int b = (int)(int16_t)(w & 0xffffu); return b < -kBiasMax ? -kBiasMax : (b > kBiasMax ? kBiasMax : b); }
 __device__ __forceinline__ int hint_dev(uint32_t w) { const int d = (int)(w >> 16); return d < kDevMin ? kDevInit : (d > kDevMax ? kDevMax : d); }
 
-// Staging threshold (a first-level bucket boundary) for a layer that is to select k of `size` entries and
-// has norm `norm` now; 0xffffffff = none (nothing remembered, or a layer too dense to speculate on).
-__device__ __forceinline__ uint32_t predict_cut(const LayerHint* hp, int64_t k, int64_t size, double norm) {
+// Staging threshold for a layer that is to select k of `size` entries and has norm `norm` now, a
+// multiple of `align` positions (kErrUnit: a first-level bucket boundary, which the five-step kernel
+// needs; the single-pass kernel takes a quarter of that); 0xffffffff = none (nothing remembered, or a
+// layer too dense to speculate on).
+__device__ __forceinline__ uint32_t predict_cut(const LayerHint* hp, int64_t k, int64_t size, double norm, int align) {
     if (k * kSpecDensity > size) return 0xffffffffu;
     const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(hp));
-    int pb = predict_bucket(raw, (uint32_t)k, norm);
-    if (pb == INT_MIN) return 0xffffffffu;
-    const int adj = hint_bias(raw.w) - 2 * hint_dev(raw.w);
-    pb += adj / kErrUnit;   // towards zero: a steady stream (deviation well under a bucket) cuts at the prediction
-    pb = pb < 0 ? 0 : (pb > kBins1 - 1 ? kBins1 - 1 : pb);
-    return (uint32_t)pb << kShift1;
+    const int pf = predict_pos(raw, (uint32_t)k, norm);
+    if (pf == INT_MIN) return 0xffffffffu;
+    const int at = pf + hint_bias(raw.w) - 2 * hint_dev(raw.w);
+    int pa = at >= 0 ? at / align : 0;   // rounded down to the boundary
+    const int top = (kBins1 - 1) * kErrUnit / align;
+    pa = pa > top ? top : pa;
+    return (uint32_t)(pa * align) << kFinePosShift;
 }
 
-// After a layer's selection: remembers `bucket` (the first-level bucket of the key of rank safe_rank(k) if
-// `exact`, else an upper bound of it: the bucket below the cut, when fewer than safe_rank(k) entries were
-// at or above the cut) and folds the prediction's error into the running means.  One thread.
-__device__ __forceinline__ void hint_update(LayerHint* hp, uint32_t bucket, bool exact, uint32_t k, double norm) {
+// After a layer's selection: remembers `pos` (where the key of rank safe_rank(k) was found if `exact`, else an
+// upper bound of it: just below the cut, when fewer than safe_rank(k) entries were at or above the cut)
+// and folds the prediction's error into the running means.  `slack`: half the width of the interval the
+// position is known to lie in (0 for the single-pass kernel's fine bins, half a bucket for a first-level
+// bucket), which is not counted as deviation.  One thread.
+__device__ __forceinline__ void hint_update(LayerHint* hp, uint32_t pos, bool exact, int slack, uint32_t k, double norm) {
     const uint4 raw = *reinterpret_cast<const uint4*>(hp);
-    const int pb = predict_bucket(raw, k, norm);
+    const int pf = predict_pos(raw, k, norm);
     int bias = hint_bias(raw.w), dev = hint_dev(raw.w);
-    if (pb != INT_MIN) {
-        int err = ((int)bucket - pb) * kErrUnit;
-        if (!exact) err -= kErrUnit;   // the truth lies at or below the bound
+    if (pf != INT_MIN) {
+        int err = (int)pos - pf;
+        if (!exact) err -= kErrUnit / 2;   // the truth lies at or below the bound
         err = err < -kBiasMax ? -kBiasMax : (err > kBiasMax ? kBiasMax : err);
         const int d = err - bias;
+        int ad = (d < 0 ? -d : d) - slack;
+        ad = ad < 0 ? 0 : ad;
         bias += d / 4;
-        dev += ((d < 0 ? -d : d) - dev) / 4;
-        if (d < -2 * dev - kErrUnit) dev += kErrUnit / 2;   // the found bucket lies well below what the cut allowed for: back off at once
+        dev += (ad - dev) / 4;
+        if (d < -2 * dev - kErrUnit) dev += kErrUnit / 2;   // found well below what the cut allowed for: back off at once
         dev = dev < kDevMin ? kDevMin : (dev > kDevMax ? kDevMax : dev);
     } else {
         bias = 0;
         dev = kDevInit;
     }
     uint4 out;
-    out.x = bucket + 1u;
+    out.x = pos + 1u;
     out.y = __float_as_uint((float)norm);
     out.z = safe_rank(k);
     out.w = ((uint32_t)dev << 16) | ((uint32_t)bias & 0xffffu);
@@ -745,9 +756,9 @@ __device__ __forceinline__ void hint_update(LayerHint* hp, uint32_t bucket, bool
 
 // Fills the table of the CTA's streamed layers; returns how many there are (at most
 // kMaxLocalLayers: checked on the host).
-// spec_on: layers get a speculative cut from what the previous call left behind.
+// spec_on: layers get a speculative cut (a multiple of cut_align positions) from what the previous call left behind.
 __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRange& r, LayerTable* lt,
-                                                 uint32_t* scratch, bool spec_on) {
+                                                 uint32_t* scratch, bool spec_on, int cut_align) {
     int nl = 0;
     // scratch[kMTried - kMScratch] is the CTA's "speculated" flag (same misc area)
     if (threadIdx.x == 0) scratch[kMTried - kMScratch] = 0u;
@@ -773,7 +784,7 @@ __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRa
                 sthr = p.thr_key + 1u;                       // key >= thr_key + 1  <=>  key > thr_key
             } else if (spec_on) {
                 sthr = predict_cut(p.hint + p.desc[j].layer_id, p.desc[j].k, p.desc[j].end - p.desc[j].start,
-                                   p.desc[j].norm);
+                                   p.desc[j].norm, cut_align);
                 if (sthr != 0xffffffffu) scratch[kMTried - kMScratch] = 1u;
             }
             lt->sthr[c] = sthr;

@@ -144,10 +144,11 @@ __device__ __noinline__ void step_read1(const SelParams& p, const CtaRange r, La
                     // histogram reaches that far down, else from the bucket below this call's cut
                     const double norm = p.desc[lt->j[cl]].norm;
                     if (!spec || total >= k_safe) {
-                        hint_update(p.hint + lid, misc[kMOut3 + 2], true, kk, norm);
+                        // (known to the bucket: its middle, half a bucket of slack)
+                        hint_update(p.hint + lid, misc[kMOut3 + 2] * kErrUnit + kErrUnit / 2, true, kErrUnit / 2, kk, norm);
                     } else {
-                        const uint32_t cutb = lt->sthr[cl] >> kShift1;
-                        hint_update(p.hint + lid, cutb > 0u ? cutb - 1u : 0u, false, kk, norm);
+                        const uint32_t cutp = (lt->sthr[cl] >> kShift1) * kErrUnit;
+                        hint_update(p.hint + lid, cutp > 0u ? cutp - 1u : 0u, false, 0, kk, norm);
                     }
                 }
             }
@@ -466,7 +467,7 @@ __device__ __forceinline__ void five_steps(const SelParams& p, unsigned char* sm
         r = weighted_range(p, reinterpret_cast<uint32_t*>(smem + kSmMain), reinterpret_cast<int*>(smem + kSmTf),
                            misc + kMScratch);
     const int nl = build_layer_table(p, r, lt, misc + kMScratch,
-                                     !p.fixed_thr && !p.from_retry);
+                                     !p.fixed_thr && !p.from_retry, kErrUnit);
     Stage st;
     st.res = reinterpret_cast<uint2*>(smem + kSmRes);
     st.spill = spill_base(p, r);

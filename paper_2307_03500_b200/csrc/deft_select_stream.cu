@@ -64,16 +64,16 @@ __device__ __noinline__ void push_retry(const SelParams& p, int j) {
 // unrolling, the layer's entries and its tile table fetched together.
 //
 // Which staged entries are selected is settled in two steps.  A histogram with bins of 2^kFineShift
-// keys counted from the cut (1/256 octave; the first-level buckets are 1/16, and the staged keys crowd
+// keys counted from the cut (1/4096 octave over one octave; the first-level buckets are 1/16, and the staged keys crowd
 // into the few buckets right above the cut) gives the bin `a` of the k-th largest key: everything in a
 // higher bin is selected, nothing in a lower one.  The few entries of bin a (the candidates) are ranked
 // among themselves by (key descending, index ascending); the first k - (entries above bin a) of them
 // are selected and get a flag in their entry.  No threshold key is ever needed.
-constexpr int kFineShift = 15;
+constexpr int kFineShift = 11;
 constexpr int kFineBins = kBins1;   // the top bin takes everything beyond
 constexpr uint32_t kCandMax = 1024; // candidates that can be ranked; a layer with more goes to the retry list
 constexpr uint32_t kSelFlag = 0x80000000u;   // in an entry's .y: a candidate that is selected
-static_assert(kCandMax * 12 <= kSmAuxBytes && kShift1 > kFineShift && kSelWarps == 16 &&
+static_assert(kCandMax * 12 <= kSmAuxBytes && kFineShift <= kFinePosShift && kSelWarps == 16 &&
               DEFT_MAX_LAYER_ELEMS / kTile < (1 << 20),
               "candidates live in the aux region; bit 31 of .y is free; a warp id fits four bits");
 
@@ -135,7 +135,7 @@ struct Lap {
 
 // One layer, finished by the CTA that completed its last tile.  c: local layer; S: entries staged for
 // the layer by all CTAs; flooded: some CTA stopped staging.
-__device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, int c, uint32_t S, uint32_t flooded,
+__device__ __noinline__ bool finish_layer(const SelParams& p, LayerTable* lt, int c, uint32_t S, uint32_t flooded,
                                           TileTable* tt, unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint32_t* scratch = misc + kMScratch;
@@ -154,7 +154,7 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
             atomicAdd(p.spec_ctl + 5, 1u);
             push_retry(p, lt->j[c]);
         }
-        return;
+        return false;
     }
     Staged f;
     f.S = S;
@@ -166,8 +166,11 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
     // the entries and (the first pass of) the tile table are fetched together
     {
         const uint32_t nres = S < kStreamRes ? S : kStreamRes;
-#pragma unroll 4
-        for (uint32_t pos = tid; pos < nres; pos += kSelThreads) f.res[pos] = f.src[pos];
+        // (two entries per load: regions start on 128-byte boundaries and have slack behind them)
+        const uint4* src2 = reinterpret_cast<const uint4*>(f.src);
+        uint4* res2 = reinterpret_cast<uint4*>(f.res);
+#pragma unroll 8
+        for (uint32_t pos = tid; pos < (nres + 1u) / 2u; pos += kSelThreads) res2[pos] = src2[pos];
 #pragma unroll 4
         for (int t = tid; t < np0; t += kSelThreads) tt->first[t] = __ldcg(tab + t).x;
     }
@@ -189,40 +192,41 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
             atomicAdd(p.spec_ctl + 5, 1u);
             push_retry(p, lt->j[c]);
         }
-        return;
+        return false;
     }
     if (tid == kSelThreads - 1) {   // (not thread 0: the loads it waits for are off the CTA's critical path this way)
         // what the next call starts from: the first-level bucket of the k_safe-th key if that many were
         // staged, else the bucket below this call's cut
         const double norm = p.desc[lt->j[c]].norm;
         if (S >= k_safe) {
-            hint_update(hp, (cut + (a_safe << kFineShift)) >> kShift1, true, k, norm);
+            hint_update(hp, (cut >> kFinePosShift) + (a_safe >> (kFinePosShift - kFineShift)), true, 0, k, norm);
         } else {
-            const uint32_t cutb = cut >> kShift1;
-            hint_update(hp, cutb > 0u ? cutb - 1u : 0u, false, k, norm);
+            const uint32_t cutp = cut >> kFinePosShift;
+            hint_update(hp, cutp > 0u ? cutp - 1u : 0u, false, 0, k, norm);
         }
         atomicAdd(p.spec_ctl + 4, 1u);
     }
-    // the candidates: (key, index order, where the entry lives); the histogram's room is free now
-    uint32_t* ckey = h;
-    uint32_t* cy = h + kCandMax;
+    // the candidates: (key, index order) as one 64-bit word that sorts the way the selection wants
+    // (larger key first, then lower index: .y grows with the index and bit 31 of it is free), and
+    // where the entry lives; the histogram's room is free now
+    unsigned long long* cword = reinterpret_cast<unsigned long long*>(h);
     uint32_t* cpos = h + 2 * kCandMax;
     for_each_entry(f, [&](const uint2 ent, uint32_t pos) {
         if (fine_bin(key_of(ent.x), cut) == a) {
             const uint32_t i = atomicAdd(misc + kMFlag, 1u);
-            ckey[i] = key_of(ent.x);
-            cy[i] = ent.y;
+            cword[i] = ((unsigned long long)key_of(ent.x) << 32) | (0x7fffffffu - ent.y);
             cpos[i] = pos;
         }
     });
     __syncthreads();
     for (uint32_t i = tid; i < C; i += kSelThreads) {
-        const uint32_t key = ckey[i], y = cy[i];
+        const unsigned long long mine = cword[i];
         uint32_t before = 0;
-        for (uint32_t j = 0; j < C; ++j) before += (ckey[j] > key) || (ckey[j] == key && cy[j] < y);
+#pragma unroll 8
+        for (uint32_t j = 0; j < C; ++j) before += cword[j] > mine ? 1u : 0u;
         if (before < krem) {
             const uint32_t pos = cpos[i];
-            if (pos < kStreamRes) f.res[pos].y = y | kSelFlag; else f.src[pos].y = y | kSelFlag;
+            if (pos < kStreamRes) f.res[pos].y |= kSelFlag; else f.src[pos].y |= kSelFlag;
         }
     }
     __syncthreads();
@@ -238,14 +242,22 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
     // Up to kMaxLocalTiles tiles of the layer per round.
     float* const val = p.val;
     int64_t* const idx = p.idx;
-    float* const acc_rw = p.acc_rw;
     const int64_t cap = p.out_cap;
     const int64_t tile0 = lt->start[c] / kTile;
     const int64_t out_off = lt->out_off[c];
-    uint32_t* wtot = misc + kMWarpCnt;   // per warp: selected entries of its range, then their exclusive prefix
-    const uint32_t per_warp = ((S + kSelWarps - 1) / kSelWarps + 127u) & ~127u;
-    const uint32_t w_lo = (uint32_t)warp * per_warp < S ? (uint32_t)warp * per_warp : S;
-    const uint32_t w_hi = w_lo + per_warp < S ? w_lo + per_warp : S;
+    // Each warp walks two ranges: its share of the entries held in shared memory, then its share of
+    // those left in the region (reading those costs a round trip to L2 per batch: they are spread over
+    // all warps instead of falling to the last few).  2 * kSelWarps ranges in region order.
+    uint32_t* wtot = misc + kMWarpCnt;   // per range: selected entries, then their exclusive prefix
+    const uint32_t n_sm = S < kStreamRes ? S : kStreamRes;
+    uint32_t w_lo_[2], w_hi_[2];
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+        const uint32_t p0 = part ? n_sm : 0u, p1 = part ? S : n_sm;
+        const uint32_t per = ((p1 - p0 + kSelWarps - 1) / kSelWarps + 127u) & ~127u;
+        w_lo_[part] = p0 + (uint32_t)warp * per < p1 ? p0 + (uint32_t)warp * per : p1;
+        w_hi_[part] = w_lo_[part] + per < p1 ? w_lo_[part] + per : p1;
+    }
     uint32_t base = 0;
     for (int tp = 0; tp < tn; tp += kMaxLocalTiles) {
         const int np = tn - tp < kMaxLocalTiles ? tn - tp : kMaxLocalTiles;
@@ -256,8 +268,11 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
         for (int t = tid; t < np; t += kSelThreads) tt->ge[t] = 0u;
         __syncthreads();
         // pass 1
+        for (int part = 0; part < 2; ++part) {
+        const uint32_t w_hi = part ? w_hi_[1] : w_hi_[0];
+        const uint32_t vw = (uint32_t)(part * kSelWarps + warp);
         uint32_t run = 0;
-        for (uint32_t p4 = w_lo; p4 < w_hi; p4 += 128) {   // four steps' entries are fetched together
+        for (uint32_t p4 = part ? w_lo_[1] : w_lo_[0]; p4 < w_hi; p4 += 128) {   // four steps' entries are fetched together
             uint2 e4[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -273,16 +288,27 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
                 const bool here = valid && t < (uint32_t)np;
                 const bool sel = here && ((fine_bin(key_of(ent.x), cut) > a) || (ent.y & kSelFlag));
                 const unsigned ball = __ballot_sync(0xffffffffu, sel);
-                if (here && tt->first[t] == pos) tt->first[t] = 0x80000000u | ((uint32_t)warp << 27) | (run + __popc(ball & ((1u << lane) - 1u)));
-                if (sel) atomicAdd(&tt->ge[t], 1u);
+                if (here && tt->first[t] == pos) tt->first[t] = 0x80000000u | (vw << 26) | (run + __popc(ball & ((1u << lane) - 1u)));
+                // a tile's entries are neighbours: the first lane of every run of equal tiles adds the run's count
+                const uint32_t tkey = here ? t : 0xffffffffu;
+                const uint32_t tprev = __shfl_up_sync(0xffffffffu, tkey, 1);
+                const bool starts = lane == 0 || tkey != tprev;
+                const unsigned sb = __ballot_sync(0xffffffffu, starts);
+                if (starts && here) {
+                    const unsigned above = sb & ~((2u << lane) - 1u);   // (2u << 31 == 0: nothing above lane 31)
+                    const unsigned upto = above ? ((1u << (__ffs((int)above) - 1)) - 1u) : 0xffffffffu;
+                    const uint32_t cnt = __popc(ball & upto & ~((1u << lane) - 1u));
+                    if (cnt) atomicAdd(&tt->ge[t], cnt);
+                }
                 run += __popc(ball);
             }
         }
-        if (lane == 0) wtot[warp] = run;
+        if (lane == 0) wtot[vw] = run;
+        }
         __syncthreads();
         lap.lap(24);
         if (warp == 0) {
-            const uint32_t x = lane < kSelWarps ? wtot[lane] : 0u;
+            const uint32_t x = wtot[lane];
             wtot[lane] = warp_incl_scan(x, lane) - x;
         }
         // exclusive prefix of the tiles' counts: each thread a run of consecutive tiles
@@ -300,8 +326,10 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
         __syncthreads();
         lap.lap(25);
         // pass 2
-        run = wtot[warp];
-        for (uint32_t p4 = w_lo; p4 < w_hi; p4 += 128) {
+        for (int part = 0; part < 2; ++part) {
+        const uint32_t w_hi = part ? w_hi_[1] : w_hi_[0];
+        uint32_t run = wtot[part * kSelWarps + warp];
+        for (uint32_t p4 = part ? w_lo_[1] : w_lo_[0]; p4 < w_hi; p4 += 128) {
             uint2 e4[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -319,23 +347,24 @@ __device__ __noinline__ void finish_layer(const SelParams& p, LayerTable* lt, in
             const unsigned ball = __ballot_sync(0xffffffffu, sel);
             if (sel) {
                 const uint32_t mark = tt->first[t];   // where the tile's first entry stood: warp, running count
-                const uint32_t at_first = wtot[(mark >> 27) & 15u] + (mark & 0x7ffffffu);
+                const uint32_t at_first = wtot[(mark >> 26) & 31u] + (mark & 0x3ffffffu);
                 const int64_t o = out_off + tt->ge[t] + (run + __popc(ball & ((1u << lane) - 1u)) - at_first);
                 const int64_t elem = (tile0 + tp + t) * kTile + (int64_t)y_off(ent.y);
                 if (o < cap) {
                     val[o] = __uint_as_float(ent.x);
                     idx[o] = elem;
                 }
-                if (acc_rw) acc_rw[elem] = 0.0f;
             }
             run += __popc(ball);
             }
+        }
         }
         base += total;
         __syncthreads();   // the tables are rewritten by the next round
         lap.lap(26);
     }
     if (p.timing && tid == 0) atomicAdd(p.timing + 28, 1ull);
+    return true;
 }
 
 // Out of line: the rare path must not cost the kernel's main loop registers.
@@ -373,7 +402,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     r.il = 0; r.q0tab = nullptr; r.nsuper = 0;
     r.q0 = 0; r.q1 = p.tiles; r.nloc = 0;
     r.jA = 0; r.jB = p.n_my - 1;
-    const int nl = build_layer_table(p, r, lt, misc + kMScratch, true);   // every streamed layer of the call
+    const int nl = build_layer_table(p, r, lt, misc + kMScratch, true, kErrUnit / 4);   // every streamed layer of the call
     const int nstripe = (p.tiles + kStripe - 1) / kStripe;
     const int nloc = (b < nstripe ? (nstripe - b + G - 1) / G : 0) * kStripe;
     if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMTileCtr] = 0; misc[kMBudget] = 4096u; }
@@ -474,7 +503,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     stamp(p, 2);
 
     // ---- small layers, handed out one at a time (the counter is cleared with the plan upload) ----
-    {
+    // With streamed layers in the call they wait until the CTA has nothing left to finish: most CTAs
+    // have time on their hands then, while the largest layers are still being finished.
+    auto small_layers = [&]() {
         uint32_t* next = &p.state[p.desc[0].layer_id].pad[0];
         for (;;) {
             __syncthreads();
@@ -484,25 +515,77 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
             if (j >= p.n_my) break;
             if (is_direct(p, j)) resolve_direct(p, j, smem);   // uniform over the CTA
         }
+    };
+    if (!has_streamed) {   // uniform over the grid: small layers only
+        small_layers();
+        return;
     }
-    stamp(p, 6);
-    if (!has_streamed) return;   // uniform over the grid: small layers only
 
     // ---- every layer's entries are in its region: the layers are finished one per CTA, round-robin ----
     __threadfence();
     grid.sync();
-    for (int c = b; c < nl; c += G) {
-        if (lt->sthr[c] == 0xffffffffu) continue;
-        const uint32_t S = __ldcg(&p.state[lt->lid[c]].cursor);
-        const uint32_t flooded = __ldcg(&p.state[lt->lid[c]].spec_bad);
-        finish_layer(p, lt, c, S, flooded, tt, smem);
-        __syncthreads();
+    // largest first (a layer's cost grows with what was staged for it): the order is worked out by
+    // every CTA for itself; CTA b starts with the b-th largest, the rest are taken from a counter
+    // (cleared with the plan upload) as CTAs become free
+    for (int c = threadIdx.x; c < nl; c += kSelThreads)
+        lt->v0[c] = lt->sthr[c] == 0xffffffffu ? 0u : __ldcg(&p.state[lt->lid[c]].cursor);
+    __syncthreads();
+    for (int c = threadIdx.x; c < nl; c += kSelThreads) {
+        const uint32_t s = lt->v0[c];
+        int before = 0;
+        for (int o = 0; o < nl; ++o) {
+            const uint32_t so = lt->v0[o];
+            before += (so > s || (so == s && o < c)) ? 1 : 0;
+        }
+        lt->v1[before] = (uint32_t)c;
+    }
+    __syncthreads();
+    {
+        uint32_t* next = &p.state[p.desc[0].layer_id].pad[1];
+        int slot = b;
+        while (slot < nl) {
+            const int c = (int)lt->v1[slot];
+            bool done = false;
+            if (lt->sthr[c] != 0xffffffffu) {
+                const uint32_t flooded = __ldcg(&p.state[lt->lid[c]].spec_bad);
+                done = finish_layer(p, lt, c, lt->v0[c], flooded, tt, smem);
+            }
+            if (!done && p.acc_rw) {
+                // the layer is on the retry list: its part of the index output must not be mistaken for
+                // selected entries by the pass that clears them
+                const int64_t o0 = lt->out_off[c];
+                for (int64_t i = threadIdx.x; i < (int64_t)lt->k[c]; i += kSelThreads)
+                    if (o0 + i < p.out_cap) p.idx[o0 + i] = -1;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) misc[kMTileCtr] = (uint32_t)G + atomicAdd(next, 1u);
+            __syncthreads();
+            slot = (int)misc[kMTileCtr];
+        }
     }
     stamp(p, 5);
+    small_layers();
+    stamp(p, 6);
 
     // ---- what is left over: the five steps on the retry list, by the whole grid ----
     __threadfence();
     grid.sync();
+    // The selected entries are cleared in the accumulator by the whole grid (one SM gets through about
+    // one scattered 4-byte store per clock: a large layer's would hold its finishing CTA up for
+    // microseconds).  Small layers and the retry list clear their own.
+    if (p.acc_rw) {
+        const int64_t n_out = p.out_total < p.out_cap ? p.out_total : p.out_cap;
+        const int64_t step = (int64_t)G * kSelThreads;
+        for (int64_t i0 = (int64_t)b * kSelThreads + threadIdx.x; i0 < n_out; i0 += 4 * step) {
+            int64_t at[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) at[u] = i0 + u * step < n_out ? __ldcg(p.idx + i0 + u * step) : -1;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (at[u] >= 0) p.acc_rw[at[u]] = 0.0f;
+        }
+    }
+    stamp(p, 3);
     const unsigned long long packed = __ldcg(&p.retry->packed);
     if ((packed >> 32) == 0ull) return;   // uniform over the grid
     __syncthreads();

@@ -86,6 +86,16 @@ DEFT_API int32_t deft_last_cuda_error(void);
 DEFT_API void deft_debug_select_kernel(int32_t single_pass);
 
 /*
+ * Diagnostic: how the single-pass kernel reads the vector.  on != 0 (the default): whole tiles come
+ * through a ring of sixteen 8 KB stages in shared memory filled by bulk copies (cp.async.bulk, one
+ * mbarrier per stage), which keeps 128 KB per SM in flight whatever the warps are busy with; the ring
+ * takes its room from the shared-memory staging area.  on = 0: every warp loads its tile into
+ * registers with sixteen 16-byte loads per lane and waits for them.  Results never differ.  Not
+ * thread-safe; for measurements and tests.
+ */
+DEFT_API void deft_debug_select_ring(int32_t on);
+
+/*
  * Diagnostic: when timing_d (DEVICE, 1024 x uint64, zeroed by the caller) is not NULL every
  * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs) and counters.
  * Both kernels: [0] kernel start, [14] / [15] staged entries (max over CTAs or layers / total).
@@ -207,7 +217,8 @@ DEFT_API deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_
  * Diagnostic counters of the single-pass selection kernel, summed over every call on this workspace
  * since deft_workspace_init: stats_h[0] layers it finished in one read, [1] layers whose remembered
  * cut failed (too few or far too many entries staged), [2] layers it had no usable cut for (nothing
- * remembered yet, or too dense); [1] and [2] were handed to the five-step kernel.  [3] is reserved.
+ * remembered yet, or too dense); [1] and [2] were handed to the five-step kernel; [3] waits on the
+ * bulk-copy ring that gave up (always 0 on a healthy device; see deft_debug_select_ring).
  * stats_h: HOST, 4 x uint64.  Waits for `stream`.  Errors: INVALID_ARG, CAPACITY, CUDA.
  */
 DEFT_API deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layers, uint64_t* stats_h,

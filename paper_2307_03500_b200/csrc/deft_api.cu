@@ -12,6 +12,7 @@ namespace deft {
 static thread_local int32_t g_last_cuda_error = 0;
 static unsigned long long* g_select_timing = nullptr;
 static int g_stream_kernel = -1;   // deft_debug_select_kernel: -1 by size, 0 never, 1 whenever possible
+static int g_stream_ring = 1;      // deft_debug_select_ring: the single-pass kernel reads through a ring of bulk copies
 
 // Limits of the single-pass selection kernel (see select_rank).
 constexpr int64_t kStreamMaxK = 65536;              // entries one layer may select
@@ -261,7 +262,7 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
         int n_streamed = 0;
         // every CTA keeps a table of all streamed layers and a map of all layers; its stripes are tiles / grid tiles
         bool ok = R.elems <= kStreamMaxElems && R.n_my <= kStreamMaxLayers &&
-                  (int64_t)R.tiles / p.grid + 2 * kSuper <= kMaxLocalTiles;
+                  (int64_t)R.tiles / p.grid + 2 * kSuper <= kStreamLocalTiles;
         for (int j = 0; j < R.n_my && ok; ++j) {
             const int64_t size = hd[j].end - hd[j].start;
             if (size <= kDirectElems) continue;
@@ -273,7 +274,7 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
             }
         }
         if (ok && (streamed == 0 || 2 * sparse >= streamed)) {
-            return launch_select_stream(p, streamed != 0, stream);
+            return launch_select_stream(p, streamed != 0, g_stream_ring != 0, stream);
         }
     }
     if (R.n_my > 1 && R.n_my <= kMaxWeightedLayers && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) {
@@ -331,6 +332,7 @@ void deft_debug_select_timing(void* timing_d) { g_select_timing = static_cast<un
 
 int64_t deft_select_launch_max_elems(void) { return (int64_t)sm_count() * kMaxLocalTiles * kTile; }
 
+void deft_debug_select_ring(int32_t on) { g_stream_ring = on != 0 ? 1 : 0; }
 void deft_debug_select_kernel(int32_t single_pass) { g_stream_kernel = single_pass < 0 ? -1 : (single_pass != 0 ? 1 : 0); }
 
 deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_layers, void* stream) {
@@ -346,14 +348,14 @@ deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layer
     if (!ws_d || !stats_h || n_layers < 1) return DEFT_ERR_INVALID_ARG;
     const WsLayout w = ws_layout(1, n_layers, 1);
     if (w.hint + 256 > ws_bytes) return DEFT_ERR_CAPACITY;
-    uint32_t words[8];
+    uint32_t words[9];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DEFT_CUDA_TRY(cudaMemcpyAsync(words, static_cast<const char*>(ws_d) + w.hint, sizeof(words), cudaMemcpyDeviceToHost, st));
     DEFT_CUDA_TRY(cudaStreamSynchronize(st));
     stats_h[0] = words[4];
     stats_h[1] = words[5];
     stats_h[2] = words[6];
-    stats_h[3] = words[7];
+    stats_h[3] = words[8];
     return DEFT_OK;
 }
 

@@ -36,6 +36,7 @@ constexpr int kDirectElems = 16384;
 constexpr int kResident = 8192;
 // Limits of one CTA's share of a rank (checked on the host before launch).
 constexpr int kMaxLocalTiles = 4096;    // tiles per CTA
+constexpr int kStreamLocalTiles = 2048;  // tiles per CTA in the single-pass kernel (its read keeps a smaller tile table)
 constexpr int kMaxLocalLayers = 256;    // streamed layers per CTA
 // A rank that is one layer of at least kInterleaveTiles tiles per CTA is split over the CTAs in
 // super-tiles of kSuper tiles dealt out round-robin instead of one contiguous run per CTA.
@@ -280,7 +281,7 @@ deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t 
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
                                double* partial_d, cudaStream_t stream, double* norms_host_mapped = nullptr);
 deft_status launch_select(const SelParams& p, cudaStream_t stream);
-deft_status launch_select_stream(const SelParams& p, bool has_streamed, cudaStream_t stream);
+deft_status launch_select_stream(const SelParams& p, bool has_streamed, bool ring, cudaStream_t stream);
 deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t count,
                                    cudaStream_t stream);
 deft_status launch_gather_update(float* acc_d, const int64_t* idx_d, int64_t count, float* val_d,

@@ -415,32 +415,35 @@ __device__ __forceinline__ bool marks_single(uint32_t k0, uint32_t k1) {
     return !__any_sync(0xffffffffu, (m0 | m1) != 0u);
 }
 
-// Marked components of the tile when marks_single() holds.
+// Bit 4 * i of the result: load i of the lane (nibble i of k) has a mark.
+__device__ __forceinline__ uint32_t marked_loads(uint32_t k) { return (k | (k >> 1) | (k >> 2) | (k >> 3)) & 0x11111111u; }
+
+// Marked components of the tile when marks_single() holds (one per marked load).
 __device__ __forceinline__ uint32_t count_single(uint32_t k0, uint32_t k1) {
-    uint32_t n = 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i)
-        n += __popc(__ballot_sync(0xffffffffu, (((i < 8 ? k0 : k1) >> (4 * (i & 7))) & 0xfu) != 0u));
-    return n;
+    return __reduce_add_sync(0xffffffffu, (uint32_t)(__popc(marked_loads(k0)) + __popc(marked_loads(k1))));
 }
 
 // marks_single() holds: put(position, value bits, offset in tile) for every marked component; the tile's
-// entries take positions first, first + 1, ... in index order.
+// entries take positions first, first + 1, ... in index order.  Loads in which no lane has a mark (most
+// of them, when the cut is high) cost a test of a warp-wide mask and nothing else.
 template <typename Put>
 __device__ __forceinline__ void write_single(const TileRegs& t, uint32_t k0, uint32_t k1, uint32_t first, int lane,
                                              Put put) {
     const uint32_t below = (1u << lane) - 1u;
+    const uint32_t u0 = __reduce_or_sync(0xffffffffu, marked_loads(k0)), u1 = __reduce_or_sync(0xffffffffu, marked_loads(k1));
     uint32_t run = first;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-        const uint32_t nib = ((i < 8 ? k0 : k1) >> (4 * (i & 7))) & 0xfu;
-        const uint32_t bal = __ballot_sync(0xffffffffu, nib != 0u);
-        if (nib) {
-            const uint32_t c = (uint32_t)__ffs((int)nib) - 1u;
-            const uint32_t bits = pick4(t.v[i].x, t.v[i].y, t.v[i].z, t.v[i].w, (int)c);
-            put(run + (uint32_t)__popc(bal & below), bits, (uint32_t)((i * 32 + lane) * 4) + c);
+        if (((i < 8 ? u0 : u1) >> (4 * (i & 7))) & 1u) {   // uniform over the warp
+            const uint32_t nib = ((i < 8 ? k0 : k1) >> (4 * (i & 7))) & 0xfu;
+            const uint32_t bal = __ballot_sync(0xffffffffu, nib != 0u);
+            if (nib) {
+                const uint32_t c = (uint32_t)__ffs((int)nib) - 1u;
+                const uint32_t bits = pick4(t.v[i].x, t.v[i].y, t.v[i].z, t.v[i].w, (int)c);
+                put(run + (uint32_t)__popc(bal & below), bits, (uint32_t)((i * 32 + lane) * 4) + c);
+            }
+            run += (uint32_t)__popc(bal);
         }
-        run += (uint32_t)__popc(bal);
     }
 }
 

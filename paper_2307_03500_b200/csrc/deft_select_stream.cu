@@ -376,8 +376,66 @@ __device__ __noinline__ void retry_steps(const SelParams& q, unsigned char* smem
 // even sample of every layer of the call, so the layers whose entries crowd (large k_l / size_l) are
 // everybody's business, and so is the second look at a layer whose cut failed.
 constexpr int kStripe = 16;
-static_assert(kMaxLocalTiles % kStripe == 0 && kTfCache * 2 <= kSmSuperBytes, "stripes; the layer map lives in the super-tile area");
 
+// ---- the read through a ring of bulk copies (the kernel's second form) ----
+// Instead of every warp loading its tile into registers and waiting for it, the CTA keeps
+// kRingStages whole tiles in flight as bulk copies (cp.async.bulk, completion counted on an mbarrier
+// per stage) into a ring in shared memory.  Tiles are handed to the warps in ascending order from a
+// counter, so tile number n of the CTA always uses stage n % kRingStages; the warp that has taken
+// tile n out of its stage (into registers) starts the copy of tile n + kRingStages into it.  Only whole
+// tiles of layers with a cut go through the ring; for any other tile the stage's barrier just gets an
+// arrival, so that every use of a stage is one phase of its barrier.  A parity wait can only tell a
+// phase from its neighbour, so a warp first waits until its use of the stage has been started (a
+// sequence word per stage, written after the copy is issued) and only then for the phase to complete.
+// The ring takes its room from the shared-memory staging area, which keeps kRingRes entries during the read.
+constexpr int kRingStages = 16;
+constexpr uint32_t kTileBytes = kTile * 4;
+// During the read the kernel's tile table (StreamTiles) sits in the second half of the tile-table area;
+// the first half, the aux area and the main area are one stretch of shared memory for the staged entries and the ring.
+struct StreamTiles {                 // per local tile of the CTA, see TileTable
+    uint32_t first[kStreamLocalTiles];
+    uint32_t ge[kStreamLocalTiles];
+    uint16_t n[kStreamLocalTiles];
+};
+constexpr int kSmStreamTiles = kSmTile + kSmTileBytes - (int)sizeof(StreamTiles);
+constexpr uint32_t kRingRes = (uint32_t)(kSmStreamTiles - kSmMain - kRingStages * (int)kTileBytes) / 8;
+constexpr int kMRingBar = 164;    // misc words, two per stage: the stages' mbarriers
+constexpr int kMRingDead = 162;   // misc word: a wait on the ring gave up; the CTA reads with plain loads from then on
+constexpr int kMRingSeq = 200;    // misc words, one per stage: uses of the stage started so far
+static_assert(kSmAux == kSmMain + kSmMainBytes && kSmTile == kSmAux + kSmAuxBytes && kSmStreamTiles % 128 == 0 &&
+              kRingRes >= 4096 && (kRingRes * 8) % 128 == 0 && kMRingBar + 2 * kRingStages <= kMRingSeq && kMRingSeq + kRingStages <= 256 && kMRingBar % 2 == 0 &&
+              kMWarpCnt + 32 <= kMRingDead, "ring: room, alignment, misc words");
+
+__device__ __forceinline__ uint32_t smem_addr(const void* ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded: a copy that has not landed after this many polls (seconds) never will.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int i = 0; i < (1 << 22); ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+static_assert(kStreamLocalTiles % kStripe == 0 && kTfCache * 2 <= kSmSuperBytes, "stripes; the layer map lives in the super-tile area");
+
+template <bool kRing>
 __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParams p_in, const int has_streamed) {
     extern __shared__ __align__(16) unsigned char smem[];
     cg::grid_group grid = cg::this_grid();
@@ -388,7 +446,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
         p.timing[0] = t;
     }
     LayerTable* lt = reinterpret_cast<LayerTable*>(smem + kSmLayer);
-    TileTable* tt = reinterpret_cast<TileTable*>(smem + kSmTile);
+    TileTable* tt = reinterpret_cast<TileTable*>(smem + kSmTile);                  // the finishing CTA's
+    StreamTiles* rt = reinterpret_cast<StreamTiles*>(smem + kSmStreamTiles);       // the read's
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
     uint32_t* wbase = reinterpret_cast<uint32_t*>(smem + kSmWBase);
     uint2* res = reinterpret_cast<uint2*>(smem + kSmMain);
@@ -406,6 +465,33 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     const int nstripe = (p.tiles + kStripe - 1) / kStripe;
     const int nloc = (b < nstripe ? (nstripe - b + G - 1) / G : 0) * kStripe;
     if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMTileCtr] = 0; misc[kMBudget] = 4096u; }
+    constexpr uint32_t kReadRes = kRing ? kRingRes : kStreamRes;   // staged entries the CTA keeps in shared memory during the read
+    uint64_t* const bars = reinterpret_cast<uint64_t*>(misc + kMRingBar);
+    unsigned char* const ring = smem + kSmMain + kRingRes * 8;
+    if (kRing && threadIdx.x == 0) {
+        misc[kMRingDead] = 0u;
+        for (int sg = 0; sg < kRingStages; ++sg) { mbar_init(bars + sg, 1); misc[kMRingSeq + sg] = 0u; }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // Starts the use of its stage by local tile lq (one thread): the copy of a whole tile of a layer with a cut, else an arrival.
+    auto ring_issue = [&](int lq) {
+        const int q = kStripe * (b + (lq / kStripe) * G) + lq % kStripe;
+        const int sg = lq % kRingStages;
+        uint64_t* bar = bars + sg;
+        bool copied = false;
+        const uint32_t m = rt->first[lq];   // the tile's layer (filled in before the read starts)
+        if (m != 0xffffu) {
+            const TileSpan ts = tile_span(lt->start[m], lt->end[m], lt->tf[m], q);
+            if (ts.s == 0 && ts.e == kTile) {
+                mbar_expect_tx(bar, kTileBytes);
+                bulk_load(ring + (size_t)sg * kTileBytes, p.acc + ts.lo, kTileBytes, bar);
+                copied = true;
+            }
+        }
+        if (!copied) mbar_arrive(bar);
+        __threadfence_block();
+        *reinterpret_cast<volatile uint32_t*>(misc + kMRingSeq + sg) = (uint32_t)(lq / kRingStages) + 1u;
+    };
     __syncthreads();
     for (int c = threadIdx.x; c < nl; c += kSelThreads) {
         jmap[lt->j[c]] = (uint16_t)c;
@@ -430,23 +516,62 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     __syncthreads();
     stamp(p, 8);
     const uint32_t budget = misc[kMBudget] < 0x7fffffffu ? misc[kMBudget] : 0x7fffffffu;
+    // which layer (of those with a cut) every tile of the CTA belongs to: looked up once, here; the tile's
+    // slot in the table is rewritten when the tile has been read
+    for (int lq = threadIdx.x; lq < nloc; lq += kSelThreads) {
+        const int q = kStripe * (b + (lq / kStripe) * G) + lq % kStripe;
+        uint32_t m = 0xffffu;
+        if (q < p.tiles) {
+            m = jmap[layer_of_tile_sh(tfc, p.n_my, q)];
+            if (m != 0xffffu && lt->sthr[m] == 0xffffffffu) m = 0xffffu;
+        }
+        rt->first[lq] = m;
+    }
+    __syncthreads();
+    if (kRing && (int)threadIdx.x < kRingStages && (int)threadIdx.x < nloc) ring_issue((int)threadIdx.x);
 
     // ---- the read: every tile of the CTA once ----
     for (int lq = grab_tile(misc + kMTileCtr, lane); lq < nloc; lq = grab_tile(misc + kMTileCtr, lane)) {
         const int q = kStripe * (b + (lq / kStripe) * G) + lq % kStripe;
         uint32_t first = 0, n = 0, off = 0;
-        int cl = -1;
-        if (q < p.tiles) {
-            const uint32_t m = jmap[layer_of_tile_sh(tfc, p.n_my, q)];
-            if (m != 0xffffu && lt->sthr[m] != 0xffffffffu) cl = (int)m;
+        const uint32_t m = rt->first[lq];
+        const int cl = m != 0xffffu ? (int)m : -1;
+        TileSpan ts;
+        ts.lo = 0; ts.s = 0; ts.e = 0;
+        if (cl >= 0) ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
+        TileRegs t;
+        uint32_t vm[2], keep[2];
+        bool have = false;   // the tile is in registers already (it came through the ring)
+        if (kRing) {
+            const bool dead = *reinterpret_cast<volatile uint32_t*>(misc + kMRingDead) != 0u;
+            bool landed = false;
+            if (!dead) {
+                const uint32_t use = (uint32_t)(lq / kRingStages);
+                const volatile uint32_t* seq = misc + kMRingSeq + lq % kRingStages;
+                bool started = false;
+                for (int i = 0; i < (1 << 24) && !started; ++i) started = *seq > use;
+                landed = started && mbar_wait(bars + lq % kRingStages, use & 1u);
+            }
+            if (!dead && !landed) {   // never expected: remember it, and read the rest of the CTA's tiles the plain way
+                if (lane == 0) { misc[kMRingDead] = 1u; atomicAdd(p.spec_ctl + 8, 1u); }
+            }
+            if (landed && cl >= 0 && ts.s == 0 && ts.e == kTile) {
+                const uint4* st4 = reinterpret_cast<const uint4*>(ring + (size_t)(lq % kRingStages) * kTileBytes) + lane;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) t.v[i] = st4[i * 32];
+                vm[0] = vm[1] = 0xffffffffu;
+                have = true;
+            }
+            __syncwarp();
+            if (landed && lane == 0 && lq + kRingStages < nloc) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage's reads come before the copy that refills it
+                ring_issue(lq + kRingStages);
+            }
         }
         if (cl >= 0 && *reinterpret_cast<volatile uint32_t*>(misc + kMCursor) > budget) {
             if (lane == 0) atomicOr(&p.state[lt->lid[cl]].spec_bad, 1u);
         } else if (cl >= 0) {
-            const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-            TileRegs t;
-            uint32_t vm[2], keep[2];
-            load_tile(p.acc, ts, lane, t, vm);
+            if (!have) load_tile(p.acc, ts, lane, t, vm);
             if (mark_tile(t, vm, lt->sthr[cl], keep)) {
                 // room in the CTA's shared memory, or, when that is full, straight in the layer's region
                 const bool single = marks_single(keep[0], keep[1]);   // uniform over the warp
@@ -457,7 +582,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
                 first = __shfl_sync(0xffffffffu, first, 0);
                 uint2* dst = res;
                 uint32_t ytag = pack_y(0u, (uint32_t)cl, 0u);
-                const bool to_global = first + n > kStreamRes;
+                const bool to_global = first + n > kReadRes;
                 if (lane == 0) off = to_global ? atomicAdd(&p.state[lt->lid[cl]].cursor, n) : atomicAdd(&lt->v0[cl], n);
                 off = __shfl_sync(0xffffffffu, off, 0);
                 if (to_global) {
@@ -473,7 +598,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
                 if (to_global) { first = kTileGlobal; n = 0; }
             }
         }
-        if (lane == 0) { tt->first[lq] = first; tt->n[lq] = (uint16_t)n; tt->ge[lq] = off; }
+        if (lane == 0) { rt->first[lq] = first; rt->n[lq] = (uint16_t)n; rt->ge[lq] = off; }
     }
     __syncthreads();
     stamp(p, 1);
@@ -487,11 +612,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     __syncthreads();
     for (int lq = threadIdx.x; lq < nloc; lq += kSelThreads) {
         const int q = kStripe * (b + (lq / kStripe) * G) + lq % kStripe;
-        const uint32_t n = tt->n[lq], first = tt->first[lq];
+        const uint32_t n = rt->n[lq], first = rt->first[lq];
         if (q >= p.tiles || first == kTileGlobal) continue;
         if (n == 0) { p.runge[q] = make_uint2(0u, 0u); continue; }
         const int cl = (int)y_layer(res[first].y);
-        const uint32_t g = lt->v1[cl] + tt->ge[lq];
+        const uint32_t g = lt->v1[cl] + rt->ge[lq];
         p.runge[q] = make_uint2(g, n);
         uint2* dst = p.staging + lt->elem_off[cl] + g;
         const uint32_t yt = region_y(0u, (uint32_t)(q - lt->tf[cl]));
@@ -601,19 +726,20 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
 
 }  // namespace
 
-deft_status launch_select_stream(const SelParams& p, bool has_streamed, cudaStream_t stream) {
+deft_status launch_select_stream(const SelParams& p, bool has_streamed, bool ring, cudaStream_t stream) {
     static thread_local int attr_dev = -1;
     int dev = 0;
     DEFT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != attr_dev) {
-        DEFT_CUDA_TRY(cudaFuncSetAttribute(k_select_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        DEFT_CUDA_TRY(cudaFuncSetAttribute(k_select_stream<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        DEFT_CUDA_TRY(cudaFuncSetAttribute(k_select_stream<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_dev = dev;
     }
     SelParams args = p;
     int hs = has_streamed ? 1 : 0;
     void* kargs[] = {&args, &hs};
-    DEFT_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_select_stream), dim3(p.grid), dim3(kSelThreads),
-                                              kargs, kSmemBytes, stream));
+    void* fn = ring ? reinterpret_cast<void*>(k_select_stream<true>) : reinterpret_cast<void*>(k_select_stream<false>);
+    DEFT_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3(p.grid), dim3(kSelThreads), kargs, kSmemBytes, stream));
     return DEFT_OK;
 }
 

@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.deft_debug_select_timing.argtypes = [vp]
         L.deft_debug_select_kernel.restype = None
         L.deft_debug_select_kernel.argtypes = [i32]
+        L.deft_debug_select_ring.restype = None
+        L.deft_debug_select_ring.argtypes = [i32]
         L.deft_select_stats.restype = i32
         L.deft_select_stats.argtypes = [vp, sz, i32, vp, vp]
         L.deft_select_launch_max_elems.restype = i64
@@ -323,11 +325,16 @@ def deft_debug_select_kernel(single_pass) -> None:
     lib().deft_debug_select_kernel(-1 if single_pass is None else (1 if single_pass else 0))
 
 
+def deft_debug_select_ring(on: bool) -> None:
+    """The single-pass kernel reads through a ring of bulk copies (True, the default) or with plain loads (False)."""
+    lib().deft_debug_select_ring(1 if on else 0)
+
+
 def deft_select_stats(ws, n_layers: int, stream=None) -> dict:
     out = np.zeros(4, dtype=np.uint64)
     _check("deft_select_stats", lib().deft_select_stats(_dp(ws), ws.numel() * ws.element_size(), n_layers,
                                                         _hp(out), _stream(stream)))
-    return {"one_read": int(out[0]), "cut_failed": int(out[1]), "no_cut": int(out[2])}
+    return {"one_read": int(out[0]), "cut_failed": int(out[1]), "no_cut": int(out[2]), "ring_gave_up": int(out[3])}
 
 
 def deft_select_launch_max_elems() -> int:

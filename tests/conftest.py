@@ -19,12 +19,16 @@ def golden_dir():
 
 @pytest.fixture(autouse=True, scope="session")
 def _selection_kernel_choice():
-    """DEFT_SINGLE_PASS=1 / 0 runs the whole GPU suite with the single-pass selection kernel forced on / off
-    (results must not depend on the choice; the default picks by call size)."""
+    """DEFT_SINGLE_PASS=1 / 0 runs the whole GPU suite with the single-pass selection kernel forced on / off,
+    DEFT_RING=0 with that kernel reading with plain loads instead of through its ring of bulk copies
+    (results must not depend on either choice; the default picks the kernel by call size)."""
     import os
-    if os.environ.get("DEFT_SINGLE_PASS") in ("0", "1"):
+    if os.environ.get("DEFT_SINGLE_PASS") in ("0", "1") or os.environ.get("DEFT_RING") == "0":
         from paper_2307_03500_b200 import build as deft_build
         deft_build.build()
         from paper_2307_03500_b200 import deft
-        deft.deft_debug_select_kernel(os.environ["DEFT_SINGLE_PASS"] == "1")
+        if os.environ.get("DEFT_SINGLE_PASS") in ("0", "1"):
+            deft.deft_debug_select_kernel(os.environ["DEFT_SINGLE_PASS"] == "1")
+        if os.environ.get("DEFT_RING") == "0":
+            deft.deft_debug_select_ring(False)
     yield

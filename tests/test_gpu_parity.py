@@ -472,3 +472,135 @@ def test_capacity_errors_are_reported_not_faulted(deft):
     with pytest.raises(deft.DeftError) as ei:
         deft.deft_select(acc_d, start, np.array([5]), np.array([0], dtype=np.int32), val_d, idx_d, small)
     assert ei.value.status == deft.ERR_CAPACITY
+
+
+# ------------------------------------------------------------------------------------------
+# the forms of the selection kernel, the workspace's memory, limits
+# ------------------------------------------------------------------------------------------
+def test_every_form_of_the_selection_kernel_gives_the_same_bits(deft):
+    """Five-step kernel, single-pass kernel with plain loads, single-pass kernel reading through its ring
+    of bulk copies: three steps with the residual carried over (so that the later calls run on remembered
+    cuts), every form on its own workspace, each compared with the oracle."""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.scaled_down(W.bert_large(), 16)
+    N = w.n_workers
+    start, _ = oracle.split_layers(w.sizes, N)
+    size = np.diff(start)
+    forms = [(False, True), (True, False), (True, True)]     # (single pass, ring)
+    try:
+        runs = []
+        for single, ring in forms:
+            deft.deft_debug_select_kernel(single)
+            deft.deft_debug_select_ring(ring)
+            ds = DeftStep(w.sizes, N, w.density)
+            e = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+            outs = []
+            for t in range(3):
+                plan = ds.step_fused(e, _dev(w.gradient(t)), iteration=t)
+                torch.cuda.synchronize()
+                outs.append((plan, ds.val_d[:plan.sum_k].cpu().numpy(), ds.idx_d[:plan.sum_k].cpu().numpy(), e.cpu().numpy()))
+            st = deft.deft_select_stats(ds.ws, ds.L)
+            assert st["ring_gave_up"] == 0
+            if single:   # the second and third step found cuts for the layers of the first
+                assert st["one_read"] > 0
+            runs.append(outs)
+    finally:
+        deft.deft_debug_select_kernel(None)
+        deft.deft_debug_select_ring(True)
+    acc = np.zeros(w.n_g, dtype=np.float32)
+    for t in range(3):
+        oracle.accumulate(acc, w.gradient(t))
+        plan = runs[0][t][0]
+        want_val, want_idx = [], []
+        for r in range(N):
+            v, i = oracle.select_rank(acc, start, plan.k_l, oracle.my_layers(plan.bin_of_layer, t, r, N))
+            want_val.append(v)
+            want_idx.append(i)
+        want_val, want_idx = np.concatenate(want_val), np.concatenate(want_idx)
+        acc[want_idx] = 0.0
+        for outs in runs:
+            _, val, idx, e_now = outs[t]
+            assert np.array_equal(idx, want_idx) and val.tobytes() == want_val.tobytes()
+            assert e_now.tobytes() == acc.tobytes()
+    assert size.sum() == w.n_g
+
+
+@pytest.mark.parametrize("L", [1, 2, 3, 4])
+def test_few_large_layers_keep_their_remembered_cuts_across_the_norms_pass(deft, L):
+    """The norms pass and the selection share one workspace.  With one to four layers of a few million
+    elements the norm partials are many and the remembered cuts few: the second step must still find the
+    cuts of the first (every streamed layer finished in one read), and both steps must match the oracle."""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    sizes = [3_000_000 + 4099 * i for i in range(L)]
+    ds = DeftStep(sizes, 1, 0.002)
+    assert ds.L == L
+    n = int(sum(sizes))
+    e = torch.zeros(n, dtype=torch.float32, device="cuda")
+    start = np.asarray(ds.layer_start)
+    before = deft.deft_select_stats(ds.ws, ds.L)
+    mid = None
+    for t in range(2):
+        acc = W.adversarial_vector("gauss", n, seed=40 + t)      # a fresh draw of the same distribution, no gradient added
+        e.copy_(_dev(acc))
+        plan = ds.step_fused(e, None, iteration=t)
+        torch.cuda.synchronize()
+        k_l, _ = oracle.allocate_k(oracle.layer_norms(acc, start), np.diff(start), ds.k, oracle.MODE_EXACT)
+        assert plan.k_l.tolist() == k_l.tolist()
+        want_val, want_idx = oracle.select_rank(acc, start, k_l, np.arange(L, dtype=np.int32))
+        assert np.array_equal(ds.idx_d[:plan.sum_k].cpu().numpy(), want_idx)
+        assert ds.val_d[:plan.sum_k].cpu().numpy().tobytes() == want_val.tobytes()
+        acc[want_idx] = 0.0
+        assert e.cpu().numpy().tobytes() == acc.tobytes()
+        st = deft.deft_select_stats(ds.ws, ds.L)
+        if t == 1:
+            assert st["cut_failed"] == before["cut_failed"], "the cuts of the first step were lost or wrong"
+            assert st["no_cut"] == mid["no_cut"], "the second step had no cut for a layer the first step finished"
+            assert st["one_read"] == mid["one_read"] + L
+        mid = st
+
+
+def test_whole_step_with_pageable_host_norms(deft):
+    """deft_step hands the norms to the host through norms_h: pinned memory is read in place while the
+    device still works; ordinary pageable memory takes the copy-and-wait path.  Same result."""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.scaled_down(W.bert_large(), 64)
+    N = w.n_workers
+    ds_a = DeftStep(w.sizes, N, w.density)
+    ds_b = DeftStep(w.sizes, N, w.density)
+    ds_b.norms_h = torch.empty(ds_b.L, dtype=torch.float64)        # pageable
+    assert not ds_b.norms_h.is_pinned()
+    e_a = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+    e_b = torch.zeros_like(e_a)
+    for t in range(2):
+        g_d = _dev(w.gradient(t))
+        plan_a = ds_a.step_fused(e_a, g_d, iteration=t)
+        plan_b = ds_b.step_fused(e_b, g_d, iteration=t)
+        torch.cuda.synchronize()
+        assert plan_a.k_l.tolist() == plan_b.k_l.tolist() and plan_a.bin_of_layer.tolist() == plan_b.bin_of_layer.tolist()
+        s = plan_a.sum_k
+        assert torch.equal(ds_a.idx_d[:s], ds_b.idx_d[:s]) and torch.equal(ds_a.val_d[:s], ds_b.val_d[:s])
+        assert torch.equal(e_a, e_b)
+        assert ds_a.norms_h.numpy().tobytes() == ds_b.norms_h.numpy().tobytes()
+
+
+def test_beyond_one_launch_is_reported_not_attempted(deft):
+    """A single layer larger than what one selection launch can scan (every CTA owns a bounded number of
+    tiles) comes back as DEFT_ERR_TOO_LARGE before any kernel runs: the vector is never read, so it can be
+    left uninitialised.  About 16 GB of device memory for the vector and the workspace."""
+    n = deft.deft_select_launch_max_elems() + 4096
+    assert n < 2 ** 31 - 1
+    free, _ = torch.cuda.mem_get_info()
+    need = 4 * n + deft.deft_workspace_bytes(n, 1) + (1 << 30)
+    if free < need:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
+    acc_d = torch.empty(n, dtype=torch.float32, device="cuda")
+    ws = deft.alloc_workspace(n, 1)
+    val_d = torch.full((16,), 7.0, dtype=torch.float32, device="cuda")
+    idx_d = torch.full((16,), -7, dtype=torch.int64, device="cuda")
+    with pytest.raises(deft.DeftError) as ei:
+        deft.deft_topk_baseline(acc_d, 8, val_d[:8], idx_d[:8], ws)
+    assert ei.value.status == deft.ERR_TOO_LARGE
+    torch.cuda.synchronize()
+    assert torch.all(val_d == 7.0) and torch.all(idx_d == -7)
+    del acc_d, ws
+    torch.cuda.empty_cache()

@@ -186,3 +186,28 @@ def test_device_calls_reject_bad_arguments_without_touching_the_gpu():
     kl[1] = 50
     assert L.deft_select(fake, p(ls), p(kl), p(my), 2, fake, fake, 10, fake, 1 << 20, None) == deft.ERR_CAPACITY
     assert L.deft_select(fake, p(ls), p(kl), p(my), 2, fake, fake, 600, fake, 64, None) == deft.ERR_CAPACITY
+
+
+def test_size_limits_are_the_header_s():
+    """The header's limits are the ones the host code enforces: a layer of DEFT_MAX_LAYER_ELEMS elements is
+    planned, one element more is an invalid argument (before anything touches a GPU); the status that says
+    "beyond one launch" has its own name."""
+    header = open(os.path.join(ROOT, "include", "deft.h")).read()
+    limit = int(re.search(r"#define\s+DEFT_MAX_LAYER_ELEMS\s+(\d+)LL", header).group(1))
+    assert limit == 2 ** 31 - 1
+    assert int(re.search(r"#define\s+DEFT_ERR_TOO_LARGE\s+(-\d+)", header).group(1)) == deft.ERR_TOO_LARGE
+    assert deft.status_string(deft.ERR_TOO_LARGE) == "DEFT_ERR_TOO_LARGE"
+    bins = np.array([0, 1], dtype=np.int32)
+    k_l = np.array([7, 9], dtype=np.int64)
+    ok = deft.deft_plan_build(np.array([0, limit, limit + 4096], dtype=np.int64), k_l, bins, 2, 0)
+    n_layers, elems, k, off = deft.deft_plan_rank_table(ok, 2)
+    assert n_layers.tolist() == [1, 1] and elems.tolist() == [limit, 4096] and k.tolist() == [7, 9] and off.tolist() == [0, 7]
+    with pytest.raises(deft.DeftError) as ei:
+        deft.deft_plan_build(np.array([0, limit + 1, limit + 4097], dtype=np.int64), k_l, bins, 2, 0)
+    assert ei.value.status == deft.ERR_INVALID_ARG
+    # Top-k and the hard threshold take the same limit for their n (checked before the pointers are used)
+    L = deft.lib()
+    fake = ctypes.c_void_p(0x1000)
+    assert L.deft_topk_baseline(fake, limit + 1, 3, fake, fake, fake, 1 << 40, None) == deft.ERR_INVALID_ARG
+    # the workspace for the largest layer is a finite, monotone number
+    assert deft.deft_workspace_bytes(limit, 1) > 8 * limit

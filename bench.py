@@ -427,6 +427,10 @@ def run_ours(args):
     deft_build.build()
     from paper_2307_03500_b200 import deft
     from paper_2307_03500_b200.pipeline import DeftStep
+    if args.select_kernel != "auto":
+        deft.deft_debug_select_kernel(args.select_kernel == "single-pass")
+    if args.no_ring:
+        deft.deft_debug_select_ring(False)
 
     w = make_workload(args)
     N = w.n_workers
@@ -440,6 +444,7 @@ def run_ours(args):
     # to step), generated on the device BEFORE the timed region and kept resident; at most
     # args.pool draws (memory), cycled beyond that.
     pool = []
+    n_pool = 0
     if args.mode == "step":
         free_b, _ = torch.cuda.mem_get_info(dev)
         fit = int(max(1, (free_b - 24e9) // (4 * n_g)))
@@ -749,8 +754,9 @@ def run_ours(args):
                        "sum_k": int(plan.sum_k), "seed": w.seed, "k_mode": "EXACT",
                        "l2": "inputs larger than L2 (%.2f GB vector, no flush)" % (4.0 * n_g / 1e9),
                        "gradient_stream": "%d independent seeded draws generated on the device before timing, "
-                                          "one per step%s" % (len(pool), "" if len(pool) >= args.warmup + args.steps
+                                          "one per step%s" % (n_pool, "" if n_pool >= args.warmup + args.steps
                                                               else ", cycled"),
+                       "select_kernel": args.select_kernel, "single_pass_read": "plain loads" if args.no_ring else "bulk-copy ring",
                        "multi_gpu": "replicas only"},
             "clocks": clocks,
             "e2e": {"value": world * n_g / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
@@ -830,6 +836,10 @@ def main():
     ap.add_argument("--cpu-ranks", type=int, default=4, help="ranks the oracle runs for the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--select-kernel", default="auto", choices=["auto", "five-step", "single-pass"],
+                    help="which selection kernel runs (auto: by call size); for comparisons and profiles")
+    ap.add_argument("--no-ring", action="store_true",
+                    help="the single-pass kernel reads with plain loads instead of through its ring of bulk copies")
     ap.add_argument("--pool", type=int, default=105,
                     help="independent gradient draws kept on the device (one per step; cycled beyond that)")
     ap.add_argument("--mode", default="step", choices=["step", "topk", "norms", "select", "sweep", "trace"],

@@ -431,12 +431,17 @@ def run_ours(args):
         deft.deft_debug_select_kernel(args.select_kernel == "single-pass")
     if args.no_ring:
         deft.deft_debug_select_ring(False)
+    if args.no_staging:
+        deft.deft_debug_step_staging(False)
 
     w = make_workload(args)
     N = w.n_workers
     g_host = torch.from_numpy(w.gradient(0)).pin_memory()
     ds = DeftStep(w.sizes, N, w.density, device=dev)
     n_g, L, k = ds.n_g, ds.L, ds.k
+    # deft_step stages during the accumulate pass when the single-pass selection kernel takes the call
+    staged_step = (not args.no_staging) and args.select_kernel != "five-step" and L <= 1024 and \
+        (n_g >= 48_000_000 or args.select_kernel == "single-pass") and n_g <= 600_000_000
     g = g_host.to(dev)
     e = torch.zeros(n_g, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
@@ -479,7 +484,7 @@ def run_ours(args):
             th0 = time.perf_counter()
             plan = ds.step_fused(e, grad, it, -1, evs if rec is not None else None)
             th1 = time.perf_counter()
-            launches["n"] += 3                   # k_accum_norms, k_norm_finalize, k_select_fused
+            launches["n"] += 4 if staged_step else 3   # (k_stage_prepare,) k_accum_norms, k_norm_finalize, selection kernel
             if rec is not None:
                 rec.append({"acc": (evs[0], evs[1]), "sel": (evs[2], evs[3]), "gap": (evs[1], evs[2]),
                             "host_s": th1 - th0, "ranks": None, "plan": plan})
@@ -562,7 +567,7 @@ def run_ours(args):
     total_ms = t_begin.elapsed_time(t_end)
     gpu_launches = launches["n"]
     stats1 = deft.deft_select_stats(ds.ws, L)
-    layer_stats = {kk: stats1[kk] - stats0[kk] for kk in stats1}   # streamed layers over the timed steps
+    layer_stats = {kk: (stats1[kk] - stats0[kk]) % (1 << 32) for kk in stats1}   # streamed layers over the timed steps
 
     # a second, non-stationary stream: a pool of 4 draws cycled (the accumulated vector and with it every
     # layer's threshold keep shifting against the norms), same step, same timing
@@ -583,7 +588,26 @@ def run_ours(args):
     s_b = deft.deft_select_stats(ds.ws, L)
     ns_ms = tn0.elapsed_time(tn1) / ns_steps
     ns_sel = np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in ns_recs])
-    ns_stats = {kk: s_b[kk] - s_a[kk] for kk in s_b}
+    ns_stats = {kk: (s_b[kk] - s_a[kk]) % (1 << 32) for kk in s_b}
+
+    # the selection launch on its own (it reads the vector itself), for the kernel's own roofline when the
+    # timed step stages during the accumulate pass
+    alone = None
+    if staged_step:
+        deft.deft_debug_step_staging(False)
+        al_recs = []
+        s_c = deft.deft_select_stats(ds.ws, L)
+        fresh = torch.empty_like(g)
+        for it in range(3 + 10):
+            W.device_gradient(w, 10_000 + it, dev, out=fresh)   # a draw of its own every step, as in the timed region
+            one_step(args.warmup + args.steps + 64 + it, al_recs if it >= 3 else None, fresh)
+        stream.synchronize()
+        s_d = deft.deft_select_stats(ds.ws, L)
+        deft.deft_debug_step_staging(True)
+        alone = {"sel": np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in al_recs]),
+                 "acc": np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in al_recs]),
+                 "stats": {kk: (s_d[kk] - s_c[kk]) % (1 << 32) for kk in s_d}}
+        del fresh
 
     # per-call statistics from the events recorded inside the timed region
     t_acc = np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in recs])
@@ -605,7 +629,9 @@ def run_ours(args):
     plan_w = rank_recs[-1]["plan"]
     sel_med = np.median(t_sel, axis=0)
     t_host = t_gap
-    worker_ms = float(np.median(t_acc) + np.median(t_gap) + np.max(sel_med))
+    # (the per-worker passes run the plain accumulate + norms kernel: a worker's own launch reads its partition itself)
+    t_acc_w = np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in rank_recs])
+    worker_ms = float(np.median(t_acc_w) + np.median(t_gap) + np.max(sel_med))
 
     # load-model ablation: the same per-worker passes with layers packed by size instead of Eq. 3
     ds.cost_model = deft.COST_SIZE
@@ -697,15 +723,17 @@ def run_ours(args):
         # more in the five-step kernel, twice in all on the single-pass kernel's retry list).  The layer
         # counters of the library say how many layers went which way; layers are weighted equally here.
         traffic = ncu_traffic() or {}
-        all_ms = float(np.median(t_all))
+        sel_times = alone["sel"] if alone is not None else t_all
+        sel_stats = alone["stats"] if alone is not None else layer_stats
+        all_ms = float(np.median(sel_times))
         all_bytes = 8.0 * n_g + 12.0 * float(plan.sum_k)
         all_gbs = all_bytes / (all_ms * 1e-3) / 1e9
-        n_layers_seen = max(1, sum(layer_stats.values()))
-        reread = (layer_stats["cut_failed"] + layer_stats["no_cut"]) / n_layers_seen
+        n_layers_seen = max(1, sel_stats["one_read"] + sel_stats["cut_failed"] + sel_stats["no_cut"])
+        reread = (sel_stats["cut_failed"] + sel_stats["no_cut"]) / n_layers_seen
         moved_bytes = 4.0 * n_g * (1.0 + 2.0 * reread) + 12.0 * float(plan.sum_k)
         moved_gbs = moved_bytes / (all_ms * 1e-3) / 1e9
         sel_traffic = traffic.get("selection_one_read")
-        roof_sel = {"bound": "hbm", "kernel": "selection of all %d workers' partitions in one launch "
+        roof_sel = {"bound": "hbm", "kernel": "selection of all %d workers' partitions in one launch reading the vector itself "
                                               "(k_select_stream for calls of 48 M elements or more, else k_select_fused)" % N,
                     "achieved": moved_gbs, "peak": peak, "unit": "GB/s", "frac": moved_gbs / peak, "peak_kind": peak_kind,
                     "achieved_note": "bytes moved per launch (4 B per element read once where the remembered cut held, "
@@ -713,15 +741,43 @@ def run_ours(args):
                     "traffic": (sel_traffic["dram_bytes_per_elem"] * n_g if sel_traffic else None),
                     "traffic_note": ("per launch, scaled by elements from the ncu capture in %s" % sel_traffic["source"])
                                     if sel_traffic else "no ncu summary found",
-                    "bytes_per_launch": moved_bytes, "ms_per_launch": all_ms, "share_of_step": all_ms / ms_per_step,
-                    "ms_per_launch_mean": float(np.mean(t_all)), "ms_per_launch_max": float(np.max(t_all)),
-                    "layers_one_read": layer_stats["one_read"], "layers_cut_failed": layer_stats["cut_failed"],
-                    "layers_no_cut": layer_stats["no_cut"], "share_of_layers_read_again": reread,
+                    "bytes_per_launch": moved_bytes, "ms_per_launch": all_ms,
+                    "ms_per_launch_mean": float(np.mean(sel_times)), "ms_per_launch_max": float(np.max(sel_times)),
+                    "layers_one_read": sel_stats["one_read"], "layers_cut_failed": sel_stats["cut_failed"],
+                    "layers_no_cut": sel_stats["no_cut"], "share_of_layers_read_again": reread,
                     "frac_algorithmic": all_gbs / peak,
                     "frac_algorithmic_note": "two-read definition: (8 B per element + 12 B per selected entry) / time / peak; "
                                              "half of those bytes are never moved when the cut holds"}
+        if alone is not None:
+            roof_sel["where"] = ("10 steps after the timed region with staging in the accumulate pass switched off "
+                                 "(--no-staging runs the whole benchmark that way): step %.4f ms = accumulate+norms %.4f ms + "
+                                 "host gap + this launch" % (float(np.median(alone["acc"])) + float(np.median(t_gap)) + all_ms,
+                                                             float(np.median(alone["acc"]))))
+        else:
+            roof_sel["share_of_step"] = all_ms / ms_per_step
+        roof_finish = None
+        if staged_step:
+            fin_ms = float(np.median(t_all))
+            staged_per_step = layer_stats["staged_entries"] / max(1, args.steps)
+            fin_bytes = 8.0 * staged_per_step + 16.0 * float(plan.sum_k)
+            roof_finish = {"bound": "hbm", "kernel": "k_select_stream on entries staged by the accumulate pass (no read of the vector)",
+                           "achieved": fin_bytes / (fin_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                           "frac": fin_bytes / (fin_ms * 1e-3) / 1e9 / peak, "peak_kind": peak_kind,
+                           "achieved_note": "8 B per staged entry (read once into shared memory) + 16 B per selected entry "
+                                            "(value, index, cleared element); the launch is bound by latency, not bytes: "
+                                            "one CTA finishes a layer, and the largest layers take most of the launch",
+                           "traffic": None, "bytes_per_launch": fin_bytes, "ms_per_launch": fin_ms,
+                           "ms_per_launch_mean": float(np.mean(t_all)), "ms_per_launch_max": float(np.max(t_all)),
+                           "share_of_step": fin_ms / ms_per_step, "staged_entries_per_step": staged_per_step,
+                           "staged_over_selected": staged_per_step / max(1.0, float(plan.sum_k)),
+                           "layers_finished_from_staged": layer_stats["one_read"], "layers_cut_failed": layer_stats["cut_failed"],
+                           "layers_no_cut": layer_stats["no_cut"]}
         acc_traffic = traffic.get("k_accum_norms")
-        roof_acc = {"bound": "hbm", "kernel": "k_accum_norms (+k_norm_finalize, <1%)", "achieved": acc_gbs,
+        if staged_step:   # the pass also writes the staged entries
+            acc_bytes += 8.0 * layer_stats["staged_entries"] / max(1, args.steps)
+            acc_gbs = acc_bytes / (acc_ms * 1e-3) / 1e9
+        roof_acc = {"bound": "hbm", "kernel": ("k_accum_norms staging above the remembered cuts (+k_stage_prepare, k_norm_finalize, <1%)"
+                                               if staged_step else "k_accum_norms (+k_norm_finalize, <1%)"), "achieved": acc_gbs,
                     "peak": peak, "unit": "GB/s", "frac": min(1.0, acc_gbs / peak), "frac_uncapped": acc_gbs / peak,
                     "frac_note": "the denominator is a measured copy (half reads, half writes); this kernel reads two "
                                  "bytes for every byte it writes and runs a little above it: capped at 1",
@@ -731,7 +787,7 @@ def run_ours(args):
                                     if acc_traffic else "no ncu summary found",
                     "bytes_per_launch": acc_bytes, "ms_per_launch": acc_ms, "share_of_step": acc_ms / ms_per_step,
                     "frac_of_nominal_8TBs": acc_gbs / 8000.0}
-        sel_dominant = all_ms >= acc_ms
+        sel_dominant = (not staged_step) and all_ms >= acc_ms
         cpu = None
         if not args.no_cpu_baseline:
             c = oracle_step_sample(w, g_host.numpy(), args.cpu_ranks, threads=0, topk_slice=1 << 25)
@@ -756,7 +812,7 @@ def run_ours(args):
                        "gradient_stream": "%d independent seeded draws generated on the device before timing, "
                                           "one per step%s" % (n_pool, "" if n_pool >= args.warmup + args.steps
                                                               else ", cycled"),
-                       "select_kernel": args.select_kernel, "single_pass_read": "plain loads" if args.no_ring else "bulk-copy ring",
+                       "staging_in_accumulate_pass": bool(staged_step), "select_kernel": args.select_kernel, "single_pass_read": "plain loads" if args.no_ring else "bulk-copy ring",
                        "multi_gpu": "replicas only"},
             "clocks": clocks,
             "e2e": {"value": world * n_g / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
@@ -764,7 +820,8 @@ def run_ours(args):
             "gpu_launches": gpu_launches,
             # the dominant kernel of the timed step by time, then the other one
             "roofline": roof_sel if sel_dominant else roof_acc,
-            "roofline_other": roof_acc if sel_dominant else roof_sel,
+            "roofline_other": roof_acc if sel_dominant else (roof_finish if staged_step else roof_sel),
+            "roofline_select_standalone": roof_sel if staged_step else None,
             "roofline_select_per_worker": {
                 "bound": "hbm", "call": "one selection launch per worker (timed outside the step)",
                 "unit": "GB/s", "peak": peak,
@@ -779,12 +836,12 @@ def run_ours(args):
                 "note": "ranks of 8-16 M elements are latency-bound: 33-60 MB take 13-15 us to stream even for a bare "
                         "read kernel timed the same way; setup, four grid barriers and the steps between them add the rest"},
             "worker_view": {"ms_per_step_slowest_worker": worker_ms, "gelems": n_g / (worker_ms * 1e-3) / 1e9,
-                            "t_acc_norms_ms": acc_ms, "t_host_ms": float(np.median(t_host)),
+                            "t_acc_norms_ms": float(np.median(t_acc_w)), "t_host_ms": float(np.median(t_host)),
                             "t_host_note": "device-idle time between the norms and the selection launch: D2H copy of "
                                            "the norms, Algorithms 3 + 4, plan build and upload",
                             "select_ms_max": float(sel_med.max()), "select_ms_mean": float(sel_med[busy].mean()),
                             "select_ms_min": float(sel_med[busy].min()),
-                            "select_all_workers_one_launch_ms": all_ms,
+                            "select_all_workers_one_launch_ms": float(np.median(t_all)),
                             "select_gelems_system": n_g / (float(sel_med.max()) * 1e-3) / 1e9,
                             "slowest_rank": r_max, "slowest_rank_elems": int(plan_w.rank_elems[r_max]),
                             "slowest_rank_k": int(plan_w.rank_k[r_max]),
@@ -814,7 +871,7 @@ def run_ours(args):
                 "layers_no_cut": ns_stats["no_cut"]},
             "stream_stationary": {
                 "stream": "stationary", "what": "an independent draw every step", "steps": args.steps,
-                "ms_per_step": ms_per_step, "select_ms_median": all_ms, "select_ms_mean": float(np.mean(t_all)),
+                "ms_per_step": ms_per_step, "select_ms_median": float(np.median(t_all)), "select_ms_mean": float(np.mean(t_all)),
                 "select_ms_max": float(np.max(t_all)), "layers_one_read": layer_stats["one_read"],
                 "layers_cut_failed": layer_stats["cut_failed"], "layers_no_cut": layer_stats["no_cut"]},
             "extra": extra,
@@ -838,6 +895,8 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--select-kernel", default="auto", choices=["auto", "five-step", "single-pass"],
                     help="which selection kernel runs (auto: by call size); for comparisons and profiles")
+    ap.add_argument("--no-staging", action="store_true",
+                    help="the selection launch reads the vector itself instead of finding its entries staged by the accumulate pass")
     ap.add_argument("--no-ring", action="store_true",
                     help="the single-pass kernel reads with plain loads instead of through its ring of bulk copies")
     ap.add_argument("--pool", type=int, default=105,

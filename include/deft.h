@@ -96,6 +96,19 @@ DEFT_API void deft_debug_select_kernel(int32_t single_pass);
 DEFT_API void deft_debug_select_ring(int32_t on);
 
 /*
+ * Diagnostic: whether deft_step, when it runs all workers' selections in one launch on a vector the
+ * single-pass kernel takes, stages during the accumulate pass.  on != 0 (the default): the kernel that
+ * adds the gradient and sums the squares also puts every entry at or above its layer's remembered cut
+ * into the layer's staging region (the cut is taken from where the previous step found the layer's
+ * threshold, lowered by how much that has been moving from step to step: this step's norms and k_l do
+ * not exist yet), and the selection launch, which then knows k_l, finishes every layer for which at
+ * least k_l entries were staged without reading the vector at all; the other layers are read and
+ * searched in full inside the same launch.  on = 0: the selection launch does its own read.  Results
+ * never differ.  Not thread-safe; for measurements and tests.
+ */
+DEFT_API void deft_debug_step_staging(int32_t on);
+
+/*
  * Diagnostic: when timing_d (DEVICE, 1024 x uint64, zeroed by the caller) is not NULL every
  * later selection launch records GPU-timer stamps in nanoseconds (max over CTAs) and counters.
  * Both kernels: [0] kernel start, [14] / [15] staged entries (max over CTAs or layers / total).
@@ -218,8 +231,9 @@ DEFT_API deft_status deft_workspace_init(void* ws_d, size_t ws_bytes, int32_t n_
  * since deft_workspace_init: stats_h[0] layers it finished in one read, [1] layers whose remembered
  * cut failed (too few or far too many entries staged), [2] layers it had no usable cut for (nothing
  * remembered yet, or too dense); [1] and [2] were handed to the five-step kernel; [3] waits on the
- * bulk-copy ring that gave up (always 0 on a healthy device; see deft_debug_select_ring).
- * stats_h: HOST, 4 x uint64.  Waits for `stream`.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ * bulk-copy ring that gave up (always 0 on a healthy device; see deft_debug_select_ring); [4] entries
+ * staged for the layers counted in [0], modulo 2^32; [5..7] reserved (0).
+ * stats_h: HOST, 8 x uint64.  Waits for `stream`.  Errors: INVALID_ARG, CAPACITY, CUDA.
  */
 DEFT_API deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layers, uint64_t* stats_h,
                                        void* stream);

@@ -12,6 +12,7 @@ namespace deft {
 static thread_local int32_t g_last_cuda_error = 0;
 static unsigned long long* g_select_timing = nullptr;
 static int g_stream_kernel = -1;   // deft_debug_select_kernel: -1 by size, 0 never, 1 whenever possible
+static int g_step_fused = 1;       // deft_debug_step_staging: deft_step for all workers stages during the accumulate pass
 static int g_stream_ring = 1;      // deft_debug_select_ring: the single-pass kernel reads through a ring of bulk copies
 
 // Limits of the single-pass selection kernel (see select_rank).
@@ -38,6 +39,9 @@ int sm_count() {
 }
 
 namespace {
+
+// select_rank(prestaged = true): the call's layers do not suit the single-pass kernel (internal, never returned to callers)
+constexpr deft_status kNotPrestaged = 1000;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -186,7 +190,8 @@ struct FixedThreshold {
 
 deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan_d, int32_t rank,
                         float* val_d, int64_t* idx_d, int64_t out_cap, void* ws_d, size_t ws_bytes,
-                        cudaStream_t stream, bool zero_selected = false, FixedThreshold fixed = FixedThreshold()) {
+                        cudaStream_t stream, bool zero_selected = false, FixedThreshold fixed = FixedThreshold(),
+                        bool prestaged = false) {
     const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
     if (rank < 0 || rank > hdr->N) return DEFT_ERR_INVALID_ARG;   // rank N = all ranks' layers as one list
     const RankInfo& R = plan_ranks(plan_h)[rank];
@@ -210,6 +215,8 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     p.retry = reinterpret_cast<RetryHeader*>(ws + w.retry);
     p.retry_desc = reinterpret_cast<LayerDesc*>(ws + w.retry_desc);
     p.from_retry = 0;
+    p.prestaged = 0;
+    p.stage_tab = reinterpret_cast<const StageTab*>(ws + w.stage_tab);
     p.retry_elem_base = R.elem_base;
     p.runge = reinterpret_cast<uint2*>(ws + w.runge) + 2 * ((size_t)R.tile_base + (size_t)rank);
     p.staging = reinterpret_cast<uint2*>(ws + w.staging);
@@ -274,9 +281,11 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
             }
         }
         if (ok && (streamed == 0 || 2 * sparse >= streamed)) {
+            p.prestaged = prestaged ? 1 : 0;
             return launch_select_stream(p, streamed != 0, g_stream_ring != 0, stream);
         }
     }
+    if (prestaged) return kNotPrestaged;   // the caller clears what the accumulate pass staged and calls again
     if (R.n_my > 1 && R.n_my <= kMaxWeightedLayers && (int64_t)R.tiles >= (int64_t)kInterleaveTiles * p.grid) {
         const int n = R.n_my;
         std::vector<uint32_t> Wp((size_t)n + 1), wt((size_t)n);
@@ -332,6 +341,7 @@ void deft_debug_select_timing(void* timing_d) { g_select_timing = static_cast<un
 
 int64_t deft_select_launch_max_elems(void) { return (int64_t)sm_count() * kMaxLocalTiles * kTile; }
 
+void deft_debug_step_staging(int32_t on) { g_step_fused = on != 0 ? 1 : 0; }
 void deft_debug_select_ring(int32_t on) { g_stream_ring = on != 0 ? 1 : 0; }
 void deft_debug_select_kernel(int32_t single_pass) { g_stream_kernel = single_pass < 0 ? -1 : (single_pass != 0 ? 1 : 0); }
 
@@ -348,7 +358,7 @@ deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layer
     if (!ws_d || !stats_h || n_layers < 1) return DEFT_ERR_INVALID_ARG;
     const WsLayout w = ws_layout(1, n_layers, 1);
     if (w.hint + 256 > ws_bytes) return DEFT_ERR_CAPACITY;
-    uint32_t words[9];
+    uint32_t words[10];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DEFT_CUDA_TRY(cudaMemcpyAsync(words, static_cast<const char*>(ws_d) + w.hint, sizeof(words), cudaMemcpyDeviceToHost, st));
     DEFT_CUDA_TRY(cudaStreamSynchronize(st));
@@ -356,6 +366,8 @@ deft_status deft_select_stats(const void* ws_d, size_t ws_bytes, int32_t n_layer
     stats_h[1] = words[5];
     stats_h[2] = words[6];
     stats_h[3] = words[8];
+    stats_h[4] = words[9];
+    stats_h[5] = stats_h[6] = stats_h[7] = 0;
     return DEFT_OK;
 }
 
@@ -661,15 +673,45 @@ deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, cons
     volatile uint64_t* slots = reinterpret_cast<volatile uint64_t*>(norms_h);
     if (mapped)
         for (int32_t l = 0; l < L; ++l) slots[l] = kUnset | (uint32_t)l;
+    // With all workers in one launch and a vector the single-pass selection kernel takes, the accumulate pass
+    // stages every entry above its layer's remembered cut on the way (the per-layer counters are cleared
+    // BEFORE it then): the selection launch finds its entries staged and reads nothing.
+    const WsLayout wl = ws_layout(1, L, 1);   // the cleared area's place depends on the layer count only
+    if (wl.zero_end > ws_bytes) return DEFT_ERR_CAPACITY;
+    bool fused = g_step_fused != 0 && g_stream_kernel != 0 && rank < 0 && L <= kStreamMaxLayers && n_g <= kStreamMaxElems &&
+                 (g_stream_kernel > 0 || n_g >= kStreamMinElems);
+    StageLaunch sl{};
+    if (fused) {
+        int64_t tiles_all = 0;
+        for (int32_t l = 0; l < L; ++l) {
+            const int64_t a = layer_start_h[l], b = layer_start_h[l + 1];
+            if (a < 0 || b <= a) { fused = false; break; }
+            tiles_all += (b - 1) / kTile - a / kTile + 1;
+        }
+        if (fused && layer_start_h[L] == n_g && tiles_all <= INT32_MAX) {
+            const WsLayout w = ws_layout(n_g, L, tiles_all);
+            if (w.total > ws_bytes) return DEFT_ERR_CAPACITY;
+            char* ws = static_cast<char*>(ws_d);
+            sl.hint = reinterpret_cast<const LayerHint*>(ws + w.hint + 256);
+            sl.tab = reinterpret_cast<StageTab*>(ws + w.stage_tab);
+            sl.state = reinterpret_cast<LayerState*>(ws + w.state);
+            sl.runge = reinterpret_cast<uint2*>(ws + w.runge) + 2 * (size_t)N;   // the all-layers list's table
+            sl.staging = reinterpret_cast<uint2*>(ws + w.staging);
+        } else {
+            fused = false;
+        }
+    }
+    if (fused)
+        DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + wl.zero_begin, 0, wl.zero_end - wl.zero_begin, st));
     DEFT_CUDA_TRY(mark(0));
     deft_status s = launch_layer_norms(resid_acc_d, grad_d, n_g, layer_start_d, L, norms_d,
-                                       reinterpret_cast<double*>(static_cast<char*>(ws_d) + part), st, mapped);
+                                       reinterpret_cast<double*>(static_cast<char*>(ws_d) + part), st, mapped,
+                                       fused ? &sl : nullptr);
     if (s != DEFT_OK) return s;
     DEFT_CUDA_TRY(mark(1));
     // the per-layer counters of the selection are cleared while the host plans
-    const WsLayout wl = ws_layout(1, L, 1);   // the cleared area's place depends on the layer count only
-    if (wl.zero_end > ws_bytes) return DEFT_ERR_CAPACITY;
-    DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + wl.zero_begin, 0, wl.zero_end - wl.zero_begin, st));
+    if (!fused)
+        DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + wl.zero_begin, 0, wl.zero_end - wl.zero_begin, st));
     bool have = false;
     if (mapped) {
         const auto t0 = std::chrono::steady_clock::now();
@@ -691,7 +733,22 @@ deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, cons
     if (sp < 0) return sp;
     DEFT_CUDA_TRY(mark(2));
     if (rank < 0) {
-        s = deft_select_update_all(resid_acc_d, n_g, plan_h, plan_d, val_d, idx_d, out_cap, ws_d, ws_bytes, stream);
+        s = kNotPrestaged;
+        if (fused) {
+            const PlanHeader* hdr = static_cast<const PlanHeader*>(plan_h);
+            const RankInfo& M = plan_ranks(plan_h)[hdr->N];
+            if (!val_d || !idx_d) return DEFT_ERR_INVALID_ARG;
+            if (out_cap < hdr->total_k) return DEFT_ERR_CAPACITY;
+            if (M.n_my == L)
+                s = select_rank(resid_acc_d, plan_h, plan_d, hdr->N, val_d, idx_d, M.k, ws_d, ws_bytes, st, true,
+                                FixedThreshold(), true);
+            if (s == kNotPrestaged || s == DEFT_ERR_TOO_LARGE) {   // not this step: forget what was staged
+                DEFT_CUDA_TRY(cudaMemsetAsync(static_cast<char*>(ws_d) + wl.zero_begin, 0, wl.zero_end - wl.zero_begin, st));
+                s = kNotPrestaged;
+            }
+        }
+        if (s == kNotPrestaged)
+            s = deft_select_update_all(resid_acc_d, n_g, plan_h, plan_d, val_d, idx_d, out_cap, ws_d, ws_bytes, stream);
     } else {
         const RankInfo& R = plan_ranks(plan_h)[rank];
         if (!val_d || !idx_d) return DEFT_ERR_INVALID_ARG;

@@ -164,14 +164,27 @@ static_assert(sizeof(LayerState) == 64, "LayerState layout");
 
 // What a selection leaves behind per layer for the next call on the same workspace (the only
 // per-layer data that lives across calls; it steers speed, never results).
-struct LayerHint {                   // 16 bytes
+struct LayerHint {                   // 32 bytes
     uint32_t pos_p1;                 // 1 + position (key >> 15: 1/16 first-level bucket) of the `rank`-th largest key; 0 = nothing remembered
     uint32_t norm_bits;              // that call's layer norm (float bits)
     uint32_t rank;                   // the rank the bucket belongs to (k + margin of that call)
     uint32_t err;                    // how the predictions have been doing, in the same unit: running mean of (found -
                                      // predicted) as int16 in the low half, running mean deviation in the high half
+    uint32_t err_same;               // the same two numbers for the prediction "where it was last time" (no norm, no rank
+                                     // known yet): what staging during the accumulate pass goes by
+    uint32_t pad[3];
 };
-static_assert(sizeof(LayerHint) == 16, "LayerHint layout");
+static_assert(sizeof(LayerHint) == 32, "LayerHint layout");
+
+// Staging during the accumulate pass (before the step's plan exists): where a layer's staged entries and
+// its tiles' table entries go follows from the layer table alone: the layout the plan gives the list of
+// all layers in address order.  Written by a small kernel before the accumulate pass.
+struct StageTab {                    // per layer, 16 bytes
+    uint32_t cut;                    // entries with key >= cut are staged (0xffffffff: none for this layer)
+    int32_t tile_first;              // the layer's first tile in the all-layers list
+    int64_t elem_off;                // first slot of the layer's staging region
+};
+static_assert(sizeof(StageTab) == 16, "StageTab layout");
 
 // Layers the single-pass kernel could not finish (no usable cut, cut too high, too dense) are
 // appended here for a following launch of the five-step kernel on exactly those layers.
@@ -192,6 +205,7 @@ struct WsLayout {
     size_t norm_partial;             // partial sums of the accumulate + norm call (its place depends on L only)
     size_t runge, staging;
     size_t hint;                     // 256 bytes of control words, then one LayerHint per layer; kept across calls
+    size_t stage_tab;                // one StageTab per layer (+ 1): rewritten by every step that stages during the accumulate pass
     size_t total;
 };
 
@@ -208,6 +222,7 @@ inline WsLayout ws_layout(int64_t elems, int64_t L, int64_t tiles) {
     w.zero_end = off;
     w.hint = off;     off += 256 + align_up(sizeof(LayerHint) * (size_t)L, 256);   // control words, then one entry per layer
     w.retry_desc = off; off += align_up(sizeof(LayerDesc) * (size_t)(L + 1), 256);
+    w.stage_tab = off; off += align_up(sizeof(StageTab) * (size_t)(L + 1), 256);
     w.norm_partial = off; off += align_up(sizeof(double) * (size_t)((elems + kTileA - 1) / kTileA + L + 1), 256);
     const size_t slots = 2 * (size_t)tiles + 2 * (size_t)kMaxRanks;   // rank r starts at 2*(tile_base + r)
     w.runge = off;    off += align_up(sizeof(uint2) * slots, 256);
@@ -242,7 +257,8 @@ struct SelParams {
                                      // that have finished this call, [3] layers whose speculative cut failed in this
                                      // call, [7] calls in which some cut failed (running total); single-pass kernel,
                                      // running totals: [4] layers it finished, [5] layers whose cut failed, [6]
-                                     // layers it had no usable cut for
+                                     // layers it had no usable cut for, [8] waits on its ring that gave up, [9] staged
+                                     // entries of the layers it finished (modulo 2^32)
     LayerHint* hint;                 // [L] what the previous call found; read and updated
     uint2* runge;                    // five-step kernel: this rank's (CTA, layer) pairs (slot = CTA + layer position):
                                      // totals.  Single-pass kernel: per tile of the rank (first entry within the layer's
@@ -250,6 +266,8 @@ struct SelParams {
     RetryHeader* retry;              // layers left for a following launch, see RetryHeader
     LayerDesc* retry_desc;           // [L + 1]
     int32_t from_retry;              // five steps: 1 = the layer list is the retry list (no speculation, no small layers)
+    int32_t prestaged;               // single-pass kernel: 1 = the accumulate pass has staged already (cuts in stage_tab): no read
+    const StageTab* stage_tab;       // [L] by layer id
     int64_t retry_elem_base;         // staging index at which the retry list's layers are placed
     uint2* staging;                  // absolute base of the spill area; (value bits, offset in tile)
     float* val;                      // the rank's output
@@ -277,9 +295,18 @@ int sm_count();
     } while (0)
 
 // Launchers (each enqueues on `stream` and returns a status).
+// stage != NULL: the pass also stages every entry at or above its layer's remembered cut (see deft_norms.cu)
+struct StageLaunch {
+    const LayerHint* hint;           // [L] what the previous selection left behind
+    StageTab* tab;                   // [L + 1] written by the call
+    LayerState* state;               // [L] cleared before the call
+    uint2* runge;                    // tile table of the all-layers list
+    uint2* staging;
+};
 deft_status launch_layer_norms(float* resid_acc_d, const float* grad_d, int64_t n_g,
                                const int64_t* layer_start_d, int32_t L, double* norms_d,
-                               double* partial_d, cudaStream_t stream, double* norms_host_mapped = nullptr);
+                               double* partial_d, cudaStream_t stream, double* norms_host_mapped = nullptr,
+                               const StageLaunch* stage = nullptr);
 deft_status launch_select(const SelParams& p, cudaStream_t stream);
 deft_status launch_select_stream(const SelParams& p, bool has_streamed, bool ring, cudaStream_t stream);
 deft_status launch_residual_update(float* acc_d, const int64_t* idx_d, int64_t count,

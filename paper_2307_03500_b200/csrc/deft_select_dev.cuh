@@ -725,36 +725,65 @@ __device__ __forceinline__ uint32_t predict_cut(const LayerHint* hp, int64_t k, 
     return (uint32_t)(pa * align) << kFinePosShift;
 }
 
+// Folds one prediction error into a packed (running mean, running mean deviation) word.
+__device__ __forceinline__ uint32_t fold_error(uint32_t w, int err, int slack, int dev_max) {
+    int bias = hint_bias(w), dev = (int)(w >> 16);
+    dev = dev < kDevMin ? kDevInit : (dev > dev_max ? dev_max : dev);
+    err = err < -kBiasMax ? -kBiasMax : (err > kBiasMax ? kBiasMax : err);
+    const int d = err - bias;
+    int ad = (d < 0 ? -d : d) - slack;
+    ad = ad < 0 ? 0 : ad;
+    bias += d / 4;
+    dev += (ad - dev) / 4;
+    if (d < -2 * dev - kErrUnit) dev += kErrUnit / 2;   // found well below what the cut allowed for: back off at once
+    dev = dev < kDevMin ? kDevMin : (dev > dev_max ? dev_max : dev);
+    return ((uint32_t)dev << 16) | ((uint32_t)bias & 0xffffu);
+}
+constexpr int kDevSameMax = 4 * kErrUnit;
+
 // After a layer's selection: remembers `pos` (where the key of rank safe_rank(k) was found if `exact`, else an
 // upper bound of it: just below the cut, when fewer than safe_rank(k) entries were at or above the cut)
-// and folds the prediction's error into the running means.  `slack`: half the width of the interval the
-// position is known to lie in (0 for the single-pass kernel's fine bins, half a bucket for a first-level
-// bucket), which is not counted as deviation.  One thread.
+// and folds the errors of two predictions into their running means: the one from this call's norm and
+// rank (predict_pos), and "where it was last time" (what a pass that runs before the norms and the
+// ranks are known has to go by).  `slack`: half the width of the interval the position is known to lie
+// in (0 for the single-pass kernel's fine bins, half a bucket for a first-level bucket), which is not
+// counted as deviation.  One thread.
 __device__ __forceinline__ void hint_update(LayerHint* hp, uint32_t pos, bool exact, int slack, uint32_t k, double norm) {
     const uint4 raw = *reinterpret_cast<const uint4*>(hp);
     const int pf = predict_pos(raw, k, norm);
-    int bias = hint_bias(raw.w), dev = hint_dev(raw.w);
+    const int low = exact ? 0 : kErrUnit / 2;   // the truth lies at or below a bound
+    uint32_t w = ((uint32_t)kDevInit << 16), w_same = ((uint32_t)(2 * kDevInit) << 16);
     if (pf != INT_MIN) {
-        int err = (int)pos - pf;
-        if (!exact) err -= kErrUnit / 2;   // the truth lies at or below the bound
-        err = err < -kBiasMax ? -kBiasMax : (err > kBiasMax ? kBiasMax : err);
-        const int d = err - bias;
-        int ad = (d < 0 ? -d : d) - slack;
-        ad = ad < 0 ? 0 : ad;
-        bias += d / 4;
-        dev += (ad - dev) / 4;
-        if (d < -2 * dev - kErrUnit) dev += kErrUnit / 2;   // found well below what the cut allowed for: back off at once
-        dev = dev < kDevMin ? kDevMin : (dev > kDevMax ? kDevMax : dev);
-    } else {
-        bias = 0;
-        dev = kDevInit;
+        w = fold_error(raw.w, (int)pos - pf - low, slack, kDevMax);
+        w_same = fold_error(hp->err_same, (int)pos - ((int)raw.x - 1) - low, slack, kDevSameMax);
     }
     uint4 out;
     out.x = pos + 1u;
     out.y = __float_as_uint((float)norm);
     out.z = safe_rank(k);
-    out.w = ((uint32_t)dev << 16) | ((uint32_t)bias & 0xffffu);
+    out.w = w;
     *reinterpret_cast<uint4*>(hp) = out;
+    hp->err_same = w_same;
+}
+
+// The cut a pass stages by when it runs BEFORE the step's norms and ranks exist (the accumulate pass): the
+// place the previous call found, lowered by the running mean and twice the deviation of how that simple
+// prediction has been doing for the layer (changes of the norm and of k_l from step to step are in
+// there), rounded down to a quarter bucket.  The rank of the previous call stands in for k_l in the density
+// test.  0xffffffff = none.
+__device__ __forceinline__ uint32_t prestage_cut(const LayerHint* hp, int64_t size) {
+    const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(hp));
+    if (raw.x == 0u || raw.x > (uint32_t)kBins1 * kErrUnit) return 0xffffffffu;
+    if ((int64_t)raw.z * kSpecDensity > size) return 0xffffffffu;
+    const uint32_t w = __ldcg(&hp->err_same);
+    int dev = (int)(w >> 16);
+    dev = dev < kDevMin ? 2 * kDevInit : (dev > kDevSameMax ? kDevSameMax : dev);
+    const int at = (int)raw.x - 1 + hint_bias(w) - 2 * dev - kErrUnit / 4;
+    constexpr int align = kErrUnit / 4;
+    int pa = at >= 0 ? at / align : 0;
+    const int top = (kBins1 - 1) * kErrUnit / align;
+    pa = pa > top ? top : pa;
+    return (uint32_t)(pa * align) << kFinePosShift;
 }
 
 // Fills the table of the CTA's streamed layers; returns how many there are (at most
@@ -785,6 +814,9 @@ __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRa
             uint32_t sthr = 0xffffffffu;
             if (p.fixed_thr) {
                 sthr = p.thr_key + 1u;                       // key >= thr_key + 1  <=>  key > thr_key
+            } else if (spec_on && p.prestaged) {
+                sthr = p.stage_tab[p.desc[j].layer_id].cut;   // what the accumulate pass staged by
+                if (sthr != 0xffffffffu) scratch[kMTried - kMScratch] = 1u;
             } else if (spec_on) {
                 sthr = predict_cut(p.hint + p.desc[j].layer_id, p.desc[j].k, p.desc[j].end - p.desc[j].start,
                                    p.desc[j].norm, cut_align);

@@ -205,6 +205,7 @@ __device__ __noinline__ bool finish_layer(const SelParams& p, LayerTable* lt, in
             hint_update(hp, cutp > 0u ? cutp - 1u : 0u, false, 0, k, norm);
         }
         atomicAdd(p.spec_ctl + 4, 1u);
+        atomicAdd(p.spec_ctl + 9, S);
     }
     // the candidates: (key, index order) as one 64-bit word that sorts the way the selection wants
     // (larger key first, then lower index: .y grows with the index and bit 31 of it is free), and
@@ -463,7 +464,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     r.jA = 0; r.jB = p.n_my - 1;
     const int nl = build_layer_table(p, r, lt, misc + kMScratch, true, kErrUnit / 4);   // every streamed layer of the call
     const int nstripe = (p.tiles + kStripe - 1) / kStripe;
-    const int nloc = (b < nstripe ? (nstripe - b + G - 1) / G : 0) * kStripe;
+    // (prestaged: the accumulate pass has staged the call's entries and filled the tile table: nothing to read)
+    const int nloc = p.prestaged ? 0 : (b < nstripe ? (nstripe - b + G - 1) / G : 0) * kStripe;
     if (threadIdx.x == 0) { misc[kMCursor] = 0; misc[kMTileCtr] = 0; misc[kMBudget] = 4096u; }
     constexpr uint32_t kReadRes = kRing ? kRingRes : kStreamRes;   // staged entries the CTA keeps in shared memory during the read
     uint64_t* const bars = reinterpret_cast<uint64_t*>(misc + kMRingBar);
@@ -647,8 +649,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     }
 
     // ---- every layer's entries are in its region: the layers are finished one per CTA, round-robin ----
-    __threadfence();
-    grid.sync();
+    if (!p.prestaged) {   // uniform over the grid
+        __threadfence();
+        grid.sync();
+    }
     // largest first (a layer's cost grows with what was staged for it): the order is worked out by
     // every CTA for itself; CTA b starts with the b-th largest, the rest are taken from a counter
     // (cleared with the plan upload) as CTAs become free

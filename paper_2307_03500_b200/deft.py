@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.deft_debug_select_kernel.argtypes = [i32]
         L.deft_debug_select_ring.restype = None
         L.deft_debug_select_ring.argtypes = [i32]
+        L.deft_debug_step_staging.restype = None
+        L.deft_debug_step_staging.argtypes = [i32]
         L.deft_select_stats.restype = i32
         L.deft_select_stats.argtypes = [vp, sz, i32, vp, vp]
         L.deft_select_launch_max_elems.restype = i64
@@ -330,11 +332,17 @@ def deft_debug_select_ring(on: bool) -> None:
     lib().deft_debug_select_ring(1 if on else 0)
 
 
+def deft_debug_step_staging(on: bool) -> None:
+    """deft_step for all workers stages during the accumulate pass (True, the default) or leaves the read to the
+    selection launch (False)."""
+    lib().deft_debug_step_staging(1 if on else 0)
+
+
 def deft_select_stats(ws, n_layers: int, stream=None) -> dict:
-    out = np.zeros(4, dtype=np.uint64)
+    out = np.zeros(8, dtype=np.uint64)
     _check("deft_select_stats", lib().deft_select_stats(_dp(ws), ws.numel() * ws.element_size(), n_layers,
                                                         _hp(out), _stream(stream)))
-    return {"one_read": int(out[0]), "cut_failed": int(out[1]), "no_cut": int(out[2]), "ring_gave_up": int(out[3])}
+    return {"one_read": int(out[0]), "cut_failed": int(out[1]), "no_cut": int(out[2]), "ring_gave_up": int(out[3]), "staged_entries": int(out[4])}
 
 
 def deft_select_launch_max_elems() -> int:

@@ -604,3 +604,50 @@ def test_beyond_one_launch_is_reported_not_attempted(deft):
     assert torch.all(val_d == 7.0) and torch.all(idx_d == -7)
     del acc_d, ws
     torch.cuda.empty_cache()
+
+
+def test_staging_in_the_accumulate_pass_never_changes_the_result(deft):
+    """deft_step for all workers stages above the remembered cuts while it accumulates, before this step's
+    norms and k_l exist.  Steps whose gradients jump up (far too many entries staged: the per-tile lists
+    overflow) and down (too few staged) must come out like every other step: the layers concerned are
+    searched in full.  Every step is compared with the oracle, and with the same step without staging."""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.scaled_down(W.bert_large(), 16)
+    N = w.n_workers
+    start, _ = oracle.split_layers(w.sizes, N)
+    scales = [1.0, 1.0, 1.0, 64.0, 1.0, 1.0 / 4096.0, 1.0, 1.0]
+    try:
+        deft.deft_debug_select_kernel(True)      # the vector is below the size at which the default takes this path
+        ds = {True: DeftStep(w.sizes, N, w.density), False: DeftStep(w.sizes, N, w.density)}
+        e = {True: torch.zeros(w.n_g, dtype=torch.float32, device="cuda"),
+             False: torch.zeros(w.n_g, dtype=torch.float32, device="cuda")}
+        acc = np.zeros(w.n_g, dtype=np.float32)
+        for t, sc in enumerate(scales):
+            g = (w.gradient(t) * np.float32(sc)).astype(np.float32)
+            g_d = _dev(g)
+            plans = {}
+            for staged in (True, False):
+                deft.deft_debug_step_staging(staged)
+                plans[staged] = ds[staged].step_fused(e[staged], g_d, iteration=t)
+                torch.cuda.synchronize()
+            oracle.accumulate(acc, g)
+            plan = plans[True]
+            assert plan.k_l.tolist() == plans[False].k_l.tolist()
+            want_val, want_idx = [], []
+            for r in range(N):
+                v, i = oracle.select_rank(acc, start, plan.k_l, oracle.my_layers(plan.bin_of_layer, t, r, N))
+                want_val.append(v)
+                want_idx.append(i)
+            want_val, want_idx = np.concatenate(want_val), np.concatenate(want_idx)
+            acc[want_idx] = 0.0
+            for staged in (True, False):
+                s = plan.sum_k
+                assert np.array_equal(ds[staged].idx_d[:s].cpu().numpy(), want_idx), (t, staged)
+                assert ds[staged].val_d[:s].cpu().numpy().tobytes() == want_val.tobytes(), (t, staged)
+                assert e[staged].cpu().numpy().tobytes() == acc.tobytes(), (t, staged)
+        st = deft.deft_select_stats(ds[True].ws, ds[True].L)
+        assert st["one_read"] > 0 and st["staged_entries"] > 0      # layers were finished from what the pass staged
+        assert st["cut_failed"] > 0                                   # and the jumps made cuts fail
+    finally:
+        deft.deft_debug_select_kernel(None)
+        deft.deft_debug_step_staging(True)

@@ -772,7 +772,7 @@ def run_ours(args):
                            "staged_over_selected": staged_per_step / max(1.0, float(plan.sum_k)),
                            "layers_finished_from_staged": layer_stats["one_read"], "layers_cut_failed": layer_stats["cut_failed"],
                            "layers_no_cut": layer_stats["no_cut"]}
-        acc_traffic = traffic.get("k_accum_norms")
+        acc_traffic = traffic.get("k_accum_norms_staging" if staged_step else "k_accum_norms")
         if staged_step:   # the pass also writes the staged entries
             acc_bytes += 8.0 * layer_stats["staged_entries"] / max(1, args.steps)
             acc_gbs = acc_bytes / (acc_ms * 1e-3) / 1e9

@@ -9,7 +9,7 @@ namespace deft {
 namespace {
 
 // Speculative staging (see the head of this file).  The cut a call leaves for the next one is the
-// position of the (k + max(k / 4, kSpecSlack))-th largest key: a margin in rank, so that it
+// position of the (k + max(k / 8, kSpecSlack))-th largest key: a margin in rank, so that it
 // adapts to the tail of the layer's distribution and to k (the k-th largest of a handful moves
 // by several buckets from draw to draw, the k-th of a million hardly at all).
 constexpr uint32_t kSpecSlack = 48;
@@ -675,7 +675,7 @@ __device__ __forceinline__ bool is_direct(const SelParams& p, int j) {
 // The rank whose key the remembered bucket belongs to: some way below the k-th largest, so that the
 // cut holds when the distribution moves a little (the k-th largest of a handful moves by several
 // buckets from draw to draw, the k-th of a million hardly at all).
-__device__ __forceinline__ uint32_t safe_rank(uint32_t k) { return k + (k / 4 > kSpecSlack ? k / 4 : kSpecSlack); }
+__device__ __forceinline__ uint32_t safe_rank(uint32_t k) { return k + (k / 8 > kSpecSlack ? k / 8 : kSpecSlack); }
 
 // ---- the speculative cut of a layer, from what the previous call on the workspace left behind ----
 // Remembered per layer: where the previous call found the key of rank safe_rank(k), as a position on the
@@ -778,7 +778,7 @@ __device__ __forceinline__ uint32_t prestage_cut(const LayerHint* hp, int64_t si
     const uint32_t w = __ldcg(&hp->err_same);
     int dev = (int)(w >> 16);
     dev = dev < kDevMin ? 2 * kDevInit : (dev > kDevSameMax ? kDevSameMax : dev);
-    const int at = (int)raw.x - 1 + hint_bias(w) - 2 * dev - kErrUnit / 4;
+    const int at = (int)raw.x - 1 + hint_bias(w) - 2 * dev - kErrUnit / 8;
     constexpr int align = kErrUnit / 4;
     int pa = at >= 0 ? at / align : 0;
     const int top = (kBins1 - 1) * kErrUnit / align;

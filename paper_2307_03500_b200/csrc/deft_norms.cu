@@ -89,25 +89,30 @@ k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
         const int64_t hi = (lo + kTileA < n) ? lo + kTileA : n;
         int l = layer_of(ls, L, lo);
         const int l_first = l;
+        const bool whole = hi - lo == kTileA && __ldg(ls + l + 1) >= hi;   // the tile lies inside layer l
         if (kStage) {
             __syncthreads();   // the lists of the previous tile have been written out
             if (threadIdx.x < kStageLists) ss->cnt[threadIdx.x] = 0u;
             if (threadIdx.x == 0) {
-                // the (at most two) staged layers that overlap [lo, hi)
+                // the (at most two) staged layers that overlap [lo, hi); a tile inside one layer needs no search
                 int found = 0;
                 ss->layer[0] = ss->layer[1] = -1;
                 ss->cut[0] = ss->cut[1] = 0xffffffffu;
-                for (int ll = l_first; ll < L && __ldg(ls + ll) < hi && found < 2; ++ll) {
-                    if (__ldg(ls + ll + 1) - __ldg(ls + ll) > kDirectElems) {
-                        ss->layer[found] = ll;
-                        ss->cut[found] = sa.tab[ll].cut;
-                        ++found;
+                if (whole) {
+                    if (__ldg(ls + l + 1) - __ldg(ls + l) > kDirectElems) ss->layer[0] = l;   // (its cut: every thread reads it itself)
+                } else {
+                    for (int ll = l_first; ll < L && __ldg(ls + ll) < hi && found < 2; ++ll) {
+                        if (__ldg(ls + ll + 1) - __ldg(ls + ll) > kDirectElems) {
+                            ss->layer[found] = ll;
+                            ss->cut[found] = sa.tab[ll].cut;
+                            ++found;
+                        }
                     }
                 }
             }
             __syncthreads();
         }
-        if (hi - lo == kTileA && __ldg(ls + l + 1) >= hi) {
+        if (whole) {
             // whole tile inside layer l: 8 float4 per thread, squares in fp32 per 8 elements
             float4* e4 = reinterpret_cast<float4*>(e + lo);
             const float4* g4 = reinterpret_cast<const float4*>(g + lo);
@@ -115,7 +120,8 @@ k_accum_norms(float* __restrict__ e, const float* __restrict__ g, int64_t n,
             uint32_t cut = 0xffffffffu;
             float cutf = 0.0f;
             if (kStage) {
-                cut = ss->layer[0] == l ? ss->cut[0] : 0xffffffffu;
+                cut = (__ldg(ls + l + 1) - __ldg(ls + l) > kDirectElems) ? sa.tab[l].cut : 0xffffffffu;
+                if (threadIdx.x == 0) ss->cut[0] = cut;   // for the warps that write the lists out (behind a barrier)
                 cutf = __uint_as_float(cut < 0x7f800000u ? cut : 0x7f800000u);
             }
 #pragma unroll

@@ -20,6 +20,46 @@ struct SortKey {
     int32_t id;
     bool operator<(const SortKey& o) const { return key != o.key ? key < o.key : id < o.id; }
 };
+
+// Sorts keys (filled by the caller, keys[i].id == i) ascending.  The order a planner needs changes little
+// from one step to the next, so the keys are first laid out in the order the previous call on this thread
+// ended with and finished by insertion (a handful of moves per step instead of L log L compares); when
+// the moves add up (a different model, a shuffled vector) the standard sort takes over.  The order is
+// total (ties by id), so the result does not depend on the starting point.  `order` is kept by the caller
+// per planner (thread-local).
+void sort_from_last_order(std::vector<SortKey>& keys, std::vector<int32_t>& order, std::vector<SortKey>& tmp) {
+    const size_t n = keys.size();
+    bool usable = order.size() == n;
+    if (usable) {
+        tmp.resize(n);
+        for (size_t i = 0; i < n; ++i) {
+            const int32_t id = order[i];
+            if (id < 0 || (size_t)id >= n) { usable = false; break; }
+            tmp[i] = keys[(size_t)id];
+        }
+    }
+    if (usable) {
+        size_t moves = 0;
+        const size_t budget = 8 * n + 64;
+        size_t i = 1;
+        for (; i < n && moves <= budget; ++i) {
+            const SortKey x = tmp[i];
+            size_t j = i;
+            while (j > 0 && x < tmp[j - 1]) {
+                tmp[j] = tmp[j - 1];
+                --j;
+                ++moves;
+            }
+            tmp[j] = x;
+        }
+        if (i < n) std::sort(tmp.begin(), tmp.end());   // (a permutation of the keys either way)
+        keys.swap(tmp);
+    } else {
+        std::sort(keys.begin(), keys.end());
+    }
+    order.resize(n);
+    for (size_t i = 0; i < n; ++i) order[i] = keys[i].id;
+}
 }  // namespace
 
 extern "C" {
@@ -109,7 +149,9 @@ deft_status deft_allocate_k(const double* norms_h, const int64_t* layer_size_h, 
         std::memcpy(&bits, &v, 8);
         keys[l] = SortKey{~bits, l};
     }
-    std::sort(keys.begin(), keys.end());
+    static thread_local std::vector<int32_t> last_order;
+    static thread_local std::vector<SortKey> sort_tmp;
+    sort_from_last_order(keys, last_order, sort_tmp);
     for (int32_t p = 0; p < L; ++p) prio[p] = keys[p].id;
 
     // tail[p] = norms of priority positions p, p+1, ..., L-1 added from the back.
@@ -206,7 +248,9 @@ deft_status deft_partition_model(const int64_t* layer_size_h, const int64_t* k_l
         std::memcpy(&bits, &v, 8);
         keys[l] = SortKey{~bits, l};
     }
-    std::sort(keys.begin(), keys.end());
+    static thread_local std::vector<int32_t> last_order;
+    static thread_local std::vector<SortKey> sort_tmp;
+    sort_from_last_order(keys, last_order, sort_tmp);
     load.assign((size_t)N, 0.0);
     typedef std::pair<double, int32_t> Bin;   // (load, id): smallest load first, then lowest id
     static thread_local std::vector<Bin> heap;

@@ -405,7 +405,7 @@ def run_extra(dev):
     rows.append(r)
     for d in (0.1, 0.001):
         for N in (1, 8, 64):
-            rows.append(config(W.gpt2_medium(N, d), 3, 3))
+            rows.append(config(W.gpt2_medium(N, d), 6, 6))
     return rows
 
 

@@ -789,7 +789,7 @@ def run_ours(args):
                     "frac_of_nominal_8TBs": acc_gbs / 8000.0}
         sel_dominant = (not staged_step) and all_ms >= acc_ms
         cpu = None
-        if not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline:   # the oracle is timed on a single-GPU run only
             c = oracle_step_sample(w, g_host.numpy(), args.cpu_ranks, threads=0, topk_slice=1 << 25)
             cpu = {"value": n_g / c["est_step_s"] / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                    "estimated": True, "sample": c["sample"], "est_ms_per_step": c["est_step_s"] * 1e3,

@@ -16,7 +16,6 @@ static int g_step_fused = 1;       // deft_debug_step_staging: deft_step for all
 static int g_stream_ring = 1;      // deft_debug_select_ring: the single-pass kernel reads through a ring of bulk copies
 
 // Limits of the single-pass selection kernel (see select_rank).
-constexpr int64_t kStreamMaxK = 65536;              // entries one layer may select
 constexpr int64_t kStreamMaxElems = 600000000;      // elements of one call
 constexpr int64_t kStreamMinElems = 48000000;       // below this the five-step kernel is the faster one (measured)
 constexpr int kStreamMaxLayers = 1024;              // layers of one call (its layer map lives in shared memory)
@@ -259,11 +258,13 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
     std::vector<int> q0((size_t)p.grid + 1);
     for (int b = 0; b <= p.grid; ++b) q0[b] = (int)((int64_t)R.tiles * b / p.grid);
     if (!within_limits(q0)) return DEFT_ERR_TOO_LARGE;
-    // The single-pass kernel takes the call when most of what it streams can be speculated on (sparse
-    // layers of moderate k; whether a cut is remembered for them only the device knows: layers without
-    // one go on its retry list, which the same launch works off with the five steps behind a grid barrier).  Its finishing CTA handles a layer alone, so layers that select very many
-    // entries, and calls too large for the retry list's split to stay within a CTA's limits, are left to
-    // the five-step kernel alone.
+    // The single-pass kernel takes the call when at least half of what it streams can be speculated on (sparse
+    // layers of moderate k; whether a cut is remembered for them only the device knows).  Its finishing CTA
+    // handles a layer alone, so dense layers, layers that select very many entries and layers without a
+    // remembered cut go on its retry list, which the same launch works off with the five steps behind a grid
+    // barrier: those steps then split only THESE layers' tiles over the CTAs, which balances a call that
+    // mixes sparse and dense layers better than one split over all of them (0.62 against 1.1 ms on a 355 M-element
+    // vector at density 0.01); a call that is mostly dense is better off with the five steps alone.
     if (!fixed.on && (g_stream_kernel > 0 || (g_stream_kernel < 0 && R.elems >= kStreamMinElems))) {
         int64_t streamed = 0, sparse = 0;
         int n_streamed = 0;
@@ -275,10 +276,7 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
             if (size <= kDirectElems) continue;
             streamed += size;
             if (++n_streamed > kMaxLocalLayers) ok = false;
-            if (hd[j].k * kSpecDensity <= size) {
-                sparse += size;
-                if (hd[j].k > kStreamMaxK) ok = false;
-            }
+            if (hd[j].k * kSpecDensity <= size && stream_can_finish(hd[j].k, size)) sparse += size;   // layers it can finish itself
         }
         if (ok && (streamed == 0 || 2 * sparse >= streamed)) {
             p.prestaged = prestaged ? 1 : 0;

@@ -60,6 +60,15 @@ constexpr int kMaxWeightedLayers = 8192;
 #define DEFT_HD
 #endif
 
+// Layers the single-pass kernel's finishing CTA takes (one CTA per layer: 2 to 7 us per 1000 staged entries, the
+// more the fewer of them fit in shared memory): those that select up to 16384 entries.  A layer that selects more
+// is read again by the whole grid instead, which is faster however large it is.
+constexpr int64_t kStreamMaxK = 16384;
+DEFT_HD inline bool stream_can_finish(int64_t k, int64_t size) {
+    (void)size;
+    return k <= kStreamMaxK;
+}
+
 // Cost of one tile of a layer in units of 1/64 of a tile that stages nothing (constants fitted
 // to step timings on B200: +50 % once most 16-byte loads of the tile hold an entry, +0.55 % per
 // staged entry for the later passes).  Layers that are not streamed cost nothing.

@@ -147,7 +147,9 @@ __device__ __noinline__ bool finish_layer(const SelParams& p, LayerTable* lt, in
     Lap lap;
     lap.start(p.timing);
     LayerHint* hp = p.hint + lid;
-    if (S < k || flooded) {
+    // (far more staged than selected: one CTA would take longer over them than the grid takes to read the
+    // layer again)
+    if (S < k || flooded || (unsigned long long)S > 6ull * k + 8192ull) {
         // the cut was too high (fewer than k entries reached the staging area) or far too low (a CTA
         // stopped staging): the layer goes to the retry list; a cut that was too high lowers the next ones
         if (tid == 0) {
@@ -462,7 +464,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) k_select_stream(const SelParam
     r.il = 0; r.q0tab = nullptr; r.nsuper = 0;
     r.q0 = 0; r.q1 = p.tiles; r.nloc = 0;
     r.jA = 0; r.jB = p.n_my - 1;
-    const int nl = build_layer_table(p, r, lt, misc + kMScratch, true, kErrUnit / 4);   // every streamed layer of the call
+    const int nl = build_layer_table(p, r, lt, misc + kMScratch, true, kErrUnit / 4, true);   // every streamed layer of the call
     const int nstripe = (p.tiles + kStripe - 1) / kStripe;
     // (prestaged: the accumulate pass has staged the call's entries and filled the tile table: nothing to read)
     const int nloc = p.prestaged ? 0 : (b < nstripe ? (nstripe - b + G - 1) / G : 0) * kStripe;

@@ -276,7 +276,10 @@ deft_status select_rank(const float* acc_d, const void* plan_h, const void* plan
             if (size <= kDirectElems) continue;
             streamed += size;
             if (++n_streamed > kMaxLocalLayers) ok = false;
-            if (hd[j].k * kSpecDensity <= size && stream_can_finish(hd[j].k, size)) sparse += size;   // layers it can finish itself
+            if (hd[j].k * kSpecDensity <= size) {
+                if (!prestaged && hd[j].k > kStreamMaxK) ok = false;   // (reading for itself it takes all sparse layers or none)
+                if (stream_can_finish(hd[j].k, prestaged)) sparse += size;   // layers it can finish itself
+            }
         }
         if (ok && (streamed == 0 || 2 * sparse >= streamed)) {
             p.prestaged = prestaged ? 1 : 0;

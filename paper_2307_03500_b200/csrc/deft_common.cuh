@@ -61,12 +61,12 @@ constexpr int kMaxWeightedLayers = 8192;
 #endif
 
 // Layers the single-pass kernel's finishing CTA takes (one CTA per layer: 2 to 7 us per 1000 staged entries, the
-// more the fewer of them fit in shared memory): those that select up to 16384 entries.  A layer that selects more
-// is read again by the whole grid instead, which is faster however large it is.
-constexpr int64_t kStreamMaxK = 16384;
-DEFT_HD inline bool stream_can_finish(int64_t k, int64_t size) {
-    (void)size;
-    return k <= kStreamMaxK;
+// more the fewer of them fit in shared memory).  When the kernel stages for itself (tight cuts: about two
+// staged entries per selected one) those that select up to 65536 entries; when the accumulate pass has staged
+// (wider margins) up to 16384: a layer that selects more is read again by the whole grid instead.
+constexpr int64_t kStreamMaxK = 65536, kStreamMaxKPrestaged = 16384;
+DEFT_HD inline bool stream_can_finish(int64_t k, bool prestaged) {
+    return k <= (prestaged ? kStreamMaxKPrestaged : kStreamMaxK);
 }
 
 // Cost of one tile of a layer in units of 1/64 of a tile that stages nothing (constants fitted

@@ -774,7 +774,7 @@ __device__ __forceinline__ void hint_update(LayerHint* hp, uint32_t pos, bool ex
 __device__ __forceinline__ uint32_t prestage_cut(const LayerHint* hp, int64_t size) {
     const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(hp));
     if (raw.x == 0u || raw.x > (uint32_t)kBins1 * kErrUnit) return 0xffffffffu;
-    if ((int64_t)raw.z * kSpecDensity > size || !stream_can_finish((int64_t)raw.z * 8 / 9, size)) return 0xffffffffu;
+    if ((int64_t)raw.z * kSpecDensity > size || !stream_can_finish((int64_t)raw.z * 8 / 9, true)) return 0xffffffffu;
     const uint32_t w = __ldcg(&hp->err_same);
     int dev = (int)(w >> 16);
     dev = dev < kDevMin ? 2 * kDevInit : (dev > kDevSameMax ? kDevSameMax : dev);
@@ -814,7 +814,7 @@ __device__ __forceinline__ int build_layer_table(const SelParams& p, const CtaRa
             uint32_t sthr = 0xffffffffu;
             if (p.fixed_thr) {
                 sthr = p.thr_key + 1u;                       // key >= thr_key + 1  <=>  key > thr_key
-            } else if (spec_on && one_cta_finishes && !stream_can_finish(p.desc[j].k, p.desc[j].end - p.desc[j].start)) {
+            } else if (spec_on && one_cta_finishes && !stream_can_finish(p.desc[j].k, p.prestaged != 0)) {
                 sthr = 0xffffffffu;                          // too many entries for the caller's way of finishing a layer
             } else if (spec_on && p.prestaged) {
                 sthr = p.stage_tab[p.desc[j].layer_id].cut;   // what the accumulate pass staged by

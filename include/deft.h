@@ -78,8 +78,8 @@ DEFT_API int32_t deft_last_cuda_error(void);
 
 /*
  * Diagnostic: which selection kernel later calls use.  single_pass = 0: the five-step kernel alone;
- * 1: the single-pass kernel whenever a call's layers allow it (sparse layers of moderate k_l, at most
- * 1024 layers of which at most 256 larger than 16384 elements); -1 (the default): the single-pass
+ * 1: the single-pass kernel whenever a call's layers allow it (at least half of its elements in sparse
+ * layers of moderate k_l, at most 1024 layers of which at most 256 larger than 16384 elements); -1 (the default): the single-pass
  * kernel for such calls of 48 M elements or more, the five-step kernel for smaller ones.  Results never
  * differ.  Not thread-safe; for measurements and tests.
  */
@@ -423,6 +423,9 @@ DEFT_API deft_status deft_select_update_all(float* acc_d, int64_t n_g, const voi
  * synchronising the stream; any other host memory takes the copy + synchronise route.
  * events: NULL, or 4 cudaEvent_t handles (HOST array) recorded on `stream` before and after
  * the accumulate+norms kernels and before and after the selection launch.
+ * With rank = -1 on a vector the single-pass selection kernel takes (48 M to 600 M elements, at most 1024
+ * layers) the accumulate pass also stages every entry at or above its layer's remembered cut for the
+ * selection, whose launch then reads nothing (see deft_debug_step_staging); the results are the same.
  * All other arguments, results and errors as in the calls it is made of.
  */
 DEFT_API deft_status deft_step(float* resid_acc_d, const float* grad_d, int64_t n_g, const int64_t* layer_start_h,

@@ -1,26 +1,24 @@
-// Layer-wise top-k selection for one worker (Algorithm 5) in ONE pass over the worker's part of the
-// vector, without grid-wide barriers: the kernel for calls whose layers were selected from before on
-// the same workspace (a training loop).
+// Layer-wise top-k selection (Algorithm 5) in ONE pass over the call's part of the vector: the kernel for
+// large calls whose layers were selected from before on the same workspace (a training loop).
 //
-// Every layer comes with a remembered cut: the first-level bucket (key bits 30..19) in which the
-// previous call found a key some way below the layer's k-th largest, moved by the change of the
-// layer's norm (predict_cut).  One CTA of 512 threads per SM owns a contiguous run of the call's
-// tiles.  A warp holds a whole tile in registers, tests it against the cut (one floating-point
-// test per 16-byte load, the exact test only where that one passes) and moves the entries at or
-// above the cut, in index order, into the CTA's shared memory.  At the end of its run the CTA
-// copies what it staged into the layer's region of the staging area (one atomic per CTA and layer
-// reserves the room) and publishes (first entry, entries) for each of its tiles.
+// Every layer comes with a remembered cut (predict_cut in deft_select_dev.cuh).  One CTA of 512 threads
+// per SM; the call's tiles are dealt to the CTAs in stripes.  Whole tiles arrive through a ring of
+// bulk copies in shared memory (or, in the kernel's other form, by plain loads); a warp takes a tile into
+// registers, tests it against the cut (one floating-point test per 16-byte load, the exact test only
+// where that one passes) and moves the entries at or above the cut, in index order, into the CTA's shared
+// memory.  At the end of its read the CTA copies what it staged into the layers' regions of the staging
+// area (one atomic per CTA and layer reserves the room) and writes (first entry, entries) per tile.
+// With `prestaged` the accumulate pass has done all of this already and the kernel starts here:
 //
-// The CTA that completes a layer's last tile (a ticket per layer) finishes the layer on its own while
-// the others are still reading: if at least k entries were staged, the k largest of the layer are
-// among them, so a three-level radix select over the staged entries (shared memory) gives the exact
-// threshold key T and the number of entries equal to T to take; the per-tile counts, a prefix over
-// the layer's tiles and the ordered write (value, int64 index; ascending index, equal keys: lowest
-// indices first; optionally clearing the selected entries of the vector) follow from the published
-// tile table.  The result never depends on the cut: a layer with fewer than k staged entries, or
-// without a usable cut, or too dense to speculate on, is appended to a retry list, and the five-step
-// kernel (deft_select.cu), launched right behind this one, selects exactly those layers with its two
-// reads (it returns at once when the list is empty).
+// Behind a grid barrier every layer is finished by one CTA (largest first, from a queue): if at least k
+// entries were staged, the k largest of the layer are among them; a histogram of fine bins counted from
+// the cut gives the bin of the k-th largest, the few entries of that bin are ranked among themselves,
+// and the selected entries are written in ascending index (value, int64 index; equal keys: lowest indices
+// first) from the tile table: per-tile counts, a prefix over the layer's tiles, an ordered write.
+// Behind a second barrier the whole grid clears the selected entries in the vector, and the layers that
+// could not be finished (fewer than k staged entries, far too many, no usable cut, too dense, k too
+// large for one CTA) go through the five steps (deft_select_steps.cuh) inside the same launch.
+// The result never depends on the cuts.
 //
 // Layers of at most kDirectElems elements are handed out from a counter; one CTA loads each whole.
 //

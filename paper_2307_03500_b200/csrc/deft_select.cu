@@ -5,12 +5,14 @@
 // shared memory; overflow spills to HBM), so after the reading steps all work is local to the
 // CTA that staged the data.
 //
-//   A   read 1: per-layer histogram of key bits 30..19 in shared memory, flushed with integer
-//       atomics; the CTA that flushes a layer's last tiles finds the bucket b1 holding the
-//       k-th largest key.  In the same pass every entry at or above a SPECULATIVE cut — the
-//       bucket in which the previous call found the layer's (k + max(k/2, 48))-th largest key,
-//       moved by the change of the layer's norm — is moved, in index order, behind the CTA's
-//       staging cursor.
+//   A   read 1: layers WITHOUT a remembered cut get a histogram of key bits 30..19 in shared memory,
+//       flushed with integer atomics.  Layers WITH a speculative cut (predict_cut: where the previous
+//       call found a key a little below the layer's k-th largest, moved by the change of the layer's
+//       norm, lowered by how well that has been predicting) are not histogrammed element by element:
+//       every entry at or above the cut is moved, in index order, behind the CTA's staging cursor and
+//       counted under its bucket, which gives the complete histogram from the cut upwards.  The CTA
+//       that flushes a layer's last tiles finds the bucket b1 holding the k-th largest key; a layer
+//       whose counts do not reach k has its full histogram built in a second round of this step.
 //   B   a CTA whose cuts were all at or below the true b1 already holds everything it needs
 //       and reads nothing; any other CTA drops what it staged and reads its tiles a second
 //       time with the true cut.  Then the staged entries of bucket b1 feed the level-2

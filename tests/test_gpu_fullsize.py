@@ -124,3 +124,48 @@ def test_topk_baseline_full_size(deft):
     torch.cuda.synchronize()
     keys = g.view(np.uint32) & np.uint32(0x7FFFFFFF)
     _check_layer_properties(keys, g, 0, w.n_g, k, idx_d.cpu().numpy(), val_d.cpu().numpy())
+
+
+def test_bench_step_with_staging_full_size(deft):
+    """The call the benchmark times: deft_step for all workers at full size, three steps with the residual
+    carried over, so that from the second step on the accumulate pass stages above remembered cuts and the
+    selection launch finishes from those entries.  Every layer of every step is checked through properties
+    that hold at any size (exactly k_l entries, ascending, values as in the vector, everything larger
+    selected, ties by lowest index), the residual byte for byte."""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.bert_large()
+    N = w.n_workers
+    ds = DeftStep(w.sizes, N, w.density)
+    start = np.asarray(ds.layer_start)
+    size = np.diff(start)
+    e_d = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+    acc = np.zeros(w.n_g, dtype=np.float32)
+    before = deft.deft_select_stats(ds.ws, ds.L)
+    for t in range(3):
+        g = w.gradient(t)
+        g_d = torch.from_numpy(g).cuda()
+        plan = ds.step_fused(e_d, g_d, iteration=t)
+        torch.cuda.synchronize()
+        del g_d
+        oracle.accumulate(acc, g)
+        norms = oracle.layer_norms(acc, start)
+        got = ds.norms_h.numpy()
+        assert np.all(np.abs(got - norms) <= 1e-5 * norms)
+        k_l, s = oracle.allocate_k(got, size, ds.k, oracle.MODE_EXACT)
+        bins, _ = oracle.partition(size, k_l, N)
+        assert plan.k_l.tolist() == k_l.tolist() and plan.bin_of_layer.tolist() == bins.tolist() and s == plan.sum_k
+        idx_all = ds.idx_d[: plan.sum_k].cpu().numpy()
+        val_all = ds.val_d[: plan.sum_k].cpu().numpy()
+        keys = acc.view(np.uint32) & np.uint32(0x7FFFFFFF)
+        for r in range(N):
+            pos = int(plan.rank_out_off[r])
+            for l in oracle.my_layers(bins, t, r, N):
+                kk = int(k_l[l])
+                _check_layer_properties(keys, acc, int(start[l]), int(start[l + 1]), kk, idx_all[pos:pos + kk],
+                                        val_all[pos:pos + kk])
+                pos += kk
+            assert pos == int(plan.rank_out_off[r + 1])
+        acc[idx_all] = 0.0
+        assert e_d.cpu().numpy().tobytes() == acc.tobytes()
+    st = deft.deft_select_stats(ds.ws, ds.L)
+    assert st["one_read"] > before["one_read"] and st["staged_entries"] > 0   # the later steps ran on staged entries

@@ -457,8 +457,17 @@ def run_ours(args):
         pool = [W.device_gradient(w, t, dev) for t in range(n_pool)]
         torch.cuda.synchronize()
 
+    ev_pool = []   # events made (and their handles created) ahead of a timed region, so that making them is not in it
+
     def ev():
-        return torch.cuda.Event(enable_timing=True)
+        return ev_pool.pop() if ev_pool else torch.cuda.Event(enable_timing=True)
+
+    def prepare_events(n):
+        for _ in range(n):
+            x = torch.cuda.Event(enable_timing=True)
+            x.record(stream)   # torch creates the handle on the first record
+            ev_pool.append(x)
+        stream.synchronize()
 
     def barrier():
         if world > 1:
@@ -482,7 +491,7 @@ def run_ours(args):
         if marks is None and not with_topk:
             evs = [ev(), ev(), ev(), ev()]
             th0 = time.perf_counter()
-            plan = ds.step_fused(e, grad, it, -1, evs if rec is not None else None)
+            plan = ds.step_fused(e, grad, it, -1, evs if rec is not None else None, stream)
             th1 = time.perf_counter()
             launches["n"] += 4 if staged_step else 3   # (k_stage_prepare,) k_accum_norms, k_norm_finalize, selection kernel
             if rec is not None:
@@ -557,6 +566,7 @@ def run_ours(args):
     recs = []
     launches["n"] = 0
     t_begin, t_end = ev(), ev()
+    prepare_events(4 * args.steps)
     barrier()
     t_begin.record(stream)
     for it in range(args.steps):

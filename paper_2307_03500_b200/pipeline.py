@@ -102,22 +102,58 @@ class DeftStep:
 
     # -- the whole step in ONE library call ---------------------------------------------------
     def step_fused(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, rank: int = -1,
-                   events=None) -> StepPlan:
+                   events=None, stream=None) -> StepPlan:
         """accumulate + norms -> host planning -> selection + residual update, one C call
-        (`deft_step`): all simulated workers in one launch (rank = -1) or one worker."""
+        (`deft_step`): all simulated workers in one launch (rank = -1) or one worker.
+        The pointers of the buffers this object owns are marshalled once and reused: the call is made
+        every step and the device waits for the host between its two kernels."""
+        import ctypes
         if not hasattr(self, "_k_l"):
             self._k_l = np.empty(self.L, dtype=np.int64)
             self._bins = np.empty(self.L, dtype=np.int32)
             self._load = np.empty(self.N, dtype=np.float64)
-        sum_k, _ = deft.deft_step(resid, grad, self.layer_start, self.layer_start_d, self.N, self.k, self.mode,
-                                  self.cost_model, iteration, rank, self.norms_d, self.norms_h, self._k_l, self._bins,
-                                  self._load, self.plan_h, self.plan_d, self.val_d, self.idx_d, self.ws, events)
+            self._ls_h = np.ascontiguousarray(self.layer_start, dtype=np.int64)
+            self._sum_k = ctypes.c_int64(0)
+            vp = ctypes.c_void_p
+            self._fixed = dict(
+                ls_h=vp(self._ls_h.ctypes.data), ls_d=vp(self.layer_start_d.data_ptr()), norms_d=vp(self.norms_d.data_ptr()),
+                norms_h=vp(self.norms_h.data_ptr()), k_l=vp(self._k_l.ctypes.data), sum_k=ctypes.byref(self._sum_k),
+                bins=vp(self._bins.ctypes.data), load=vp(self._load.ctypes.data), plan_h=vp(self.plan_h.ctypes.data),
+                plan_d=vp(self.plan_d.data_ptr()), val_d=vp(self.val_d.data_ptr()), idx_d=vp(self.idx_d.data_ptr()),
+                ws=vp(self.ws.data_ptr()), ws_bytes=self.ws.numel() * self.ws.element_size(),
+                out_cap=min(self.val_d.numel(), self.idx_d.numel()), plan_cap=self.plan_h.size,
+                norms_h_ptr=self.norms_h.data_ptr())
+        f = self._fixed
+        if f["norms_h_ptr"] != self.norms_h.data_ptr():      # the caller swapped the host buffer for the norms
+            f["norms_h"] = ctypes.c_void_p(self.norms_h.data_ptr())
+            f["norms_h_ptr"] = self.norms_h.data_ptr()
+        if resid.dtype != torch.float32 or not resid.is_cuda or not resid.is_contiguous() or resid.numel() != self.n_g:
+            raise ValueError("resid: a contiguous float32 CUDA tensor of n_g elements")
+        if grad is not None and (grad.dtype != torch.float32 or not grad.is_cuda or not grad.is_contiguous()
+                                 or grad.numel() != self.n_g):
+            raise ValueError("grad: a contiguous float32 CUDA tensor of n_g elements")
+        ev = None
+        if events is not None:
+            flat = []
+            for e in events:
+                if e.cuda_event == 0:   # torch creates the handle lazily, on first record
+                    e.record()
+                flat.append(e.cuda_event)
+            ev = (ctypes.c_void_p * 4)(*flat)
+        st = torch.cuda.current_stream(self.device) if stream is None else stream
+        status = deft.lib().deft_step(
+            ctypes.c_void_p(resid.data_ptr()), None if grad is None else ctypes.c_void_p(grad.data_ptr()), self.n_g,
+            f["ls_h"], f["ls_d"], self.L, self.N, int(self.k), int(self.mode), int(self.cost_model), int(iteration),
+            int(rank), f["norms_d"], f["norms_h"], f["k_l"], f["sum_k"], f["bins"], f["load"], f["plan_h"],
+            f["plan_cap"], f["plan_d"], f["val_d"], f["idx_d"], f["out_cap"], f["ws"], f["ws_bytes"], ev,
+            ctypes.c_void_p(st.cuda_stream))
+        deft._check("deft_step", status, allow_warn=True)
         n_layers, elems, rank_k, out_off = deft.deft_plan_rank_table(self.plan_h, self.N)
-        off = np.zeros(self.N + 1, dtype=np.int64)
+        off = np.empty(self.N + 1, dtype=np.int64)
         off[:-1] = out_off
         off[-1] = out_off[-1] + rank_k[-1]
-        return StepPlan(self._k_l.copy(), sum_k, self._bins.copy(), self._load.copy(), n_layers, rank_k, elems, off,
-                        self.plan_h)
+        return StepPlan(self._k_l.copy(), int(self._sum_k.value), self._bins.copy(), self._load.copy(), n_layers, rank_k,
+                        elems, off, self.plan_h)
 
     # -- the whole step for all simulated ranks ---------------------------------------------
     def step(self, resid: torch.Tensor, grad: Optional[torch.Tensor], iteration: int = 0, events=None,

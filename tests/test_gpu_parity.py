@@ -410,6 +410,7 @@ def test_whole_step_in_one_call_matches_the_separate_calls(deft):
         plan_b = ds_b.step_fused(e_b, g_d, iteration=t)              # the same through deft_step
         torch.cuda.synchronize()
         assert plan_a.sum_k == plan_b.sum_k and plan_a.k_l.tolist() == plan_b.k_l.tolist()
+        assert torch.equal(ds_a.norms_d, ds_b.norms_d)                # the step's accumulate pass takes the roots itself: same bits
         assert plan_a.bin_of_layer.tolist() == plan_b.bin_of_layer.tolist()
         assert plan_a.bin_load.tobytes() == plan_b.bin_load.tobytes()
         s = plan_a.sum_k

@@ -579,6 +579,25 @@ def run_ours(args):
     stats1 = deft.deft_select_stats(ds.ws, L)
     layer_stats = {kk: (stats1[kk] - stats0[kk]) % (1 << 32) for kk in stats1}   # streamed layers over the timed steps
 
+    # the selection launch on its own (it reads the vector itself), for the kernel's own roofline when the
+    # timed step stages during the accumulate pass
+    alone = None
+    if staged_step:
+        deft.deft_debug_step_staging(False)
+        al_recs = []
+        s_c = deft.deft_select_stats(ds.ws, L)
+        fresh = torch.empty_like(g)
+        for it in range(8 + 10):
+            W.device_gradient(w, 10_000 + it, dev, out=fresh)   # a draw of its own every step, as in the timed region
+            one_step(args.warmup + args.steps + 64 + it, al_recs if it >= 8 else None, fresh)
+        stream.synchronize()
+        s_d = deft.deft_select_stats(ds.ws, L)
+        deft.deft_debug_step_staging(True)
+        alone = {"sel": np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in al_recs]),
+                 "acc": np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in al_recs]),
+                 "stats": {kk: (s_d[kk] - s_c[kk]) % (1 << 32) for kk in s_d}}
+        del fresh
+
     # a second, non-stationary stream: a pool of 4 draws cycled (the accumulated vector and with it every
     # layer's threshold keep shifting against the norms), same step, same timing
     ns_steps = max(8, min(args.steps, 40))
@@ -600,24 +619,6 @@ def run_ours(args):
     ns_sel = np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in ns_recs])
     ns_stats = {kk: (s_b[kk] - s_a[kk]) % (1 << 32) for kk in s_b}
 
-    # the selection launch on its own (it reads the vector itself), for the kernel's own roofline when the
-    # timed step stages during the accumulate pass
-    alone = None
-    if staged_step:
-        deft.deft_debug_step_staging(False)
-        al_recs = []
-        s_c = deft.deft_select_stats(ds.ws, L)
-        fresh = torch.empty_like(g)
-        for it in range(8 + 10):
-            W.device_gradient(w, 10_000 + it, dev, out=fresh)   # a draw of its own every step, as in the timed region
-            one_step(args.warmup + args.steps + 64 + it, al_recs if it >= 8 else None, fresh)
-        stream.synchronize()
-        s_d = deft.deft_select_stats(ds.ws, L)
-        deft.deft_debug_step_staging(True)
-        alone = {"sel": np.array([r["sel"][0].elapsed_time(r["sel"][1]) for r in al_recs]),
-                 "acc": np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in al_recs]),
-                 "stats": {kk: (s_d[kk] - s_c[kk]) % (1 << 32) for kk in s_d}}
-        del fresh
 
     # per-call statistics from the events recorded inside the timed region
     t_acc = np.array([r["acc"][0].elapsed_time(r["acc"][1]) for r in recs])

@@ -652,3 +652,39 @@ def test_staging_in_the_accumulate_pass_never_changes_the_result(deft):
     finally:
         deft.deft_debug_select_kernel(None)
         deft.deft_debug_step_staging(True)
+
+
+def test_many_steps_staged_and_unstaged_agree(deft):
+    """Sixty steps with the residual carried over, gradients repeated, rescaled and now and then jumping by
+    a factor of 16 or 1/64: the step that stages in its accumulate pass and the step whose selection launch
+    reads the vector itself (alternating between its two ways of reading) must leave the same bytes
+    every time.  (The unstaged step is compared with the oracle elsewhere.)"""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    w = W.scaled_down(W.bert_large(), 16)
+    N = w.n_workers
+    rng = np.random.default_rng(5)
+    try:
+        deft.deft_debug_select_kernel(True)
+        ds_a, ds_b = DeftStep(w.sizes, N, w.density), DeftStep(w.sizes, N, w.density)
+        e_a = torch.zeros(w.n_g, dtype=torch.float32, device="cuda")
+        e_b = torch.zeros_like(e_a)
+        for t in range(60):
+            g = W.device_gradient(w, t % 5 if t % 11 < 4 else 100 + t, "cuda")
+            g.mul_(float(np.exp(rng.normal(0, 0.15))) * (16.0 if t % 17 == 16 else 1.0) * (1 / 64.0 if t % 23 == 22 else 1.0))
+            deft.deft_debug_step_staging(True)
+            deft.deft_debug_select_ring(True)
+            plan_a = ds_a.step_fused(e_a, g, t)
+            deft.deft_debug_step_staging(False)
+            deft.deft_debug_select_ring(t % 2 == 0)
+            plan_b = ds_b.step_fused(e_b, g, t)
+            torch.cuda.synchronize()
+            s = plan_a.sum_k
+            assert plan_a.k_l.tolist() == plan_b.k_l.tolist(), t
+            assert torch.equal(ds_a.idx_d[:s], ds_b.idx_d[:s]) and torch.equal(ds_a.val_d[:s], ds_b.val_d[:s]), t
+            assert torch.equal(e_a, e_b), t
+        st = deft.deft_select_stats(ds_a.ws, ds_a.L)
+        assert st["one_read"] > 0 and st["cut_failed"] > 0 and st["ring_gave_up"] == 0
+    finally:
+        deft.deft_debug_select_kernel(None)
+        deft.deft_debug_step_staging(True)
+        deft.deft_debug_select_ring(True)

@@ -168,4 +168,6 @@ def test_bench_step_with_staging_full_size(deft):
         acc[idx_all] = 0.0
         assert e_d.cpu().numpy().tobytes() == acc.tobytes()
     st = deft.deft_select_stats(ds.ws, ds.L)
-    assert st["one_read"] > before["one_read"] and st["staged_entries"] > 0   # the later steps ran on staged entries
+    import os
+    if os.environ.get("DEFT_SINGLE_PASS") != "0":   # (with the five-step kernel forced there is nothing to stage for)
+        assert st["one_read"] > before["one_read"] and st["staged_entries"] > 0   # the later steps ran on staged entries

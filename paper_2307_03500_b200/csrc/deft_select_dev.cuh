@@ -475,7 +475,7 @@ __device__ __forceinline__ void write_scanned(const uint32_t* tile, uint32_t k0,
 // speculative cut), else the staged entries of bucket b1 are counted in the level-2 histogram h2 (second
 // read).  Returns (first entry, entries).
 constexpr uint32_t kCountStaged = 0xffffffffu;
-template <bool kHist>
+template <bool kHist, bool kMark = true>
 __device__ __forceinline__ uint2 read_tile(const float* acc, const TileSpan& ts, uint32_t* h, uint32_t thr,
                                            const Stage& st, uint32_t ytag, uint32_t* cursor, uint32_t* wbase,
                                            int lane, uint32_t* h2 = nullptr, uint32_t b1 = 0) {
@@ -493,6 +493,7 @@ __device__ __forceinline__ uint2 read_tile(const float* acc, const TileSpan& ts,
         // the components outside the layer were loaded as zeros
         if (lane == 0 && ts.e - ts.s != kTile) atomicSub(&h[0], (uint32_t)(kTile - (ts.e - ts.s)));
     }
+    if (!kMark) return make_uint2(0u, 0u);   // (a pass that only counts: thr is 0xffffffff)
     uint32_t keep[2];
     if (!mark_tile(t, vm, thr, keep)) return make_uint2(0u, 0u);
     auto put = [&](uint32_t pos, uint32_t bits, uint32_t off) {

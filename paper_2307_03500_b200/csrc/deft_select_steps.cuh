@@ -67,17 +67,14 @@ __device__ __noinline__ void step_read1(const SelParams& p, const CtaRange r, La
             if (cl < 0) continue;
             uint32_t* h = hist + (cl - c0) * kBins1;
             const uint32_t thr = lt->sthr[cl];
-            if (round == 1) {
-                if (lt->base_gt[cl]) {
-                    const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-                    read_tile<true>(p.acc, ts, h, 0xffffffffu, st, 0u, misc + kMCursor, wbase + 16 * warp, lane);
-                }
-                continue;
-            }
+            // round 1 reads only the layers whose cut failed, and those in full; round 0 reads a layer without
+            // a cut in full (one place in the code for both: the routine is large)
+            if (round == 1 && !lt->base_gt[cl]) continue;
             uint2 fn = make_uint2(0u, 0u);
-            if (thr == 0xffffffffu) {   // no cut: the full histogram, nothing staged
+            if (round == 1 || thr == 0xffffffffu) {   // the full histogram, nothing staged
                 const TileSpan ts = tile_span(lt->start[cl], lt->end[cl], lt->tf[cl], q);
-                read_tile<true>(p.acc, ts, h, 0xffffffffu, st, 0u, misc + kMCursor, wbase + 16 * warp, lane);
+                read_tile<true, false>(p.acc, ts, h, 0xffffffffu, st, 0u, misc + kMCursor, wbase + 16 * warp, lane);
+                if (round == 1) continue;
             } else if (*reinterpret_cast<volatile uint32_t*>(misc + kMCursor) > budget) {
                 // a cut that turns out far too low must not flood the staging area: past the budget the CTA
                 // stops staging; the layers it skips tiles of count as failed

@@ -310,7 +310,6 @@ __device__ __forceinline__ uint2 stage_get(const Stage& st, uint32_t pos) {
 // HBM round trip per entry.
 constexpr int kSpillBatch = 8;
 constexpr int kEmitBatch = 4;
-constexpr uint32_t kThreadEmit = 12;   // tiles with at most this many staged entries are written by one thread
 
 template <typename F>
 __device__ __forceinline__ void for_each_staged(const Stage& st, uint32_t total, F f) {
@@ -850,10 +849,17 @@ __device__ __forceinline__ int grab_tile(uint32_t* counter, int lane) {
 }
 
 
-// Ordered write of one batch of 32 consecutive staged entries (one per lane).  gt_before /
-// eq_before: entries above / equal to the threshold that precede the batch in the layer.
+// ---- the ordered write, by staged entry ----
+// A CTA's staged entries lie tile by tile (a tile's entries consecutive and in index order; the tiles in the
+// order the warps got to them).  Every warp walks a contiguous range of them, 32 consecutive entries per
+// step: an entry's place in the output is (entries of its layer above / equal to T in earlier tiles: pg / pe
+// of its tile) + (such entries before it in its own tile), and the second term follows from ballots over the
+// run of lanes that hold the same tile, plus what the warp carries over when a tile's entries began in an
+// earlier step.  Cost follows the entries a CTA holds, not its tiles.
 struct EmitOut { float* val; int64_t* idx; float* acc_rw; int64_t cap; };
 
+// Ordered write of one batch of 32 consecutive entries of ONE layer (one per lane; the small-layer path).
+// gt_before / eq_before: entries above / equal to the threshold that precede the batch in the layer.
 __device__ __forceinline__ void emit_batch(const EmitOut& p, int64_t out_off, int64_t elem0, bool valid,
                                            uint32_t bits, int64_t off, uint32_t T, uint32_t need,
                                            uint32_t& gt_before, uint32_t& eq_before, int lane) {
@@ -875,78 +881,72 @@ __device__ __forceinline__ void emit_batch(const EmitOut& p, int64_t out_off, in
     eq_before += __popc(eq_b);
 }
 
-// One batch of local tiles [t0, tend): pref[lq - t0] = entries above / equal to T that precede
-// tile lq in its layer.  One warp per tile writes the tile's selected entries.
-__device__ __noinline__ void emit_tiles(EmitOut out, int tiles, int il, int q0, const TileTable* tt, Stage st,
-                                        const uint2* pref, int t0, int tend, int64_t start, int tf,
-                                        int64_t out_off, uint32_t T, uint32_t need) {
+__device__ __forceinline__ void emit_entries(const SelParams& p, const CtaRange& r, const LayerTable* lt, const TileTable* tt,
+                                             const Stage& st, const uint32_t* pg, const uint32_t* pe, uint32_t total) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // the warp's next tile that needs a warp: (lq, q) advance, false when there is none
-    int lq = t0 + warp - kSelWarps, q = 0;
-    auto next_tile = [&]() {
-        for (lq += kSelWarps; lq < tend; lq += kSelWarps) {
-            q = q0 + lq;
-            if (il) {
-                q = kSuper * ((int)blockIdx.x + (lq / kSuper) * (int)gridDim.x) + lq % kSuper;
-                if (q >= tiles) continue;
-            }
-            if (tt->n[lq] > kThreadEmit) return true;   // the others: nothing staged, or written by their own thread
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const uint32_t per = ((total + kSelWarps - 1) / kSelWarps + 31u) & ~31u;
+    const uint32_t w_lo = (uint32_t)warp * per < total ? (uint32_t)warp * per : total;
+    const uint32_t w_hi = w_lo + per < total ? w_lo + per : total;
+    if (w_lo >= w_hi) return;
+    // what the warp carries: the tile of the last entry seen and that tile's entries above / equal to T so far
+    uint32_t carry_tile = 0xffffffffu, cg = 0, ce = 0;
+    {
+        const uint2 e0 = stage_get(st, w_lo);
+        const uint32_t ti = y_tile(e0.y), c = y_layer(e0.y);
+        const uint32_t first = tt->first[ti], T = lt->v0[c];
+        carry_tile = ti;
+        for (uint32_t pos = first + lane; pos < w_lo; pos += 32) {   // the part of the tile that lies in the range before
+            const uint32_t key = key_of(stage_get(st, pos).x);
+            cg += key > T ? 1u : 0u;
+            ce += key == T ? 1u : 0u;
         }
-        return false;
-    };
-    auto load_round = [&](uint32_t first, uint32_t n, uint32_t e0, uint2 (&ent)[kEmitBatch]) {
+        cg = __reduce_add_sync(0xffffffffu, cg);
+        ce = __reduce_add_sync(0xffffffffu, ce);
+    }
+    for (uint32_t p4 = w_lo; p4 < w_hi; p4 += 32 * kEmitBatch) {   // kEmitBatch steps' entries are fetched together
+        uint2 ent[kEmitBatch];
 #pragma unroll
         for (int u = 0; u < kEmitBatch; ++u) {
-            const uint32_t e = e0 + u * 32 + lane;
-            ent[u] = e < n ? stage_get(st, first + e) : make_uint2(0u, 0u);
-        }
-    };
-    bool have = next_tile();
-    uint2 ent[kEmitBatch];
-    if (have) load_round(tt->first[lq], tt->n[lq], 0u, ent);
-    while (have) {
-        const int lq_cur = lq;
-        const uint32_t n = tt->n[lq_cur], first = tt->first[lq_cur];
-        const int64_t lo = (start / kTile + (q - tf)) * kTile;
-        uint32_t gt_before = pref[lq_cur - t0].x, eq_before = pref[lq_cur - t0].y;
-        // the first round of the warp's next tile is in flight while this tile is written
-        have = next_tile();
-        uint2 ent_next[kEmitBatch];
-        if (have) load_round(tt->first[lq], tt->n[lq], 0u, ent_next);
-        for (uint32_t e0 = 0; e0 < n; e0 += 32 * kEmitBatch) {
-            if (e0) load_round(first, n, e0, ent);
-#pragma unroll
-            for (int u = 0; u < kEmitBatch; ++u) {
-                if (e0 + u * 32 < n)   // uniform over the warp
-                    emit_batch(out, out_off, lo, e0 + u * 32 + lane < n, ent[u].x, (int64_t)y_off(ent[u].y), T, need,
-                               gt_before, eq_before, lane);
-            }
+            const uint32_t pos = p4 + u * 32 + lane;
+            ent[u] = pos < w_hi ? stage_get(st, pos) : make_uint2(0u, 0u);
         }
 #pragma unroll
-        for (int u = 0; u < kEmitBatch; ++u) ent[u] = ent_next[u];
-    }
-}
-
-// Tiles with at most kThreadEmit staged entries are written by ONE thread each (thread i of a
-// batch owns tile t0 + i, whose prefix it has just computed): at a few entries per tile a warp
-// per tile leaves most lanes idle and is bound by its own instruction latency.
-__device__ __forceinline__ void emit_small_tile(const EmitOut& out, const Stage& st, uint32_t first, uint32_t n,
-                                                int64_t out_off, int64_t lo, uint32_t T, uint32_t need,
-                                                uint32_t gt_before, uint32_t eq_before) {
-    for (uint32_t e = 0; e < n; ++e) {
-        const uint2 ent = stage_get(st, first + e);
-        const uint32_t key = key_of(ent.x);
-        if (key > T || (key == T && eq_before < need)) {
-            const int64_t pos = out_off + gt_before + (eq_before < need ? eq_before : need);
-            const int64_t elem = lo + (int64_t)y_off(ent.y);
-            if (pos < out.cap) {
-                out.val[pos] = __uint_as_float(ent.x);
-                out.idx[pos] = elem;
+        for (int u = 0; u < kEmitBatch; ++u) {
+            if (p4 + u * 32 >= w_hi) break;   // uniform over the warp
+            const bool valid = p4 + u * 32 + lane < w_hi;
+            const uint32_t y = ent[u].y, bits = ent[u].x;
+            const uint32_t ti = valid ? y_tile(y) : 0xffffffffu, c = y_layer(y);
+            const uint32_t T = valid ? lt->v0[c] : 0u, need = valid ? lt->v1[c] : 0u;
+            const uint32_t key = key_of(bits);
+            const bool gt = valid && key > T, eq = valid && key == T;
+            const unsigned gtb = __ballot_sync(0xffffffffu, gt), eqb = __ballot_sync(0xffffffffu, eq);
+            const uint32_t tprev = __shfl_up_sync(0xffffffffu, ti, 1);
+            const unsigned sb = __ballot_sync(0xffffffffu, lane == 0 || ti != tprev);   // lanes at which a tile's run begins
+            const int s0 = 31 - __clz((int)(sb & (lt_mask | (1u << lane))));              // where my tile's run begins
+            const uint32_t run_before = lt_mask & ~((1u << s0) - 1u);
+            const bool carried = s0 == 0 && ti == carry_tile;
+            const uint32_t my_gt = (valid ? pg[ti] : 0u) + __popc(gtb & run_before) + (carried ? cg : 0u);
+            const uint32_t my_eq = (valid ? pe[ti] : 0u) + __popc(eqb & run_before) + (carried ? ce : 0u);
+            if (gt || (eq && my_eq < need)) {
+                // selected entries of the layer before me: every larger key, and the first `need` equal ones
+                const int q = local_tile(p, r, (int)ti);
+                const int64_t elem = (lt->start[c] / kTile + (q - lt->tf[c])) * kTile + (int64_t)y_off(y);
+                const int64_t pos = lt->out_off[c] + my_gt + (my_eq < need ? my_eq : need);
+                if (pos < p.out_cap) {
+                    p.val[pos] = __uint_as_float(bits);
+                    p.idx[pos] = elem;
+                }
+                if (p.acc_rw) p.acc_rw[elem] = 0.0f;
             }
-            if (out.acc_rw) out.acc_rw[elem] = 0.0f;
+            // carry: the run that reaches the step's last lane
+            const uint32_t t_last = __shfl_sync(0xffffffffu, ti, 31);
+            const int s_last = 31 - __clz((int)sb);
+            const uint32_t run_last = ~((1u << s_last) - 1u);
+            const uint32_t g_last = __popc(gtb & run_last), e_last = __popc(eqb & run_last);
+            if (s_last == 0 && t_last == carry_tile) { cg += g_last; ce += e_last; }
+            else { carry_tile = t_last; cg = g_last; ce = e_last; }
         }
-        gt_before += key > T;
-        eq_before += key == T;
     }
 }
 

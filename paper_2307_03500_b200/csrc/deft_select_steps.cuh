@@ -346,11 +346,14 @@ __device__ __forceinline__ void step_count(const SelParams& p, const CtaRange& r
 __device__ __noinline__ void step_emit(const SelParams& p, const CtaRange r, LayerTable* lt, int nl,
                                        const TileTable* tt, const Stage st, unsigned char* smem) {
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + kSmMisc);
-    uint2* pref = reinterpret_cast<uint2*>(smem + kSmPref);
     uint32_t* scratch = misc + kMScratch;
+    // per local tile: entries above / equal to T that precede the tile in its layer (the histograms' room is free)
+    uint32_t* pg = reinterpret_cast<uint32_t*>(smem + kSmMain);
+    uint32_t* pe = pg + kMaxLocalTiles;
+    static_assert(2 * kMaxLocalTiles * 4 <= kSlots * kBins1 * 4, "tile prefixes fit the histogram slots");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (nl == 0) return;
     if (r.il) {
-        if (nl == 0) return;
         // Prefix at each own super-tile b + mG: the totals of all super-tiles are summed in
         // windows [b + (m-1)G, b + mG) (window 0 = [0, b)), one warp per window, then scanned.
         uint2* sbase = reinterpret_cast<uint2*>(smem + kSmSuper);
@@ -372,7 +375,6 @@ __device__ __noinline__ void step_emit(const SelParams& p, const CtaRange r, Lay
             if ((int)threadIdx.x < nm) sbase[threadIdx.x] = make_uint2(e_gt + w.x, e_eq + w.y);
         }
         __syncthreads();
-        const uint32_t T = lt->v0[0], need = lt->v1[0];
         for (int t0 = 0; t0 < r.nloc; t0 += kSelThreads) {
             const int i = t0 + (int)threadIdx.x;
             const uint32_t v = i < r.nloc ? tt->ge[i] : 0u;   // counts <= kTile each: 16 of them fit 16 bits
@@ -383,71 +385,49 @@ __device__ __noinline__ void step_emit(const SelParams& p, const CtaRange r, Lay
                 if ((lane & (kSuper - 1)) >= o) incl += x;
             }
             const uint32_t ex = incl - v;
-            const uint2 sb = i < r.nloc ? sbase[i / kSuper] : make_uint2(0u, 0u);
-            pref[threadIdx.x] = make_uint2(sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
-            bool big = false;
-            {
-                const int q = i < r.nloc ? local_tile(p, r, i) : -1;
-                const uint32_t n = q >= 0 ? tt->n[i] : 0u;
-                if (n != 0 && n <= kThreadEmit)
-                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, st, tt->first[i], n, lt->out_off[0],
-                                    (lt->start[0] / kTile + (q - lt->tf[0])) * kTile, T, need,
-                                    sb.x + (ex & 0xffffu), sb.y + (ex >> 16));
-                big = n > kThreadEmit;
-            }
-            const int tend = t0 + kSelThreads < r.nloc ? t0 + kSelThreads : r.nloc;
-            if (__syncthreads_or(big ? 1 : 0))   // some tile of the batch needs a warp
-                emit_tiles(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, p.tiles, 1, 0, tt, st, pref, t0, tend, lt->start[0],
-                       lt->tf[0], lt->out_off[0], T, need);
-            __syncthreads();   // pref is rewritten by the next batch
-        }
-        return;
-    }
-    for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of earlier CTAs
-        const int j = lt->j[c];
-        uint32_t gt = 0, eq = 0;
-        for (int b = split_cta_of_tile(p, r, lt->tf[c]) + lane; b < (int)blockIdx.x; b += 32) {
-            if (split_q0(p, r, b) < split_q0(p, r, b + 1)) {
-                const uint2 v = __ldcg(p.runge + b + j);
-                gt += v.x;
-                eq += v.y;
+            if (i < r.nloc) {
+                const uint2 sb = sbase[i / kSuper];
+                pg[i] = sb.x + (ex & 0xffffu);
+                pe[i] = sb.y + (ex >> 16);
             }
         }
-        gt = __reduce_add_sync(0xffffffffu, gt);
-        eq = __reduce_add_sync(0xffffffffu, eq);
-        if (lane == 0) { lt->base_gt[c] = gt; lt->base_eq[c] = eq; }
+    } else {
+        for (int c = warp; c < nl; c += kSelWarps) {   // one warp per layer: totals of earlier CTAs
+            const int j = lt->j[c];
+            uint32_t gt = 0, eq = 0;
+            for (int b = split_cta_of_tile(p, r, lt->tf[c]) + lane; b < (int)blockIdx.x; b += 32) {
+                if (split_q0(p, r, b) < split_q0(p, r, b + 1)) {
+                    const uint2 v = __ldcg(p.runge + b + j);
+                    gt += v.x;
+                    eq += v.y;
+                }
+            }
+            gt = __reduce_add_sync(0xffffffffu, gt);
+            eq = __reduce_add_sync(0xffffffffu, eq);
+            if (lane == 0) { lt->base_gt[c] = gt; lt->base_eq[c] = eq; }
+        }
+        __syncthreads();
+        for (int c = 0; c < nl; ++c) {
+            int ta, tb;
+            local_span(r, lt, c, c, ta, tb);
+            uint32_t base_gt = lt->base_gt[c], base_eq = lt->base_eq[c];
+            for (int t0 = ta; t0 < tb; t0 += kSelThreads) {   // batches of kSelThreads tiles
+                const int i = t0 + (int)threadIdx.x;
+                const uint32_t v = i < tb ? tt->ge[i] : 0u;
+                uint32_t tot_gt, tot_eq;
+                const uint32_t e_gt = block_excl_scan(v & 0xffffu, scratch, tot_gt);
+                const uint32_t e_eq = block_excl_scan(v >> 16, scratch, tot_eq);
+                if (i < tb) {
+                    pg[i] = base_gt + e_gt;
+                    pe[i] = base_eq + e_eq;
+                }
+                base_gt += tot_gt;
+                base_eq += tot_eq;
+            }
+        }
     }
     __syncthreads();
-    for (int c = 0; c < nl; ++c) {
-        int ta, tb;
-        local_span(r, lt, c, c, ta, tb);
-        const uint32_t T = lt->v0[c], need = lt->v1[c];
-        uint32_t base_gt = lt->base_gt[c], base_eq = lt->base_eq[c];
-        for (int t0 = ta; t0 < tb; t0 += kSelThreads) {   // batches of kSelThreads tiles
-            const int i = t0 + (int)threadIdx.x;
-            const uint32_t v = i < tb ? tt->ge[i] : 0u;
-            uint32_t tot_gt, tot_eq;
-            const uint32_t e_gt = block_excl_scan(v & 0xffffu, scratch, tot_gt);
-            const uint32_t e_eq = block_excl_scan(v >> 16, scratch, tot_eq);
-            pref[threadIdx.x] = make_uint2(base_gt + e_gt, base_eq + e_eq);
-            bool big = false;
-            {
-                const uint32_t n = i < tb ? tt->n[i] : 0u;
-                if (n != 0 && n <= kThreadEmit)
-                    emit_small_tile(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, st, tt->first[i], n, lt->out_off[c],
-                                    (lt->start[c] / kTile + (r.q0 + i - lt->tf[c])) * kTile, T, need,
-                                    base_gt + e_gt, base_eq + e_eq);
-                big = n > kThreadEmit;
-            }
-            const int tend = t0 + kSelThreads < tb ? t0 + kSelThreads : tb;
-            if (__syncthreads_or(big ? 1 : 0))   // some tile of the batch needs a warp
-                emit_tiles(EmitOut{p.val, p.idx, p.acc_rw, p.out_cap}, p.tiles, 0, r.q0, tt, st, pref, t0, tend, lt->start[c],
-                       lt->tf[c], lt->out_off[c], T, need);
-            base_gt += tot_gt;
-            base_eq += tot_eq;
-            __syncthreads();   // pref is rewritten by the next batch
-        }
-    }
+    emit_entries(p, r, lt, tt, st, pg, pe, misc[kMCursor]);
 }
 
 

@@ -526,6 +526,32 @@ def test_every_form_of_the_selection_kernel_gives_the_same_bits(deft):
     assert size.sum() == w.n_g
 
 
+@pytest.mark.parametrize("density", [0.03, 0.2])
+def test_whole_step_with_layers_the_staging_pass_cannot_serve(deft, density):
+    """Two layers that select more entries each than one CTA finishes behind the staging accumulate pass
+    (density 0.03), or that are too dense for a cut at all (0.2): the step drops what was staged, or stages
+    nothing, and selects the ordinary way.  Three steps against the oracle."""
+    from paper_2307_03500_b200.pipeline import DeftStep
+    sizes = [3_000_000, 2_500_001]
+    ds = DeftStep(sizes, 1, density)
+    n = int(sum(sizes))
+    e = torch.zeros(n, dtype=torch.float32, device="cuda")
+    acc = np.zeros(n, dtype=np.float32)
+    start = np.asarray(ds.layer_start)
+    for t in range(3):
+        g = W.adversarial_vector("gauss", n, seed=70 + t)
+        plan = ds.step_fused(e, _dev(g), iteration=t)
+        torch.cuda.synchronize()
+        oracle.accumulate(acc, g)
+        k_l, _ = oracle.allocate_k(oracle.layer_norms(acc, start), np.diff(start), ds.k, oracle.MODE_EXACT)
+        assert plan.k_l.tolist() == k_l.tolist()
+        want_val, want_idx = oracle.select_rank(acc, start, k_l, np.arange(len(sizes), dtype=np.int32))
+        assert np.array_equal(ds.idx_d[:plan.sum_k].cpu().numpy(), want_idx)
+        assert ds.val_d[:plan.sum_k].cpu().numpy().tobytes() == want_val.tobytes()
+        acc[want_idx] = 0.0
+        assert e.cpu().numpy().tobytes() == acc.tobytes()
+
+
 @pytest.mark.parametrize("L", [1, 2, 3, 4])
 def test_few_large_layers_keep_their_remembered_cuts_across_the_norms_pass(deft, L):
     """The norms pass and the selection share one workspace.  With one to four layers of a few million
